@@ -1,0 +1,221 @@
+/*
+ * il_estimator.h -- C ABI of the batched InferLine Estimator for NVIDIA B200 (sm_100a).
+ *
+ * The Estimator (InferLine, arXiv 1812.01776, Section 4.2) is a discrete-event
+ * simulation: given a pipeline configuration, the per-model profiles and a
+ * sample arrival trace it replays the trace through the pipeline, queueing
+ * included, and yields the latency of every query.  The Planner (Section 4.3,
+ * Algorithms 1 and 2) asks it one question per candidate configuration --
+ * "does this configuration meet the latency objective at P99?" (Feasible) --
+ * and asks it for many candidates against the same profiles and trace.  This
+ * library answers that question for a whole batch of candidates per call:
+ * profiles and trace are bound once (create), candidates are evaluated many
+ * times (estimate).
+ *
+ * Simulated system (Section 3: centralized batched queue; Section 2.1: batches
+ * complete as a whole; configuration = per model a hardware type, a maximum
+ * batch size and a replication factor):
+ *   - every stage has one FIFO queue and R identical replicas;
+ *   - a replica that is idle while the queue is non-empty takes
+ *     min(queue length, max batch) queries from the front at once (the
+ *     lowest-id idle replica first) and is busy for
+ *     latency_us[stage][hw][b-1] microseconds, b being the batch it took;
+ *   - all queries of the batch leave the stage together; each follows the one
+ *     child edge whose condition its branch bits satisfy, with zero delay, in
+ *     batch order; a query with no such edge leaves the pipeline and its
+ *     latency is that instant minus its arrival time;
+ *   - everything at one timestamp happens as: all completions (batches
+ *     dispatched earlier first), then all trace arrivals (in trace order), then
+ *     dispatching;
+ *   - per candidate the result is the k-th smallest latency, k = ceil(0.99 n)
+ *     = (99 n + 99) / 100 in integers (Section 2: P99 objective), and the
+ *     number of queries with latency > slo_us.
+ * All times are int64 microseconds.  Results are exact integers; there is no
+ * floating point on the path.
+ *
+ * There is no CPU fallback: every entry point that computes needs a CUDA
+ * device of compute capability 10.x and fails with IL_ERR_CUDA otherwise.
+ *
+ * Threading: calls on ONE handle must not overlap.  Different handles may be
+ * used from different threads.  Unless said otherwise a call returns after all
+ * work it enqueued has completed.
+ */
+#ifndef IL_ESTIMATOR_H
+#define IL_ESTIMATOR_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define IL_API __attribute__((visibility("default")))
+#else
+#define IL_API
+#endif
+
+#define IL_MAX_STAGES     16
+#define IL_MAX_HW          8
+#define IL_MAX_BATCH      64
+#define IL_MAX_REPLICAS   32
+
+/* Return codes.  0 is success; on any error no output element is defined. */
+#define IL_OK                 0
+#define IL_ERR_INVALID_ARG   -1  /* NULL pointer, n < 0, sizes out of the limits above      */
+#define IL_ERR_BAD_TOPOLOGY  -2  /* not a tree in the accepted form (see il_profiles)      */
+#define IL_ERR_BAD_PROFILE   -3  /* a latency table entry < 1                              */
+#define IL_ERR_BAD_TRACE     -4  /* arrival times negative, decreasing, or too large       */
+#define IL_ERR_BAD_CONFIG    -5  /* a candidate with hw >= H, max_batch or replicas out of range */
+#define IL_ERR_NOMEM         -6  /* host or device allocation failed / workspace too small */
+#define IL_ERR_CUDA          -7  /* a CUDA runtime call failed; see il_last_cuda_error     */
+#define IL_ERR_ITER_LIMIT    -8  /* a device loop hit its iteration bound (internal error) */
+
+typedef struct il_estimator il_estimator;   /* opaque; owns its device copies */
+
+/*
+ * Pipeline shape and model profiles (Section 4.1: a profile gives, per
+ * hardware type and batch size, how long the model takes for that batch).
+ * All pointers are HOST pointers, read during il_estimator_create only.
+ *
+ * The pipeline is a tree.  Stage 0 is the root, parent[s] < s.  The edge
+ * parent[s] -> s is taken by query q iff cond_bit[s] < 0, or
+ * ((branch_bits[q] >> cond_bit[s]) & 1) == cond_val[s].  The children of one
+ * stage must be either a single unconditional child, or one or two children
+ * guarded by the SAME bit with different values; so a query follows at most
+ * one edge, and a guarded edge without sibling is a cascade (the other queries
+ * leave the pipeline there).
+ */
+typedef struct {
+    int32_t        n_stages;    /* S, 1..IL_MAX_STAGES                                  */
+    int32_t        n_hw;        /* H, 1..IL_MAX_HW                                      */
+    int32_t        max_batch;   /* Bmax, 1..IL_MAX_BATCH; tables are dense in b = 1..Bmax */
+    const int32_t *parent;      /* [S], parent[0] = -1                                  */
+    const int8_t  *cond_bit;    /* [S], -1 or 0..7                                      */
+    const uint8_t *cond_val;    /* [S], 0 or 1 (ignored where cond_bit < 0)             */
+    const int32_t *latency_us;  /* [S][H][Bmax] row-major, every entry >= 1             */
+} il_profiles;
+
+/*
+ * The sample arrival trace (Section 3: provided by the developer; Section 4.2:
+ * input of the Estimator).  HOST pointers, copied by il_estimator_create.
+ */
+typedef struct {
+    int64_t        n_queries;   /* n, 1 .. 2^31 - 1                                     */
+    const int64_t *arrival_us;  /* [n], >= 0 and non-decreasing; equal stamps keep trace order */
+    const uint8_t *branch_bits; /* [n]; may be NULL when no stage has cond_bit >= 0     */
+} il_trace;
+
+/* One stage of one candidate configuration (Section 2.1: hardware type,
+ * maximum batch size, replication factor).  A candidate is S of these in a
+ * row; a batch of candidates is an array [n_candidates][S]. */
+typedef struct {
+    uint8_t hw;         /* 0 .. H-1                     */
+    uint8_t max_batch;  /* 1 .. Bmax                    */
+    uint8_t replicas;   /* 1 .. IL_MAX_REPLICAS         */
+    uint8_t reserved;   /* ignored                      */
+} il_stage_config;
+
+/* Counters of the most recent il_estimate / il_estimate_device call. */
+typedef struct {
+    int64_t candidates;      /* candidates evaluated                                     */
+    int64_t query_events;    /* candidates * sum over stages of queries visiting the stage */
+    int64_t batches;         /* batches dispatched, all candidates, all stages           */
+    int64_t chunks;          /* how many (simulate, select) launch pairs the call made   */
+    int64_t kernel_launches; /* kernels launched by the call                             */
+    double  sim_ms;          /* device time of the simulation kernels (CUDA events)      */
+    double  select_ms;       /* device time of the percentile kernels (CUDA events)      */
+    double  total_ms;        /* device time of all stream work of the call               */
+} il_stats;
+
+/*
+ * Binds profiles and trace (Section 4.2: the Estimator's fixed inputs) on the
+ * current CUDA device: validates them, copies them to device memory, and
+ * precomputes from the branch bits how many queries visit each stage.
+ *   profiles, trace   host structs with host pointers (see above)
+ *   out               receives the handle; untouched on error
+ * Errors: INVALID_ARG, BAD_TOPOLOGY, BAD_PROFILE, BAD_TRACE (also when
+ * last arrival + (sum over stages of n * largest table entry) would not fit in
+ * 62 bits), NOMEM, CUDA.
+ */
+IL_API int il_estimator_create(const il_profiles *profiles, const il_trace *trace, il_estimator **out);
+
+/* Frees the handle and everything the library allocated for it.  Memory given
+ * through il_set_workspace stays the caller's.  NULL is allowed. */
+IL_API void il_estimator_destroy(il_estimator *est);
+
+/*
+ * Evaluates n candidate configurations against the bound profiles and trace
+ * (Section 4.2 run once per candidate; Section 4.3 "Feasible" is
+ * out_p99_us[c] <= slo_us, equivalently out_miss[c] <= n_queries - k).
+ *   configs      HOST pointer, [n][S] il_stage_config
+ *   n            number of candidates, >= 0 (0 is a no-op)
+ *   slo_us       latency objective for the miss count
+ *   out_p99_us   HOST pointer, [n]: k-th smallest latency of candidate c
+ *   out_miss     HOST pointer, [n]: number of queries with latency > slo_us
+ * Candidates are validated on the host before anything is launched
+ * (BAD_CONFIG names no index; nothing is written).  Copies to and from the
+ * device happen inside the call, on the handle's stream.
+ */
+IL_API int il_estimate(il_estimator *est, const il_stage_config *configs, int64_t n, int64_t slo_us,
+                       int64_t *out_p99_us, int64_t *out_miss);
+
+/*
+ * Same computation with DEVICE pointers (memory of the handle's device, e.g.
+ * owned by a torch tensor): configs [n][S], out_p99_us [n], out_miss [n].
+ * Work is enqueued on the handle's stream and the call waits for it.
+ * Candidates are validated on the device; an invalid one makes the call return
+ * BAD_CONFIG after the stream has drained, and outputs are then undefined.
+ */
+IL_API int il_estimate_device(il_estimator *est, const il_stage_config *d_configs, int64_t n,
+                              int64_t slo_us, int64_t *d_out_p99_us, int64_t *d_out_miss);
+
+/* Stream all later calls on this handle use (a cudaStream_t passed as void*;
+ * NULL = the default stream).  The stream stays the caller's. */
+IL_API int il_set_stream(il_estimator *est, void *cuda_stream);
+
+/*
+ * Scratch memory.  The simulation keeps, per resident warp, the streams of
+ * (time, query) pairs that flow between stages, and per candidate of a chunk
+ * its n latencies for the percentile kernel.
+ *   il_workspace_bytes  size that lets a call of n_candidates run at full
+ *                       occupancy (for large n_candidates: the size beyond
+ *                       which more memory no longer helps)
+ *   il_workspace_min_bytes  smallest size il_set_workspace accepts
+ *   il_set_workspace    hands the library a DEVICE buffer (256-byte aligned) of
+ *                       the given size; it stays the caller's and must outlive
+ *                       its use.  NULL/0 returns to library-owned scratch.
+ * Without il_set_workspace the library allocates its own scratch with
+ * cudaMalloc on first use (at most il_workspace_bytes, less if the device is
+ * short of memory) and keeps it until destroy.
+ */
+IL_API int il_workspace_bytes(const il_estimator *est, int64_t n_candidates, size_t *bytes);
+IL_API int il_workspace_min_bytes(const il_estimator *est, size_t *bytes);
+IL_API int il_set_workspace(il_estimator *est, void *d_workspace, size_t bytes);
+
+/* Counters of the last estimate call on this handle. */
+IL_API int il_get_stats(const il_estimator *est, il_stats *out);
+
+/* Queries visiting stage s (n_s), derived from the branch bits at create;
+ * out_visits is a HOST pointer to S int64. */
+IL_API int il_stage_visits(const il_estimator *est, int64_t *out_visits);
+
+/* Text for a return code; never NULL. */
+IL_API const char *il_strerror(int code);
+
+/* cudaError_t value of the last failing CUDA call in this thread (0 if none). */
+IL_API int il_last_cuda_error(void);
+
+/*
+ * Measures how many warp-instructions per second the device issues on a
+ * dependency-free 32-bit integer stream (every SM, every scheduler busy): the
+ * denominator for the simulation kernel's instruction-issue roofline.  Runs a
+ * few milliseconds on the current device.  out_* are HOST pointers.
+ */
+IL_API int il_measure_int_issue(void *cuda_stream, double *out_warp_inst_per_s, double *out_ms);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IL_ESTIMATOR_H */

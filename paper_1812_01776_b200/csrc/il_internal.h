@@ -1,0 +1,55 @@
+// Internal declarations shared by the host API and the kernels of the batched
+// Estimator.  Nothing here is part of the C ABI.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include "il_estimator.h"
+
+namespace il {
+
+constexpr int kWarpsPerCta = 4;
+constexpr int kSelectThreads = 256;
+
+// Everything the simulation kernel needs, passed by value as a kernel parameter.
+struct DesParams {
+    // bound inputs (device)
+    const int64_t *arrival;       // [n]
+    const uint8_t *bits;          // [n]
+    const int32_t *lat;           // [S][H][Bmax]
+    int32_t S, H, Bmax;
+    int32_t n;                    // queries
+    int32_t n_s[IL_MAX_STAGES];   // queries visiting stage s
+    int32_t buf_off[IL_MAX_STAGES];  // element offset of stage s's input stream inside a warp slot
+    int8_t  dest_a[IL_MAX_STAGES];   // next stage for branch bit 0 (or unconditional); -1 = leave
+    int8_t  dest_b[IL_MAX_STAGES];   // next stage for branch bit 1; -1 = leave
+    int8_t  bit[IL_MAX_STAGES];      // branch bit tested after stage s, -1 = none
+    // this launch
+    const il_stage_config *configs;  // [n_cand][S], already offset to the chunk
+    int64_t n_cand;
+    int64_t slot_elems;           // stream elements per warp slot
+    int64_t *ws_time;             // [slots][slot_elems]
+    int32_t *ws_qid;              // [slots][slot_elems]
+    int64_t *slab;                // [n_cand][slab_stride] exit latencies
+    int64_t slab_stride;          // n rounded up to 32
+    uint64_t *lat_or;             // [n_cand] OR of all latencies of the candidate
+    unsigned long long *counters; // [0] next candidate, [1] batches dispatched
+    int *status;                  // first error seen by any warp (0 = none)
+};
+
+struct SelectParams {
+    const int64_t *slab;          // [n_cand][slab_stride]
+    int64_t slab_stride;
+    const uint64_t *lat_or;       // [n_cand]
+    int32_t n;
+    int64_t n_cand;
+    int64_t slo_us;
+    int64_t *out_p99;             // [n_cand], already offset to the chunk
+    int64_t *out_miss;
+};
+
+cudaError_t launch_des(const DesParams &p, int grid, size_t smem, cudaStream_t stream);
+cudaError_t launch_select(const SelectParams &p, cudaStream_t stream);
+int des_max_ctas_per_sm(size_t smem);
+cudaError_t launch_int_issue(unsigned *sink, int grid, int iters, cudaStream_t stream);
+
+}  // namespace il
