@@ -1,0 +1,263 @@
+// Batched discrete-event simulation of the InferLine Estimator (Section 4.2),
+// one candidate configuration per warp.
+//
+// Formulation.  The pipeline is a feed-forward tree with zero delay between
+// stages and no back-pressure, so the arrival stream of a stage is fully
+// determined by the completion stream of its parent.  A warp therefore
+// simulates its candidate stage by stage: it turns the sorted stream of
+// (time, query) arrivals of stage s into the sorted stream of completions,
+// which is split by the branch bits into the arrival streams of the children
+// (or into exit latencies).  Within one stage the centralized batched queue
+// (Section 3) is a FIFO, so the queue is always a window [head, tail) of the
+// arrival stream, and one step of the simulation is one batch:
+//
+//     t      = max(earliest time a replica is free, arrival[head])
+//     b      = min(max batch, number of arrivals from head on with time <= t)
+//     finish = t + latency[stage][hw][b-1]            (Section 4.1 profile)
+//
+// Replicas are identical, so only the multiset of their free times matters:
+// lane r of the warp holds replica r's finish time, the replica with the
+// smallest (finish, dispatch order) is the one that is reused, and the batch it
+// held is emitted to the next stage at that moment.  Because every later batch
+// finishes strictly after the current dispatch time, batches are emitted in
+// (finish, dispatch order) order, which is the order in which the next stage's
+// queue sees them; batch-mates keep their order.
+#include "il_internal.h"
+
+namespace il {
+
+namespace {
+
+constexpr int64_t kNever = INT64_MAX;
+
+__device__ __forceinline__ int64_t warp_min_i64(int64_t v)
+{
+    // Times are non-negative or -1; compare as (hi signed, lo unsigned).
+    const int32_t hi = (int32_t)(v >> 32);
+    const int32_t mhi = __reduce_min_sync(0xffffffffu, hi);
+    const uint32_t lo = (hi == mhi) ? (uint32_t)v : 0xffffffffu;
+    const uint32_t mlo = __reduce_min_sync(0xffffffffu, lo);
+    return (int64_t)(((uint64_t)(uint32_t)mhi << 32) | (uint64_t)mlo);
+}
+
+// Where one stage's completions go.
+struct Route {
+    int64_t *a_time; int32_t *a_qid; int32_t a_tail;   // branch bit 0 / unconditional
+    int64_t *b_time; int32_t *b_qid; int32_t b_tail;   // branch bit 1
+    int bit;                                           // -1: no test
+    bool a_exit, b_exit;
+};
+
+}  // namespace
+
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+des_kernel(const __grid_constant__ DesParams p)
+{
+    extern __shared__ int32_t s_lat[];
+    const int n_tab = p.S * p.H * p.Bmax;
+    for (int i = threadIdx.x; i < n_tab; i += blockDim.x) s_lat[i] = p.lat[i];
+    __syncthreads();
+
+    const unsigned full = 0xffffffffu;
+    const int lane = threadIdx.x & 31;
+    const unsigned lt_mask = (1u << lane) - 1u;
+    const int64_t slot = (int64_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
+    int64_t *my_time = p.ws_time + slot * p.slot_elems;
+    int32_t *my_qid = p.ws_qid + slot * p.slot_elems;
+    unsigned long long batches = 0;
+
+    for (;;) {
+        unsigned long long c = 0;
+        if (lane == 0) c = atomicAdd(&p.counters[0], 1ull);
+        c = __shfl_sync(full, c, 0);
+        if (c >= (unsigned long long)p.n_cand) break;
+
+        // candidate decode: lane s reads stage s
+        il_stage_config my_cfg = {0, 1, 1, 0};
+        if (lane < p.S) my_cfg = p.configs[c * p.S + lane];
+        const bool bad = lane < p.S && (my_cfg.hw >= p.H || my_cfg.max_batch < 1 ||
+                                        my_cfg.max_batch > p.Bmax || my_cfg.replicas < 1 ||
+                                        my_cfg.replicas > IL_MAX_REPLICAS);
+        if (__any_sync(full, bad)) {
+            if (lane == 0) { atomicCAS(p.status, 0, IL_ERR_BAD_CONFIG); p.lat_or[c] = 0; }
+            for (int i = lane; i < p.n; i += 32) p.slab[c * p.slab_stride + i] = 0;
+            continue;
+        }
+
+        int64_t *slab = p.slab + c * p.slab_stride;
+        int32_t exits = 0;
+        uint64_t lat_or = 0;
+
+        for (int s = 0; s < p.S; s++) {
+            const int n_in = p.n_s[s];
+            if (n_in == 0) continue;
+            const int hw = __shfl_sync(full, (int)my_cfg.hw, s);
+            const int mb = __shfl_sync(full, (int)my_cfg.max_batch, s);
+            const int R = __shfl_sync(full, (int)my_cfg.replicas, s);
+            const int32_t *row = s_lat + (s * p.H + hw) * p.Bmax;
+            const int64_t *in_t = (s == 0) ? p.arrival : my_time + p.buf_off[s];
+            const int32_t *in_q = (s == 0) ? nullptr : my_qid + p.buf_off[s];
+
+            Route rt;
+            rt.bit = p.bit[s];
+            const int da = p.dest_a[s], db = p.dest_b[s];
+            rt.a_exit = da < 0; rt.b_exit = db < 0;
+            rt.a_time = rt.a_exit ? nullptr : my_time + p.buf_off[da];
+            rt.a_qid = rt.a_exit ? nullptr : my_qid + p.buf_off[da];
+            rt.b_time = rt.b_exit ? nullptr : my_time + p.buf_off[db];
+            rt.b_qid = rt.b_exit ? nullptr : my_qid + p.buf_off[db];
+            rt.a_tail = 0; rt.b_tail = 0;
+
+            // Emits the batch [start, start + b) of this stage's input stream,
+            // finished at time tfin, to the children / the latency slab.
+            auto emit = [&](int start, int b, int64_t tfin) {
+                for (int j0 = 0; j0 < b; j0 += 32) {
+                    const int j = j0 + lane;
+                    const bool act = j < b;
+                    int32_t q = 0;
+                    if (act) q = (s == 0) ? start + j : in_q[start + j];
+                    bool bitv = false;
+                    if (act && rt.bit >= 0) bitv = (p.bits[q] >> rt.bit) & 1;
+                    const unsigned ma = __ballot_sync(full, act && !bitv);
+                    const unsigned mb_ = __ballot_sync(full, act && bitv);
+                    if (ma) {
+                        const bool mine = act && !bitv;
+                        const int rank = __popc(ma & lt_mask);
+                        if (rt.a_exit) {
+                            if (mine) {
+                                const int64_t l = tfin - p.arrival[q];
+                                slab[exits + rank] = l;
+                                lat_or |= (uint64_t)l;
+                            }
+                            exits += __popc(ma);
+                        } else {
+                            if (mine) { rt.a_time[rt.a_tail + rank] = tfin; rt.a_qid[rt.a_tail + rank] = q; }
+                            rt.a_tail += __popc(ma);
+                        }
+                    }
+                    if (mb_) {
+                        const bool mine = act && bitv;
+                        const int rank = __popc(mb_ & lt_mask);
+                        if (rt.b_exit) {
+                            if (mine) {
+                                const int64_t l = tfin - p.arrival[q];
+                                slab[exits + rank] = l;
+                                lat_or |= (uint64_t)l;
+                            }
+                            exits += __popc(mb_);
+                        } else {
+                            if (mine) { rt.b_time[rt.b_tail + rank] = tfin; rt.b_qid[rt.b_tail + rank] = q; }
+                            rt.b_tail += __popc(mb_);
+                        }
+                    }
+                }
+            };
+
+            // replica slots: lane r < R holds replica r
+            int64_t fin = (lane < R) ? -1 : kNever;   // -1: idle since before the first arrival
+            int32_t seq = lane, sl_start = 0, sl_b = 0;
+            int32_t seq_ctr = 32;
+
+            // picks the slot with the smallest (finish, dispatch order)
+            auto pick = [&](int64_t minfin) -> int {
+                const unsigned tie = __ballot_sync(full, fin == minfin);
+                if (__popc(tie) == 1) return __ffs(tie) - 1;
+                const int32_t myseq = (fin == minfin) ? seq : INT32_MAX;
+                const int32_t mseq = __reduce_min_sync(full, myseq);
+                return __ffs(__ballot_sync(full, myseq == mseq)) - 1;
+            };
+
+            int head = 0;
+            int guard = 0;
+            while (head < n_in) {
+                const int64_t minfin = warp_min_i64(fin);
+                const int sel = pick(minfin);
+                // lookahead: how many queued arrivals are there at time t, up to mb
+                const int i0 = head + lane;
+                const int64_t v0 = (lane < mb && i0 < n_in) ? in_t[i0] : kNever;
+                const int64_t a_head = __shfl_sync(full, v0, 0);
+                const int64_t t = minfin > a_head ? minfin : a_head;
+                int cnt = __popc(__ballot_sync(full, v0 <= t));
+                if (mb > 32 && cnt == 32) {
+                    const int i1 = head + 32 + lane;
+                    const int64_t v1 = (32 + lane < mb && i1 < n_in) ? in_t[i1] : kNever;
+                    cnt += __popc(__ballot_sync(full, v1 <= t));
+                }
+                const int64_t newfin = t + (int64_t)row[cnt - 1];
+                // the slot being reused gives up the batch it held
+                const int pb = __shfl_sync(full, sl_b, sel);
+                const int ps = __shfl_sync(full, sl_start, sel);
+                if (pb > 0) emit(ps, pb, minfin);
+                if (lane == sel) { fin = newfin; seq = seq_ctr; sl_start = head; sl_b = cnt; }
+                seq_ctr++;
+                head += cnt;
+                batches++;
+                if (++guard > n_in) {   // cannot happen: every batch takes >= 1 query
+                    if (lane == 0) atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT);
+                    break;
+                }
+            }
+            // drain what is still in flight, in (finish, dispatch order) order
+            for (int k = 0; k < 32; k++) {
+                const int64_t minfin = warp_min_i64(fin);
+                if (minfin == kNever) break;
+                const int sel = pick(minfin);
+                const int pb = __shfl_sync(full, sl_b, sel);
+                const int ps = __shfl_sync(full, sl_start, sel);
+                if (pb > 0) emit(ps, pb, minfin);
+                if (lane == sel) { fin = kNever; sl_b = 0; }
+            }
+            __syncwarp();   // order this stage's stream writes before the next stage's reads
+        }
+
+        // OR-reduce the latencies' bit pattern (tells the select kernel which digits matter)
+        const uint32_t lo = __reduce_or_sync(full, (uint32_t)lat_or);
+        const uint32_t hi = __reduce_or_sync(full, (uint32_t)(lat_or >> 32));
+        if (lane == 0) {
+            p.lat_or[c] = ((uint64_t)hi << 32) | lo;
+            if (exits != p.n) atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT);
+        }
+    }
+    if (lane == 0 && batches) atomicAdd(&p.counters[1], batches);
+}
+
+cudaError_t launch_des(const DesParams &p, int grid, size_t smem, cudaStream_t stream)
+{
+    des_kernel<<<grid, kWarpsPerCta * 32, smem, stream>>>(p);
+    return cudaGetLastError();
+}
+
+int des_max_ctas_per_sm(size_t smem)
+{
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, des_kernel, kWarpsPerCta * 32, smem) != cudaSuccess)
+        return 0;
+    return n;
+}
+
+// Dependency-free integer instruction stream: 8 independent chains per thread,
+// half multiply-add and half logic/add so that both integer pipes are fed.
+// One inner step is 4 multiply-adds + 4 x (xor, add) = 12 instructions.
+__global__ void __launch_bounds__(256) int_issue_kernel(unsigned *sink, int iters)
+{
+    unsigned a0 = threadIdx.x, a1 = a0 + 1, a2 = a0 + 2, a3 = a0 + 3,
+             a4 = a0 + 4, a5 = a0 + 5, a6 = a0 + 6, a7 = a0 + 7;
+    const unsigned k = blockIdx.x | 1u;
+    for (int i = 0; i < iters; i++) {
+#pragma unroll
+        for (int u = 0; u < 16; u++) {
+            a0 = a0 * k + 1u; a1 = a1 * k + 2u; a2 = a2 * k + 3u; a3 = a3 * k + 4u;
+            a4 = (a4 ^ k) + 5u; a5 = (a5 ^ k) + 6u; a6 = (a6 ^ k) + 7u; a7 = (a7 ^ k) + 8u;
+        }
+    }
+    const unsigned r = a0 ^ a1 ^ a2 ^ a3 ^ a4 ^ a5 ^ a6 ^ a7;
+    if (r == 0x12345678u) sink[0] = r;   // keeps the loop alive
+}
+
+cudaError_t launch_int_issue(unsigned *sink, int grid, int iters, cudaStream_t stream)
+{
+    int_issue_kernel<<<grid, 256, 0, stream>>>(sink, iters);
+    return cudaGetLastError();
+}
+
+}  // namespace il

@@ -1,0 +1,547 @@
+// Host side of the C ABI declared in il_estimator.h: validation, device copies
+// of the bound inputs, workspace planning, chunked launches and error codes.
+#include "il_internal.h"
+
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+using namespace il;
+
+static thread_local int g_last_cuda_error = 0;
+
+#define IL_CUDA(call)                                   \
+    do {                                                \
+        cudaError_t e_ = (call);                        \
+        if (e_ != cudaSuccess) {                        \
+            g_last_cuda_error = (int)e_;                \
+            return IL_ERR_CUDA;                         \
+        }                                               \
+    } while (0)
+
+struct il_estimator {
+    int device = 0;
+    int num_sms = 0;
+    int ctas_per_sm = 0;
+    cudaStream_t stream = nullptr;
+
+    int32_t S = 0, H = 0, Bmax = 0;
+    int64_t n = 0;
+    int64_t n_pad = 0;                 // n rounded up to 32: one slab row
+    int64_t visits[IL_MAX_STAGES] = {};
+    int64_t events_per_candidate = 0;
+    DesParams base = {};               // bound-input part of the kernel parameters
+    size_t smem = 0;
+    int64_t slot_elems = 0;
+
+    int64_t *d_arrival = nullptr;
+    uint8_t *d_bits = nullptr;
+    int32_t *d_lat = nullptr;
+    unsigned long long *d_counters = nullptr;   // [2]
+    int *d_status = nullptr;
+    unsigned long long *h_counters = nullptr;   // pinned: [2] counters, then the status word
+    int *h_status = nullptr;
+
+    void *user_ws = nullptr; size_t user_ws_bytes = 0;
+    void *own_ws = nullptr;  size_t own_ws_bytes = 0;
+
+    il_stage_config *d_cfg = nullptr; int64_t d_cfg_cap = 0;   // staging for il_estimate
+    int64_t *d_out = nullptr; int64_t d_out_cap = 0;           // [2][cap]
+
+    std::vector<cudaEvent_t> events;
+    il_stats stats = {};
+};
+
+namespace {
+
+struct Plan {
+    int64_t slots = 0;       // warp slots with stream buffers
+    int64_t chunk = 0;       // candidates per (simulate, select) pair
+    size_t off_time = 0, off_qid = 0, off_slab = 0, off_or = 0, total = 0;
+};
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+size_t slot_bytes(const il_estimator *e) { return (size_t)e->slot_elems * 12; }
+size_t cand_bytes(const il_estimator *e) { return (size_t)e->n_pad * 8 + 8; }
+
+int64_t full_slots(const il_estimator *e)
+{
+    return (int64_t)e->num_sms * e->ctas_per_sm * kWarpsPerCta;
+}
+
+int64_t wanted_slots(const il_estimator *e, int64_t n_cand)
+{
+    const int64_t need = (n_cand + kWarpsPerCta - 1) / kWarpsPerCta * kWarpsPerCta;
+    return std::max<int64_t>(kWarpsPerCta, std::min(full_slots(e), need));
+}
+
+size_t layout(const il_estimator *e, Plan &pl)
+{
+    size_t off = 0;
+    pl.off_time = off; off = align_up(off + (size_t)pl.slots * e->slot_elems * 8, 256);
+    pl.off_qid = off;  off = align_up(off + (size_t)pl.slots * e->slot_elems * 4, 256);
+    pl.off_slab = off; off = align_up(off + (size_t)pl.chunk * e->n_pad * 8, 256);
+    pl.off_or = off;   off = align_up(off + (size_t)pl.chunk * 8, 256);
+    pl.total = off;
+    return off;
+}
+
+size_t recommended_bytes(const il_estimator *e, int64_t n_cand)
+{
+    Plan pl;
+    n_cand = std::max<int64_t>(n_cand, 1);
+    pl.slots = wanted_slots(e, n_cand);
+    pl.chunk = std::max<int64_t>(std::min<int64_t>(n_cand, 8 * full_slots(e)), pl.slots);
+    return layout(e, pl) + 1024;
+}
+
+size_t min_bytes(const il_estimator *e)
+{
+    Plan pl;
+    pl.slots = kWarpsPerCta;
+    pl.chunk = 2 * kWarpsPerCta;
+    return layout(e, pl) + 1024;
+}
+
+// Splits `bytes` of workspace between warp slots and the latency slab.
+bool make_plan(const il_estimator *e, size_t bytes, int64_t n_cand, Plan &pl)
+{
+    if (bytes < min_bytes(e)) return false;
+    const size_t usable = bytes - 1024;
+    const size_t sb = slot_bytes(e), cb = cand_bytes(e);
+    int64_t slots = std::min<int64_t>(wanted_slots(e, n_cand), (int64_t)(usable / (sb + 2 * cb)));
+    slots = slots / kWarpsPerCta * kWarpsPerCta;
+    if (slots < kWarpsPerCta) return false;
+    pl.slots = slots;
+    pl.chunk = std::min<int64_t>(n_cand, (int64_t)((usable - (size_t)slots * sb) / cb));
+    // alignment padding may push the layout over: shrink the chunk until it fits
+    while (pl.chunk > 0 && layout(e, pl) > bytes) pl.chunk -= std::max<int64_t>(1, pl.chunk / 64);
+    return pl.chunk >= 1;
+}
+
+int check_topology(const il_profiles *pr)
+{
+    const int S = pr->n_stages;
+    if (pr->parent[0] != -1) return IL_ERR_BAD_TOPOLOGY;
+    for (int s = 1; s < S; s++) {
+        if (pr->parent[s] < 0 || pr->parent[s] >= s) return IL_ERR_BAD_TOPOLOGY;
+        if (pr->cond_bit[s] < -1 || pr->cond_bit[s] > 7) return IL_ERR_BAD_TOPOLOGY;
+        if (pr->cond_bit[s] >= 0 && pr->cond_val[s] > 1) return IL_ERR_BAD_TOPOLOGY;
+    }
+    for (int par = 0; par < S; par++) {
+        int kids[IL_MAX_STAGES], nk = 0;
+        for (int c = 1; c < S; c++) if (pr->parent[c] == par) kids[nk++] = c;
+        if (nk > 2) return IL_ERR_BAD_TOPOLOGY;
+        if (nk == 2) {
+            const int a = kids[0], b = kids[1];
+            if (pr->cond_bit[a] < 0 || pr->cond_bit[b] != pr->cond_bit[a]) return IL_ERR_BAD_TOPOLOGY;
+            if (pr->cond_val[a] == pr->cond_val[b]) return IL_ERR_BAD_TOPOLOGY;
+        }
+    }
+    return IL_OK;
+}
+
+// Lays the stages' input streams out inside one warp slot.  Stage c's stream is
+// written while its parent is simulated and read while c is; stages are
+// simulated in index order, so the stream is live over the steps
+// [parent[c], c] and two streams may share memory when these ranges are disjoint.
+int64_t plan_stream_buffers(const il_profiles *pr, const int64_t *visits, int32_t *buf_off)
+{
+    const int S = pr->n_stages;
+    struct Live { int64_t off, size; int end; };
+    std::vector<Live> live;
+    std::vector<int> order;
+    for (int c = 1; c < S; c++) order.push_back(c);
+    std::stable_sort(order.begin(), order.end(),
+                     [&](int a, int b) { return pr->parent[a] < pr->parent[b]; });
+    int64_t top = 0;
+    buf_off[0] = 0;
+    for (int c : order) {
+        const int start = pr->parent[c];
+        const int64_t size = (visits[c] + 31) / 32 * 32;
+        buf_off[c] = 0;
+        if (size == 0) continue;
+        std::vector<Live> busy;
+        for (const Live &l : live) if (l.end >= start) busy.push_back(l);
+        std::sort(busy.begin(), busy.end(), [](const Live &a, const Live &b) { return a.off < b.off; });
+        int64_t off = 0;
+        for (const Live &l : busy) {
+            if (off + size <= l.off) break;
+            off = std::max(off, l.off + l.size);
+        }
+        buf_off[c] = (int32_t)off;
+        live.push_back({off, size, c});
+        top = std::max(top, off + size);
+    }
+    return top;
+}
+
+void free_device(il_estimator *e)
+{
+    cudaFree(e->d_arrival); cudaFree(e->d_bits); cudaFree(e->d_lat);
+    cudaFree(e->d_counters); cudaFree(e->d_status);
+    cudaFree(e->own_ws); cudaFree(e->d_cfg); cudaFree(e->d_out);
+    if (e->h_counters) cudaFreeHost(e->h_counters);
+    for (cudaEvent_t ev : e->events) cudaEventDestroy(ev);
+}
+
+int ensure_events(il_estimator *e, size_t count)
+{
+    while (e->events.size() < count) {
+        cudaEvent_t ev;
+        IL_CUDA(cudaEventCreate(&ev));
+        e->events.push_back(ev);
+    }
+    return IL_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *il_strerror(int code)
+{
+    switch (code) {
+    case IL_OK: return "ok";
+    case IL_ERR_INVALID_ARG: return "invalid argument";
+    case IL_ERR_BAD_TOPOLOGY: return "pipeline is not a tree of the accepted form";
+    case IL_ERR_BAD_PROFILE: return "latency table entry below 1";
+    case IL_ERR_BAD_TRACE: return "arrival trace negative, decreasing or too large";
+    case IL_ERR_BAD_CONFIG: return "candidate configuration out of range";
+    case IL_ERR_NOMEM: return "out of memory or workspace too small";
+    case IL_ERR_CUDA: return "CUDA call failed";
+    case IL_ERR_ITER_LIMIT: return "device loop exceeded its iteration bound";
+    default: return "unknown error";
+    }
+}
+
+int il_last_cuda_error(void) { return g_last_cuda_error; }
+
+int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator **out)
+{
+    if (!pr || !tr || !out) return IL_ERR_INVALID_ARG;
+    if (pr->n_stages < 1 || pr->n_stages > IL_MAX_STAGES || pr->n_hw < 1 || pr->n_hw > IL_MAX_HW ||
+        pr->max_batch < 1 || pr->max_batch > IL_MAX_BATCH)
+        return IL_ERR_INVALID_ARG;
+    if (!pr->parent || !pr->cond_bit || !pr->cond_val || !pr->latency_us || !tr->arrival_us)
+        return IL_ERR_INVALID_ARG;
+    if (tr->n_queries < 1 || tr->n_queries > INT32_MAX) return IL_ERR_INVALID_ARG;
+    int rc = check_topology(pr);
+    if (rc) return rc;
+    const int S = pr->n_stages, H = pr->n_hw, B = pr->max_batch;
+    const int64_t n = tr->n_queries;
+    bool any_cond = false;
+    for (int s = 1; s < S; s++) any_cond |= pr->cond_bit[s] >= 0;
+    if (any_cond && !tr->branch_bits) return IL_ERR_INVALID_ARG;
+
+    int64_t worst = 0;   // bound on how far the clock can run past the last arrival
+    for (int s = 0; s < S; s++) {
+        int32_t mx = 0;
+        for (int i = 0; i < H * B; i++) {
+            const int32_t v = pr->latency_us[(size_t)s * H * B + i];
+            if (v < 1) return IL_ERR_BAD_PROFILE;
+            mx = std::max(mx, v);
+        }
+        worst += n * (int64_t)mx;   // n < 2^31, mx < 2^31, S <= 16: no overflow
+    }
+    if (tr->arrival_us[0] < 0) return IL_ERR_BAD_TRACE;
+    for (int64_t i = 1; i < n; i++)
+        if (tr->arrival_us[i] < tr->arrival_us[i - 1]) return IL_ERR_BAD_TRACE;
+    if (tr->arrival_us[n - 1] > (INT64_C(1) << 62) - worst) return IL_ERR_BAD_TRACE;
+
+    int dev = 0;
+    cudaDeviceProp prop;
+    IL_CUDA(cudaGetDevice(&dev));
+    IL_CUDA(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major != 10) { g_last_cuda_error = (int)cudaErrorNoKernelImageForDevice; return IL_ERR_CUDA; }
+
+    il_estimator *e = new (std::nothrow) il_estimator();
+    if (!e) return IL_ERR_NOMEM;
+    e->device = dev;
+    e->num_sms = prop.multiProcessorCount;
+    e->S = S; e->H = H; e->Bmax = B; e->n = n;
+    e->n_pad = (n + 31) / 32 * 32;
+
+    // routing table and visits per stage
+    DesParams &bp = e->base;
+    for (int s = 0; s < IL_MAX_STAGES; s++) { bp.dest_a[s] = -1; bp.dest_b[s] = -1; bp.bit[s] = -1; }
+    for (int c = 1; c < S; c++) {
+        const int par = pr->parent[c];
+        if (pr->cond_bit[c] < 0) { bp.dest_a[par] = (int8_t)c; bp.dest_b[par] = (int8_t)c; }
+        else {
+            bp.bit[par] = pr->cond_bit[c];
+            if (pr->cond_val[c] == 0) bp.dest_a[par] = (int8_t)c; else bp.dest_b[par] = (int8_t)c;
+        }
+    }
+    e->visits[0] = n;
+    for (int64_t q = 0; q < n; q++) {   // walk every query down its path
+        int s = 0;
+        for (;;) {
+            int nxt;
+            if (bp.bit[s] < 0) nxt = bp.dest_a[s];
+            else nxt = ((tr->branch_bits[q] >> bp.bit[s]) & 1) ? bp.dest_b[s] : bp.dest_a[s];
+            if (nxt < 0) break;
+            e->visits[nxt]++;
+            s = nxt;
+        }
+    }
+    e->events_per_candidate = 0;
+    for (int s = 0; s < S; s++) e->events_per_candidate += e->visits[s];
+    e->slot_elems = std::max<int64_t>(32, plan_stream_buffers(pr, e->visits, bp.buf_off));
+    for (int s = 0; s < S; s++) bp.n_s[s] = (int32_t)e->visits[s];
+    bp.S = S; bp.H = H; bp.Bmax = B; bp.n = (int32_t)n;
+    e->smem = (size_t)S * H * B * sizeof(int32_t);
+
+    auto fail = [&](int code) { free_device(e); delete e; return code; };
+#define IL_CUDA_E(call)                                                   \
+    do { cudaError_t e_ = (call); if (e_ != cudaSuccess) {                \
+        g_last_cuda_error = (int)e_;                                      \
+        return fail(e_ == cudaErrorMemoryAllocation ? IL_ERR_NOMEM : IL_ERR_CUDA); } } while (0)
+
+    IL_CUDA_E(cudaMalloc(&e->d_arrival, (size_t)n * 8));
+    IL_CUDA_E(cudaMalloc(&e->d_bits, (size_t)n));
+    IL_CUDA_E(cudaMalloc(&e->d_lat, e->smem));
+    IL_CUDA_E(cudaMalloc(&e->d_counters, 2 * sizeof(unsigned long long)));
+    IL_CUDA_E(cudaMalloc(&e->d_status, sizeof(int)));
+    IL_CUDA_E(cudaMallocHost(&e->h_counters, 4 * sizeof(unsigned long long)));
+    e->h_status = reinterpret_cast<int *>(e->h_counters + 2);
+    IL_CUDA_E(cudaMemcpy(e->d_arrival, tr->arrival_us, (size_t)n * 8, cudaMemcpyHostToDevice));
+    if (tr->branch_bits) IL_CUDA_E(cudaMemcpy(e->d_bits, tr->branch_bits, (size_t)n, cudaMemcpyHostToDevice));
+    else IL_CUDA_E(cudaMemset(e->d_bits, 0, (size_t)n));
+    IL_CUDA_E(cudaMemcpy(e->d_lat, pr->latency_us, e->smem, cudaMemcpyHostToDevice));
+#undef IL_CUDA_E
+    bp.arrival = e->d_arrival; bp.bits = e->d_bits; bp.lat = e->d_lat;
+    bp.counters = e->d_counters; bp.status = e->d_status;
+
+    e->ctas_per_sm = des_max_ctas_per_sm(e->smem);
+    if (e->ctas_per_sm < 1) return fail(IL_ERR_CUDA);
+    *out = e;
+    return IL_OK;
+}
+
+void il_estimator_destroy(il_estimator *e)
+{
+    if (!e) return;
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaSetDevice(e->device);
+    free_device(e);
+    cudaSetDevice(prev);
+    delete e;
+}
+
+int il_set_stream(il_estimator *e, void *cuda_stream)
+{
+    if (!e) return IL_ERR_INVALID_ARG;
+    e->stream = static_cast<cudaStream_t>(cuda_stream);
+    return IL_OK;
+}
+
+int il_workspace_bytes(const il_estimator *e, int64_t n_candidates, size_t *bytes)
+{
+    if (!e || !bytes || n_candidates < 0) return IL_ERR_INVALID_ARG;
+    *bytes = recommended_bytes(e, n_candidates);
+    return IL_OK;
+}
+
+int il_workspace_min_bytes(const il_estimator *e, size_t *bytes)
+{
+    if (!e || !bytes) return IL_ERR_INVALID_ARG;
+    *bytes = min_bytes(e);
+    return IL_OK;
+}
+
+int il_set_workspace(il_estimator *e, void *d_ws, size_t bytes)
+{
+    if (!e) return IL_ERR_INVALID_ARG;
+    if (!d_ws || bytes == 0) { e->user_ws = nullptr; e->user_ws_bytes = 0; return IL_OK; }
+    if (reinterpret_cast<uintptr_t>(d_ws) % 256 != 0) return IL_ERR_INVALID_ARG;
+    if (bytes < min_bytes(e)) return IL_ERR_NOMEM;
+    e->user_ws = d_ws;
+    e->user_ws_bytes = bytes;
+    return IL_OK;
+}
+
+int il_get_stats(const il_estimator *e, il_stats *out)
+{
+    if (!e || !out) return IL_ERR_INVALID_ARG;
+    *out = e->stats;
+    return IL_OK;
+}
+
+int il_stage_visits(const il_estimator *e, int64_t *out_visits)
+{
+    if (!e || !out_visits) return IL_ERR_INVALID_ARG;
+    for (int s = 0; s < e->S; s++) out_visits[s] = e->visits[s];
+    return IL_OK;
+}
+
+int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_t n_cand,
+                       int64_t slo_us, int64_t *d_out_p99, int64_t *d_out_miss)
+{
+    if (!e || n_cand < 0) return IL_ERR_INVALID_ARG;
+    e->stats = il_stats{};
+    if (n_cand == 0) return IL_OK;
+    if (!d_configs || !d_out_p99 || !d_out_miss) return IL_ERR_INVALID_ARG;
+    IL_CUDA(cudaSetDevice(e->device));
+
+    // workspace
+    char *ws = static_cast<char *>(e->user_ws);
+    size_t ws_bytes = e->user_ws_bytes;
+    if (!ws) {
+        const size_t want = recommended_bytes(e, n_cand);
+        if (e->own_ws_bytes < want) {
+            size_t free_b = 0, total_b = 0;
+            IL_CUDA(cudaMemGetInfo(&free_b, &total_b));
+            const size_t grant = std::min(want, (size_t)((free_b + e->own_ws_bytes) * 0.8));
+            if (grant > e->own_ws_bytes) {
+                IL_CUDA(cudaStreamSynchronize(e->stream));
+                if (e->own_ws) { cudaFree(e->own_ws); e->own_ws = nullptr; e->own_ws_bytes = 0; }
+                if (grant < min_bytes(e)) return IL_ERR_NOMEM;
+                cudaError_t ce = cudaMalloc(&e->own_ws, grant);
+                if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; e->own_ws = nullptr; return IL_ERR_NOMEM; }
+                e->own_ws_bytes = grant;
+            }
+        }
+        ws = static_cast<char *>(e->own_ws);
+        ws_bytes = e->own_ws_bytes;
+    }
+    Plan pl;
+    if (!make_plan(e, ws_bytes, n_cand, pl)) return IL_ERR_NOMEM;
+
+    const int64_t n_chunks = (n_cand + pl.chunk - 1) / pl.chunk;
+    int rc = ensure_events(e, (size_t)(2 + 3 * n_chunks));
+    if (rc) return rc;
+
+    cudaStream_t st = e->stream;
+    IL_CUDA(cudaMemsetAsync(e->d_counters, 0, 2 * sizeof(unsigned long long), st));
+    IL_CUDA(cudaMemsetAsync(e->d_status, 0, sizeof(int), st));
+    IL_CUDA(cudaEventRecord(e->events[0], st));
+
+    int64_t launches = 0;
+    for (int64_t ch = 0; ch < n_chunks; ch++) {
+        const int64_t lo = ch * pl.chunk;
+        const int64_t cnt = std::min(pl.chunk, n_cand - lo);
+        DesParams p = e->base;
+        p.configs = d_configs + lo * e->S;
+        p.n_cand = cnt;
+        p.slot_elems = e->slot_elems;
+        p.ws_time = reinterpret_cast<int64_t *>(ws + pl.off_time);
+        p.ws_qid = reinterpret_cast<int32_t *>(ws + pl.off_qid);
+        p.slab = reinterpret_cast<int64_t *>(ws + pl.off_slab);
+        p.slab_stride = e->n_pad;
+        p.lat_or = reinterpret_cast<uint64_t *>(ws + pl.off_or);
+        if (ch > 0) IL_CUDA(cudaMemsetAsync(e->d_counters, 0, sizeof(unsigned long long), st));
+        const int64_t ctas = std::min<int64_t>(pl.slots / kWarpsPerCta, (cnt + kWarpsPerCta - 1) / kWarpsPerCta);
+        IL_CUDA(cudaEventRecord(e->events[2 + 3 * ch], st));
+        IL_CUDA(launch_des(p, (int)ctas, e->smem, st));
+        IL_CUDA(cudaEventRecord(e->events[3 + 3 * ch], st));
+        SelectParams sp;
+        sp.slab = p.slab; sp.slab_stride = e->n_pad; sp.lat_or = p.lat_or;
+        sp.n = (int32_t)e->n; sp.n_cand = cnt; sp.slo_us = slo_us;
+        sp.out_p99 = d_out_p99 + lo; sp.out_miss = d_out_miss + lo;
+        IL_CUDA(launch_select(sp, st));
+        IL_CUDA(cudaEventRecord(e->events[4 + 3 * ch], st));
+        launches += 2;
+    }
+    IL_CUDA(cudaEventRecord(e->events[1], st));
+    IL_CUDA(cudaMemcpyAsync(e->h_counters, e->d_counters, 2 * sizeof(unsigned long long),
+                            cudaMemcpyDeviceToHost, st));
+    IL_CUDA(cudaMemcpyAsync(e->h_status, e->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+    IL_CUDA(cudaStreamSynchronize(st));
+
+    float ms = 0.f;
+    IL_CUDA(cudaEventElapsedTime(&ms, e->events[0], e->events[1]));
+    e->stats.total_ms = ms;
+    for (int64_t ch = 0; ch < n_chunks; ch++) {
+        IL_CUDA(cudaEventElapsedTime(&ms, e->events[2 + 3 * ch], e->events[3 + 3 * ch]));
+        e->stats.sim_ms += ms;
+        IL_CUDA(cudaEventElapsedTime(&ms, e->events[3 + 3 * ch], e->events[4 + 3 * ch]));
+        e->stats.select_ms += ms;
+    }
+    e->stats.candidates = n_cand;
+    e->stats.query_events = n_cand * e->events_per_candidate;
+    e->stats.batches = (int64_t)e->h_counters[1];
+    e->stats.chunks = n_chunks;
+    e->stats.kernel_launches = launches;
+    return *e->h_status;
+}
+
+int il_estimate(il_estimator *e, const il_stage_config *configs, int64_t n_cand, int64_t slo_us,
+                int64_t *out_p99, int64_t *out_miss)
+{
+    if (!e || n_cand < 0) return IL_ERR_INVALID_ARG;
+    if (n_cand == 0) { e->stats = il_stats{}; return IL_OK; }
+    if (!configs || !out_p99 || !out_miss) return IL_ERR_INVALID_ARG;
+    const int64_t total = n_cand * e->S;
+    for (int64_t i = 0; i < total; i++) {
+        const il_stage_config &c = configs[i];
+        if (c.hw >= e->H || c.max_batch < 1 || c.max_batch > e->Bmax || c.replicas < 1 ||
+            c.replicas > IL_MAX_REPLICAS)
+            return IL_ERR_BAD_CONFIG;
+    }
+    IL_CUDA(cudaSetDevice(e->device));
+    if (e->d_cfg_cap < total) {
+        IL_CUDA(cudaStreamSynchronize(e->stream));
+        cudaFree(e->d_cfg); e->d_cfg = nullptr; e->d_cfg_cap = 0;
+        cudaError_t ce = cudaMalloc(&e->d_cfg, (size_t)total * sizeof(il_stage_config));
+        if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return IL_ERR_NOMEM; }
+        e->d_cfg_cap = total;
+    }
+    if (e->d_out_cap < n_cand) {
+        IL_CUDA(cudaStreamSynchronize(e->stream));
+        cudaFree(e->d_out); e->d_out = nullptr; e->d_out_cap = 0;
+        cudaError_t ce = cudaMalloc(&e->d_out, (size_t)n_cand * 16);
+        if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return IL_ERR_NOMEM; }
+        e->d_out_cap = n_cand;
+    }
+    IL_CUDA(cudaMemcpyAsync(e->d_cfg, configs, (size_t)total * sizeof(il_stage_config),
+                            cudaMemcpyHostToDevice, e->stream));
+    int rc = il_estimate_device(e, e->d_cfg, n_cand, slo_us, e->d_out, e->d_out + e->d_out_cap);
+    if (rc) return rc;
+    IL_CUDA(cudaMemcpyAsync(out_p99, e->d_out, (size_t)n_cand * 8, cudaMemcpyDeviceToHost, e->stream));
+    IL_CUDA(cudaMemcpyAsync(out_miss, e->d_out + e->d_out_cap, (size_t)n_cand * 8,
+                            cudaMemcpyDeviceToHost, e->stream));
+    IL_CUDA(cudaStreamSynchronize(e->stream));
+    return IL_OK;
+}
+
+int il_measure_int_issue(void *cuda_stream, double *out_warp_inst_per_s, double *out_ms)
+{
+    if (!out_warp_inst_per_s) return IL_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int dev = 0;
+    cudaDeviceProp prop;
+    IL_CUDA(cudaGetDevice(&dev));
+    IL_CUDA(cudaGetDeviceProperties(&prop, dev));
+    unsigned *sink = nullptr;
+    IL_CUDA(cudaMalloc(&sink, sizeof(unsigned)));
+    cudaEvent_t a, b;
+    IL_CUDA(cudaEventCreate(&a));
+    IL_CUDA(cudaEventCreate(&b));
+    const int grid = prop.multiProcessorCount * 8;   // 8 CTAs of 8 warps per SM
+    const int iters = 4096;
+    cudaError_t ce = launch_int_issue(sink, grid, 64, st);   // warm-up
+    float best = 1e30f;
+    for (int rep = 0; rep < 3 && ce == cudaSuccess; rep++) {
+        cudaEventRecord(a, st);
+        ce = launch_int_issue(sink, grid, iters, st);
+        cudaEventRecord(b, st);
+        if (ce == cudaSuccess) ce = cudaEventSynchronize(b);
+        float ms = 0.f;
+        if (ce == cudaSuccess) ce = cudaEventElapsedTime(&ms, a, b);
+        best = std::min(best, ms);
+    }
+    cudaEventDestroy(a); cudaEventDestroy(b); cudaFree(sink);
+    if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return IL_ERR_CUDA; }
+    // per inner step: 4 multiply-adds + 4 x (xor, add) = 12 instructions per thread
+    const double inst = (double)grid * 8.0 * iters * 16.0 * 12.0;
+    *out_warp_inst_per_s = inst / (best * 1e-3);
+    if (out_ms) *out_ms = best;
+    return IL_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,84 @@
+// Per-candidate P99 and SLO-miss count over the latency slab.
+//
+// P99 is the k-th smallest of the candidate's n latencies with
+// k = ceil(0.99 n) = (99 n + 99) / 100 (Section 2: 99% of the query latencies
+// must lie below the objective); a query misses iff latency > slo.  The k-th
+// smallest is found by most-significant-digit radix select: each pass
+// histograms one 8-bit digit of the keys that still match the prefix found so
+// far, then descends into the bucket that holds rank k.  Digits above the
+// highest set bit of any latency (known from the simulation kernel's OR) are
+// skipped.  One CTA per candidate.
+#include "il_internal.h"
+
+namespace il {
+
+__global__ void __launch_bounds__(kSelectThreads)
+select_kernel(const __grid_constant__ SelectParams p)
+{
+    __shared__ unsigned hist[256];
+    __shared__ unsigned long long s_prefix;
+    __shared__ unsigned s_rank;
+    __shared__ unsigned s_miss;
+
+    for (int64_t c = blockIdx.x; c < p.n_cand; c += gridDim.x) {
+        const int64_t *lat = p.slab + c * p.slab_stride;
+        const uint64_t bits_used = p.lat_or[c];
+        int top = 0;                                   // number of 8-bit digits that matter
+        while (top < 8 && (bits_used >> (8 * top)) != 0) top++;
+
+        if (threadIdx.x == 0) {
+            s_prefix = 0;
+            s_rank = (unsigned)((99ll * p.n + 99) / 100);   // 1-indexed rank still to find
+            s_miss = 0;
+        }
+        unsigned miss = 0;
+        bool counted_miss = false;
+        __syncthreads();
+
+        for (int d = top - 1; d >= 0; d--) {
+            hist[threadIdx.x] = 0;                     // kSelectThreads == 256 bins
+            __syncthreads();
+            const unsigned long long prefix = s_prefix;
+            const int shift = 8 * d;
+            // keys whose digits above d equal the prefix are still in the running
+            const unsigned long long himask = (d == 7) ? 0ull : (~0ull << (shift + 8));
+            for (int i = threadIdx.x; i < p.n; i += kSelectThreads) {
+                const unsigned long long v = (unsigned long long)lat[i];
+                if (!counted_miss) miss += ((int64_t)v > p.slo_us);
+                if ((v & himask) == prefix) atomicAdd(&hist[(v >> shift) & 0xff], 1u);
+            }
+            counted_miss = true;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                unsigned r = s_rank, acc = 0;
+                int b = 0;
+                for (; b < 255; b++) {
+                    if (acc + hist[b] >= r) break;
+                    acc += hist[b];
+                }
+                s_rank = r - acc;
+                s_prefix = prefix | ((unsigned long long)b << shift);
+            }
+            __syncthreads();
+        }
+        if (!counted_miss) {   // every latency is zero: cannot happen (tables >= 1); kept for safety
+            for (int i = threadIdx.x; i < p.n; i += kSelectThreads) miss += (lat[i] > p.slo_us);
+        }
+        if (miss) atomicAdd(&s_miss, miss);
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            p.out_p99[c] = (int64_t)s_prefix;
+            p.out_miss[c] = (int64_t)s_miss;
+        }
+        __syncthreads();
+    }
+}
+
+cudaError_t launch_select(const SelectParams &p, cudaStream_t stream)
+{
+    const int grid = (int)(p.n_cand < 65535 * 16 ? p.n_cand : 65535 * 16);
+    select_kernel<<<grid, kSelectThreads, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace il
