@@ -1,0 +1,176 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle: both
+outputs are integers and must be equal element by element."""
+import json
+import os
+
+import numpy as np
+import pytest
+
+import workloads
+
+pytestmark = pytest.mark.gpu
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+
+@pytest.fixture(scope="module")
+def il():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    import paper_1812_01776_b200 as il_
+    il_.load_library()
+    return il_
+
+
+def gpu_run(il, w, configs=None, slo=None, host=True, ws_bytes=None):
+    import torch
+    configs = w.configs if configs is None else configs
+    slo = w.slo_us if slo is None else slo
+    with il.Estimator.from_workload(w) as est:
+        if ws_bytes is not None:
+            est.reserve_workspace(len(configs), max_bytes=ws_bytes)
+        if host:
+            p99, miss = est.estimate(configs, slo)
+        else:
+            d = torch.from_numpy(np.ascontiguousarray(configs)).cuda()
+            a, b = est.estimate_device(d, slo)
+            p99, miss = a.cpu().numpy(), b.cpu().numpy()
+        return p99, miss, est.stats()
+
+
+def check(il, oracle, w, **kw):
+    exp_p99, exp_miss = oracle.estimate_workload(w)
+    p99, miss, st = gpu_run(il, w, **kw)
+    bad = np.nonzero((p99 != exp_p99) | (miss != exp_miss))[0]
+    assert bad.size == 0, (w.name, bad[:8], p99[bad[:8]], exp_p99[bad[:8]], miss[bad[:8]],
+                           exp_miss[bad[:8]], w.configs[bad[:2]])
+    assert st["candidates"] == w.n_candidates
+    assert st["query_events"] == w.n_candidates * w.query_events()
+    return st
+
+
+def _hand_cases():
+    with open(os.path.join(HERE, "golden", "hand_traces.json")) as f:
+        return json.load(f)["cases"]
+
+
+@pytest.mark.parametrize("case", _hand_cases(), ids=lambda c: c["name"])
+def test_hand_traces(il, case):
+    bits = np.array(case["branch_bits"], np.uint8) if "branch_bits" in case else None
+    with il.Estimator(np.array(case["parent"], np.int32), np.array(case["cond_bit"], np.int8),
+                      np.array(case["cond_val"], np.uint8), np.array(case["latency_us"], np.int32),
+                      np.array(case["arrival_us"], np.int64), bits) as est:
+        p99, miss = est.estimate(np.array([case["config"]], np.uint8), case["slo_us"])
+    assert (int(p99[0]), int(miss[0])) == (case["p99_us"], case["miss"])
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_small(il, oracle, seed):
+    w = workloads.random_small(seed, S=1 + seed % 6, H=3, Bmax=[4, 33, 64][seed % 3], n=700 + 37 * seed,
+                               C=40, max_replicas=[3, 8, 32][seed % 3], tree=(seed % 2 == 1),
+                               qps=400.0, cv=3.0, lat_lo=1, lat_hi=20000,
+                               equal_stamp_every=(3 if seed % 4 == 0 else 0))
+    check(il, oracle, w, host=(seed % 2 == 0))
+
+
+def test_config1_full(il, oracle):
+    st = check(il, oracle, workloads.make(1))
+    assert st["batches"] > 0 and st["kernel_launches"] == 2 * st["chunks"]
+
+
+@pytest.mark.parametrize("cid,n,C", [(2, 5000, 300), (3, 6001, 200), (4, 3000, 150), (5, 4097, 260)])
+def test_configs_reduced(il, oracle, cid, n, C):
+    check(il, oracle, workloads.make(cid, n_queries=n, n_candidates=C), host=False)
+
+
+def test_multi_chunk_small_workspace(il, oracle):
+    """A workspace that holds only a few candidates forces many chunks."""
+    w = workloads.make(2, n_queries=2000, n_candidates=100)
+    with il.Estimator.from_workload(w) as est:
+        lo = il.il_workspace_min_bytes(est._h)
+    st = check(il, oracle, w, ws_bytes=lo + 40 * 2000 * 8)
+    assert st["chunks"] > 1
+
+
+def test_edge_cases(il, oracle):
+    # one query, one stage
+    w = workloads.random_small(100, S=1, H=1, Bmax=1, n=1, C=1, max_replicas=1)
+    check(il, oracle, w)
+    # all queries at one instant, largest batch and replica counts
+    w = workloads.random_small(101, S=3, H=2, Bmax=64, n=1000, C=8, max_replicas=32)
+    w.arrival_us[:] = 5
+    w.configs[:, :, workloads.CFG_MAX_BATCH] = 64
+    w.configs[:, :, workloads.CFG_REPLICAS] = [[32, 1, 32]] * 8
+    check(il, oracle, w)
+    # a branch nobody takes (a stage with zero visits) and one everybody takes
+    w = workloads.make(3, n_queries=500, n_candidates=16)
+    w.branch_bits[:] = 0
+    check(il, oracle, w)
+    w.branch_bits[:] = 1
+    check(il, oracle, w)
+    # latencies beyond 32 bits: a slow single replica on a long trace
+    w = workloads.random_small(102, S=2, H=1, Bmax=2, n=3000, C=4, max_replicas=1,
+                               lat_lo=2_000_000_000, lat_hi=2_100_000_000)
+    exp = oracle.estimate_workload(w)
+    assert exp[0].max() > 2 ** 32
+    check(il, oracle, w)
+    # zero candidates is a no-op
+    with il.Estimator.from_workload(w) as est:
+        p99, miss = est.estimate(w.configs[:0], w.slo_us)
+        assert p99.shape == (0,) and miss.shape == (0,)
+
+
+def test_bad_candidates_are_rejected(il):
+    import torch
+    from paper_1812_01776_b200 import estimator as E
+    w = workloads.make(1, n_candidates=8)
+    with il.Estimator.from_workload(w) as est:
+        for col, val in [(0, 2), (1, 0), (1, 17), (2, 0), (2, 33)]:
+            bad = w.configs.copy()
+            bad[5, 1, col] = val
+            with pytest.raises(E.ILError) as ei:
+                est.estimate(bad, w.slo_us)
+            assert ei.value.code == E.IL_ERR_BAD_CONFIG
+            with pytest.raises(E.ILError) as ei:
+                est.estimate_device(torch.from_numpy(bad).cuda(), w.slo_us)
+            assert ei.value.code == E.IL_ERR_BAD_CONFIG
+        # the handle stays usable
+        p99, _ = est.estimate(w.configs, w.slo_us)
+        assert (p99 > 0).all()
+
+
+def test_repeatable_and_stream(il, oracle):
+    import torch
+    w = workloads.make(2, n_queries=3000, n_candidates=64)
+    exp = oracle.estimate_workload(w)
+    with il.Estimator.from_workload(w) as est:
+        est.reserve_workspace(64)
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            est.use_current_stream()
+            d = torch.from_numpy(w.configs).cuda()
+            for _ in range(3):
+                a, b = est.estimate_device(d, w.slo_us)
+                assert np.array_equal(a.cpu().numpy(), exp[0])
+                assert np.array_equal(b.cpu().numpy(), exp[1])
+
+
+def test_config2_full_size_sampled(il, oracle):
+    """Full trace and full candidate set in the configuration the bench times;
+    a seeded sample of candidates plus structured extremes is checked one by one."""
+    w = workloads.make(2)
+    p99, miss, st = gpu_run(il, w, host=False)
+    rng = np.random.default_rng(2)
+    idx = rng.choice(w.n_candidates, size=96, replace=False)
+    exp = oracle.estimate_many_parallel(w.parent, w.cond_bit, w.cond_val, w.latency_us,
+                                        w.arrival_us, w.branch_bits, w.configs[idx], w.slo_us)
+    assert np.array_equal(p99[idx], exp[0]) and np.array_equal(miss[idx], exp[1])
+    # extremes: every hardware type with min/max replicas and max batch 1 / 32
+    ext = np.array([[[h, mb, R, 0]] * 4 for h in range(3) for mb in (1, 32) for R in (1, 8)], np.uint8)
+    got = gpu_run(il, w, configs=ext, host=True)
+    exp = oracle.estimate_many_parallel(w.parent, w.cond_bit, w.cond_val, w.latency_us,
+                                        w.arrival_us, w.branch_bits, ext, w.slo_us)
+    assert np.array_equal(got[0], exp[0]) and np.array_equal(got[1], exp[1])
+    # properties that hold for every candidate
+    k = (99 * w.n_queries + 99) // 100
+    assert np.array_equal(p99 <= w.slo_us, miss <= w.n_queries - k)
+    assert (p99 > 0).all() and (miss >= 0).all() and (miss <= w.n_queries).all()
