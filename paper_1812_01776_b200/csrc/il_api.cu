@@ -94,7 +94,7 @@ size_t recommended_bytes(const il_estimator *e, int64_t n_cand)
     Plan pl;
     n_cand = std::max<int64_t>(n_cand, 1);
     pl.slots = wanted_slots(e, n_cand);
-    pl.chunk = std::max<int64_t>(std::min<int64_t>(n_cand, 8 * full_slots(e)), pl.slots);
+    pl.chunk = std::max<int64_t>(std::min<int64_t>(n_cand, 8 * full_slots(e)), 2 * pl.slots);
     return layout(e, pl) + 1024;
 }
 
