@@ -122,6 +122,8 @@ typedef struct {
     int64_t candidates;      /* candidates evaluated                                     */
     int64_t query_events;    /* candidates * sum over stages of queries visiting the stage */
     int64_t batches;         /* batches dispatched, all candidates, all stages           */
+    int64_t algorithmic_ops; /* integer operations the method needs: per batch R + max_batch + 4
+                                (replica min, queue count, table add, slot update), per query-event 3 */
     int64_t chunks;          /* how many (simulate, select) launch pairs the call made   */
     int64_t kernel_launches; /* kernels launched by the call                             */
     double  sim_ms;          /* device time of the simulation kernels (CUDA events)      */

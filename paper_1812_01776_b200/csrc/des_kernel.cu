@@ -65,6 +65,7 @@ des_kernel(const __grid_constant__ DesParams p)
     int64_t *my_time = p.ws_time + slot * p.slot_elems;
     int32_t *my_qid = p.ws_qid + slot * p.slot_elems;
     unsigned long long batches = 0;
+    unsigned long long alg_ops = 0;   // algorithmic integer operations: (R + mb + 4) per batch, 3 per query-event
 
     for (;;) {
         unsigned long long c = 0;
@@ -169,6 +170,8 @@ des_kernel(const __grid_constant__ DesParams p)
 
             int head = 0;
             int guard = 0;
+            const int ops_per_batch = R + mb + 4;
+            alg_ops += 3ull * (unsigned)n_in;
             while (head < n_in) {
                 const int64_t minfin = warp_min_i64(fin);
                 const int sel = pick(minfin);
@@ -192,6 +195,7 @@ des_kernel(const __grid_constant__ DesParams p)
                 seq_ctr++;
                 head += cnt;
                 batches++;
+                alg_ops += ops_per_batch;
                 if (++guard > n_in) {   // cannot happen: every batch takes >= 1 query
                     if (lane == 0) atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT);
                     break;
@@ -218,7 +222,7 @@ des_kernel(const __grid_constant__ DesParams p)
             if (exits != p.n) atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT);
         }
     }
-    if (lane == 0 && batches) atomicAdd(&p.counters[1], batches);
+    if (lane == 0 && batches) { atomicAdd(&p.counters[1], batches); atomicAdd(&p.counters[2], alg_ops); }
 }
 
 cudaError_t launch_des(const DesParams &p, int grid, size_t smem, cudaStream_t stream)

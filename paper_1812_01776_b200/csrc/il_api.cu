@@ -39,9 +39,9 @@ struct il_estimator {
     int64_t *d_arrival = nullptr;
     uint8_t *d_bits = nullptr;
     int32_t *d_lat = nullptr;
-    unsigned long long *d_counters = nullptr;   // [2]
+    unsigned long long *d_counters = nullptr;   // [4]
     int *d_status = nullptr;
-    unsigned long long *h_counters = nullptr;   // pinned: [2] counters, then the status word
+    unsigned long long *h_counters = nullptr;   // pinned: [4] counters, then the status word
     int *h_status = nullptr;
 
     void *user_ws = nullptr; size_t user_ws_bytes = 0;
@@ -304,10 +304,10 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     IL_CUDA_E(cudaMalloc(&e->d_arrival, (size_t)n * 8));
     IL_CUDA_E(cudaMalloc(&e->d_bits, (size_t)n));
     IL_CUDA_E(cudaMalloc(&e->d_lat, e->smem));
-    IL_CUDA_E(cudaMalloc(&e->d_counters, 2 * sizeof(unsigned long long)));
+    IL_CUDA_E(cudaMalloc(&e->d_counters, 4 * sizeof(unsigned long long)));
     IL_CUDA_E(cudaMalloc(&e->d_status, sizeof(int)));
-    IL_CUDA_E(cudaMallocHost(&e->h_counters, 4 * sizeof(unsigned long long)));
-    e->h_status = reinterpret_cast<int *>(e->h_counters + 2);
+    IL_CUDA_E(cudaMallocHost(&e->h_counters, 6 * sizeof(unsigned long long)));
+    e->h_status = reinterpret_cast<int *>(e->h_counters + 4);
     IL_CUDA_E(cudaMemcpy(e->d_arrival, tr->arrival_us, (size_t)n * 8, cudaMemcpyHostToDevice));
     if (tr->branch_bits) IL_CUDA_E(cudaMemcpy(e->d_bits, tr->branch_bits, (size_t)n, cudaMemcpyHostToDevice));
     else IL_CUDA_E(cudaMemset(e->d_bits, 0, (size_t)n));
@@ -417,7 +417,7 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
     if (rc) return rc;
 
     cudaStream_t st = e->stream;
-    IL_CUDA(cudaMemsetAsync(e->d_counters, 0, 2 * sizeof(unsigned long long), st));
+    IL_CUDA(cudaMemsetAsync(e->d_counters, 0, 4 * sizeof(unsigned long long), st));
     IL_CUDA(cudaMemsetAsync(e->d_status, 0, sizeof(int), st));
     IL_CUDA(cudaEventRecord(e->events[0], st));
 
@@ -448,7 +448,7 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
         launches += 2;
     }
     IL_CUDA(cudaEventRecord(e->events[1], st));
-    IL_CUDA(cudaMemcpyAsync(e->h_counters, e->d_counters, 2 * sizeof(unsigned long long),
+    IL_CUDA(cudaMemcpyAsync(e->h_counters, e->d_counters, 4 * sizeof(unsigned long long),
                             cudaMemcpyDeviceToHost, st));
     IL_CUDA(cudaMemcpyAsync(e->h_status, e->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
     IL_CUDA(cudaStreamSynchronize(st));
@@ -465,6 +465,7 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
     e->stats.candidates = n_cand;
     e->stats.query_events = n_cand * e->events_per_candidate;
     e->stats.batches = (int64_t)e->h_counters[1];
+    e->stats.algorithmic_ops = (int64_t)e->h_counters[2];
     e->stats.chunks = n_chunks;
     e->stats.kernel_launches = launches;
     return *e->h_status;

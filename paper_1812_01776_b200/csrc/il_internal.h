@@ -32,7 +32,7 @@ struct DesParams {
     int64_t *slab;                // [n_cand][slab_stride] exit latencies
     int64_t slab_stride;          // n rounded up to 32
     uint64_t *lat_or;             // [n_cand] OR of all latencies of the candidate
-    unsigned long long *counters; // [0] next candidate, [1] batches dispatched
+    unsigned long long *counters; // [0] next candidate, [1] batches dispatched, [2] algorithmic ops
     int *status;                  // first error seen by any warp (0 = none)
 };
 

@@ -57,7 +57,8 @@ class StageConfig(ctypes.Structure):
 
 class Stats(ctypes.Structure):
     _fields_ = [("candidates", ctypes.c_int64), ("query_events", ctypes.c_int64),
-                ("batches", ctypes.c_int64), ("chunks", ctypes.c_int64),
+                ("batches", ctypes.c_int64), ("algorithmic_ops", ctypes.c_int64),
+                ("chunks", ctypes.c_int64),
                 ("kernel_launches", ctypes.c_int64), ("sim_ms", ctypes.c_double),
                 ("select_ms", ctypes.c_double), ("total_ms", ctypes.c_double)]
 
