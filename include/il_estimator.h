@@ -71,6 +71,7 @@ extern "C" {
 #define IL_ERR_NOMEM         -6  /* host or device allocation failed / workspace too small */
 #define IL_ERR_CUDA          -7  /* a CUDA runtime call failed; see il_last_cuda_error     */
 #define IL_ERR_ITER_LIMIT    -8  /* a device loop hit its iteration bound (internal error) */
+#define IL_ERR_TOO_LARGE     -9  /* il_estimate_device_static: needs more than IL_STATIC_SCRATCH_BYTES */
 
 typedef struct il_estimator il_estimator;   /* opaque; owns its device copies */
 
@@ -172,6 +173,48 @@ IL_API int il_estimate(il_estimator *est, const il_stage_config *configs, int64_
  */
 IL_API int il_estimate_device(il_estimator *est, const il_stage_config *d_configs, int64_t n,
                               int64_t slo_us, int64_t *d_out_p99_us, int64_t *d_out_miss);
+
+/*
+ * Allocation-free variant of il_estimate_device (the paper has no counterpart;
+ * this is a deployment convenience of this library).
+ *
+ * Who needs it: a Planner that runs inside a serving process usually shares
+ * its GPU with a model server whose memory pool has already claimed the
+ * device's memory, so a cudaMalloc made by this library can fail there, and
+ * even when it succeeds it synchronises the whole device and stalls the
+ * inference kernels running next to it.  Such callers create the handle once
+ * at start-up (creation does allocate the device copies of trace and profiles)
+ * and afterwards use this call, which never calls cudaMalloc, cudaFree or any
+ * other allocating routine: the simulation kernel's scratch (inter-stage
+ * streams, latency slab, counters) lives in one static device array of
+ * IL_STATIC_SCRATCH_BYTES that is part of the library image, so every GPU that
+ * loads the library holds that much memory until the process exits.
+ *
+ * Arguments and results are those of il_estimate_device (DEVICE pointers,
+ * work on the handle's stream, returns after completion, same values bit for
+ * bit).  A workspace set with il_set_workspace is ignored, and il_get_stats is
+ * not updated.
+ *
+ * Limit: the whole batch is evaluated in one pass, with at most 32 warps
+ * resident, and must fit the array:
+ *     256 + 12 * slot * min(32, n rounded up to 4) + (8 * n_queries' + 8) * n
+ *         <= IL_STATIC_SCRATCH_BYTES
+ * where n_queries' is n_queries rounded up to 32 and slot is the number of
+ * stream elements one warp keeps between stages (for a linear pipeline about
+ * 2 * n_queries; never more than the query-events per candidate).  A larger
+ * request returns IL_ERR_TOO_LARGE and launches nothing; split the batch or use
+ * il_estimate_device.
+ *
+ * The first call on a device looks up the array's device address; make that
+ * first call during start-up, before any stream capture begins.  All calls, on
+ * all handles, share the one array: it keeps the previous call's contents (the
+ * call clears the counters it needs to start at zero), and two calls that
+ * overlap on the same GPU, from different handles or streams, race on it and
+ * give wrong results.  Serialise them.
+ */
+#define IL_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+IL_API int il_estimate_device_static(il_estimator *est, const il_stage_config *d_configs, int64_t n,
+                                     int64_t slo_us, int64_t *d_out_p99_us, int64_t *d_out_miss);
 
 /* Stream all later calls on this handle use (a cudaStream_t passed as void*;
  * NULL = the default stream).  The stream stays the caller's. */

@@ -200,6 +200,16 @@ int ensure_events(il_estimator *e, size_t count)
 
 }  // namespace
 
+void il::bound_view(const il_estimator *e, BoundView *out)
+{
+    out->base = e->base;
+    out->S = e->S;
+    out->n = e->n; out->n_pad = e->n_pad; out->slot_elems = e->slot_elems;
+    out->smem = e->smem;
+    out->device = e->device;
+    out->stream = e->stream;
+}
+
 extern "C" {
 
 const char *il_strerror(int code)
@@ -214,6 +224,7 @@ const char *il_strerror(int code)
     case IL_ERR_NOMEM: return "out of memory or workspace too small";
     case IL_ERR_CUDA: return "CUDA call failed";
     case IL_ERR_ITER_LIMIT: return "device loop exceeded its iteration bound";
+    case IL_ERR_TOO_LARGE: return "request needs more than the built-in static scratch (IL_STATIC_SCRATCH_BYTES)";
     default: return "unknown error";
     }
 }

@@ -47,6 +47,18 @@ struct SelectParams {
     int64_t *out_miss;
 };
 
+// Read-only view of what a handle has bound, for translation units that do not
+// see the handle's definition.
+struct BoundView {
+    DesParams base;        // bound-input part of the kernel parameters
+    int32_t S;
+    int64_t n, n_pad, slot_elems;
+    size_t smem;
+    int device;
+    cudaStream_t stream;
+};
+void bound_view(const il_estimator *est, BoundView *out);
+
 cudaError_t launch_des(const DesParams &p, int grid, size_t smem, cudaStream_t stream);
 cudaError_t launch_select(const SelectParams &p, cudaStream_t stream);
 int des_max_ctas_per_sm(size_t smem);

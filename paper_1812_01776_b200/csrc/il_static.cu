@@ -1,0 +1,103 @@
+// il_estimate_device_static: the estimate call for processes that must not
+// allocate device memory after start-up.  The scratch the simulation kernel
+// needs (inter-stage streams, latency slab, counters) is a static device array
+// that is part of this library's image; nothing here calls cudaMalloc, cudaFree
+// or any other allocating routine.
+#include "il_internal.h"
+
+#include <algorithm>
+#include <mutex>
+
+using namespace il;
+
+namespace {
+
+// The scratch itself.  In host code this name is only a handle for the runtime's
+// symbol lookup, not a device address: the address is fetched per device below.
+static __device__ __align__(256) unsigned char g_static_scratch[IL_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+constexpr int kMaxStaticSlots = 32;      // warps resident in the static variant
+constexpr size_t kHeaderBytes = 256;     // counters (4 x u64) at 0, status word at 64
+
+std::mutex g_mutex;
+unsigned char *g_scratch_addr[kMaxDevices] = {};
+
+// Device address of the array on `dev`, which must be the current device.
+// Looked up once per device.
+cudaError_t scratch_address(int dev, unsigned char **out)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (!g_scratch_addr[dev]) {
+        void *ptr = nullptr;
+        cudaError_t ce = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (ce != cudaSuccess) return ce;
+        g_scratch_addr[dev] = static_cast<unsigned char *>(ptr);
+    }
+    *out = g_scratch_addr[dev];
+    return cudaSuccess;
+}
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+extern "C" int il_estimate_device_static(il_estimator *est, const il_stage_config *d_configs,
+                                         int64_t n_cand, int64_t slo_us, int64_t *d_out_p99,
+                                         int64_t *d_out_miss)
+{
+    if (!est || n_cand < 0) return IL_ERR_INVALID_ARG;
+    if (n_cand == 0) return IL_OK;
+    if (!d_configs || !d_out_p99 || !d_out_miss) return IL_ERR_INVALID_ARG;
+    BoundView v;
+    bound_view(est, &v);
+    if (v.device < 0 || v.device >= kMaxDevices) return IL_ERR_INVALID_ARG;
+
+    // does the request fit the array?
+    const int64_t slots = std::min<int64_t>(kMaxStaticSlots,
+                                            (n_cand + kWarpsPerCta - 1) / kWarpsPerCta * kWarpsPerCta);
+    size_t off = kHeaderBytes;
+    const size_t off_time = off; off = align_up(off + (size_t)slots * v.slot_elems * 8, 256);
+    const size_t off_qid = off;  off = align_up(off + (size_t)slots * v.slot_elems * 4, 256);
+    const size_t off_slab = off;
+    // guard the multiplication before it can wrap
+    if ((size_t)n_cand > IL_STATIC_SCRATCH_BYTES / 8 || (size_t)v.n_pad > IL_STATIC_SCRATCH_BYTES / 8)
+        return IL_ERR_TOO_LARGE;
+    off = align_up(off + (size_t)n_cand * v.n_pad * 8, 256);
+    const size_t off_or = off;   off = align_up(off + (size_t)n_cand * 8, 256);
+    if (off > IL_STATIC_SCRATCH_BYTES) return IL_ERR_TOO_LARGE;
+
+    if (cudaSetDevice(v.device) != cudaSuccess) return IL_ERR_CUDA;
+    unsigned char *base = nullptr;
+    if (scratch_address(v.device, &base) != cudaSuccess) return IL_ERR_CUDA;
+
+    cudaStream_t st = v.stream;
+    // the array keeps the last call's contents: the work counter, the batch
+    // counters and the status word must start at zero
+    if (cudaMemsetAsync(base, 0, kHeaderBytes, st) != cudaSuccess) return IL_ERR_CUDA;
+
+    DesParams p = v.base;
+    p.counters = reinterpret_cast<unsigned long long *>(base);
+    p.status = reinterpret_cast<int *>(base + 64);
+    p.configs = d_configs;
+    p.n_cand = n_cand;
+    p.slot_elems = v.slot_elems;
+    p.ws_time = reinterpret_cast<int64_t *>(base + off_time);
+    p.ws_qid = reinterpret_cast<int32_t *>(base + off_qid);
+    p.slab = reinterpret_cast<int64_t *>(base + off_slab);
+    p.slab_stride = v.n_pad;
+    p.lat_or = reinterpret_cast<uint64_t *>(base + off_or);
+    if (launch_des(p, (int)(slots / kWarpsPerCta), v.smem, st) != cudaSuccess) return IL_ERR_CUDA;
+
+    SelectParams sp;
+    sp.slab = p.slab; sp.slab_stride = v.n_pad; sp.lat_or = p.lat_or;
+    sp.n = (int32_t)v.n; sp.n_cand = n_cand; sp.slo_us = slo_us;
+    sp.out_p99 = d_out_p99; sp.out_miss = d_out_miss;
+    if (launch_select(sp, st) != cudaSuccess) return IL_ERR_CUDA;
+
+    int status = 0;
+    if (cudaMemcpyAsync(&status, p.status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return IL_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return IL_ERR_CUDA;
+    return status;
+}

@@ -21,11 +21,13 @@ _lib = None
 IL_OK = 0
 IL_ERR_INVALID_ARG, IL_ERR_BAD_TOPOLOGY, IL_ERR_BAD_PROFILE, IL_ERR_BAD_TRACE = -1, -2, -3, -4
 IL_ERR_BAD_CONFIG, IL_ERR_NOMEM, IL_ERR_CUDA, IL_ERR_ITER_LIMIT = -5, -6, -7, -8
+IL_ERR_TOO_LARGE = -9
+IL_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 EXPORTS = ["il_estimator_create", "il_estimator_destroy", "il_estimate", "il_estimate_device",
            "il_set_stream", "il_workspace_bytes", "il_workspace_min_bytes", "il_set_workspace",
            "il_get_stats", "il_stage_visits", "il_strerror", "il_last_cuda_error",
-           "il_measure_int_issue"]
+           "il_measure_int_issue", "il_estimate_device_static"]
 
 
 class ILError(RuntimeError):
@@ -89,6 +91,8 @@ def load_library():
     lib.il_estimate.argtypes = [vp, vp, i64, i64, vp, vp]
     lib.il_estimate_device.restype = ctypes.c_int
     lib.il_estimate_device.argtypes = [vp, vp, i64, i64, vp, vp]
+    lib.il_estimate_device_static.restype = ctypes.c_int
+    lib.il_estimate_device_static.argtypes = [vp, vp, i64, i64, vp, vp]
     lib.il_set_stream.restype = ctypes.c_int
     lib.il_set_stream.argtypes = [vp, vp]
     lib.il_workspace_bytes.restype = ctypes.c_int
@@ -174,6 +178,15 @@ def il_estimate_device(handle, d_configs: int, n: int, slo_us: int, d_out_p99: i
     """il_estimate_device: raw device pointers (ints) in, results written in place."""
     _check(load_library().il_estimate_device(handle, d_configs, int(n), int(slo_us), d_out_p99,
                                              d_out_miss), "il_estimate_device")
+
+
+def il_estimate_device_static(handle, d_configs: int, n: int, slo_us: int, d_out_p99: int,
+                              d_out_miss: int) -> None:
+    """il_estimate_device_static: like il_estimate_device, but the library
+    allocates nothing; scratch is the static array built into the library."""
+    _check(load_library().il_estimate_device_static(handle, d_configs, int(n), int(slo_us),
+                                                    d_out_p99, d_out_miss),
+           "il_estimate_device_static")
 
 
 def il_set_stream(handle, cuda_stream: int) -> None:
