@@ -201,8 +201,8 @@ def run_cuda(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    per_rank = workloads.FULL_SIZES[WORKLOAD_ID][1]
-    w = workloads.make(WORKLOAD_ID, n_candidates=per_rank * world)
+    per_rank = args.candidates or workloads.FULL_SIZES[WORKLOAD_ID][1]
+    w = workloads.make(WORKLOAD_ID, n_queries=args.queries, n_candidates=per_rank * world)
     lo, hi = shard_range(w.n_candidates, rank, world)
     cfg_host = np.ascontiguousarray(w.configs[lo:hi])
     n_cand = hi - lo
@@ -267,7 +267,7 @@ def run_cuda(args):
         one_step_e2e()
         barrier()
         e2e_ms = []
-        for _ in range(args.steps):
+        for _ in range(1 if args.no_e2e else args.steps):
             ms, p99_h, miss_h = one_step_e2e()
             e2e_ms.append(ms)
         barrier()
@@ -286,7 +286,7 @@ def run_cuda(args):
     K = args.steps
     cand_total = n_cand * world
     value = cand_total * K / (total_ms * 1e-3)
-    e2e_value = cand_total * K / (e2e_total * 1e-3)
+    e2e_value = cand_total * (1 if args.no_e2e else K) / (e2e_total * 1e-3)
     peaks, peaks_kind = load_measured_peaks()
     sim_avg_s = (sum(sim_ms) / K) * 1e-3
     # integer-issue roofline of the simulation kernel (the dominant one)
@@ -303,7 +303,8 @@ def run_cuda(args):
         "warmup": args.warmup, "ms_per_step": total_ms / K, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
         "config": {"workload": "config2: linear 4-stage image pipeline, 50,000 gamma arrivals "
-                               "(200 qps, CV 4), 4,096 candidates per GPU",
+                               "(200 qps, CV 4), 4,096 candidates per GPU"
+                               + ("" if not (args.candidates or args.queries) else " [REDUCED for profiling]"),
                    "candidates_per_gpu": n_cand, "queries": n, "stages": S,
                    "query_events_per_candidate": events_per_cand,
                    "l2": "256 MiB buffer written between steps; working set "
@@ -348,6 +349,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--candidates", type=int, default=None,
+                    help="candidates per GPU (default: the workload's 4,096); smaller values are "
+                         "for profiler captures, not for reported numbers")
+    ap.add_argument("--queries", type=int, default=None,
+                    help="trace length (default: the workload's 50,000); for profiler captures")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer timing (profiler captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
