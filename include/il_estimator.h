@@ -239,6 +239,18 @@ IL_API int il_workspace_bytes(const il_estimator *est, int64_t n_candidates, siz
 IL_API int il_workspace_min_bytes(const il_estimator *est, size_t *bytes);
 IL_API int il_set_workspace(il_estimator *est, void *d_workspace, size_t bytes);
 
+/*
+ * Chooses the simulation kernel.  IL_VARIANT_AUTO (default) uses the
+ * packed-record kernel whenever every time the simulation can reach (last
+ * arrival + sum over stages of n * largest table entry) fits in
+ * 63 - max(5, ceil(log2 n)) bits, and the kernel with separate 64-bit time and
+ * 32-bit query streams otherwise.  IL_VARIANT_WIDE forces the latter (it is
+ * always valid; used to test it).  Both give identical results.
+ */
+#define IL_VARIANT_AUTO 0
+#define IL_VARIANT_WIDE 1
+IL_API int il_set_variant(il_estimator *est, int variant);
+
 /* Counters of the last estimate call on this handle. */
 IL_API int il_get_stats(const il_estimator *est, il_stats *out);
 

@@ -37,6 +37,10 @@ struct il_estimator {
     int64_t slot_elems = 0;
 
     int64_t *d_arrival = nullptr;
+    uint64_t *d_ptrace = nullptr;      // packed root stream
+    bool can_pack = false;             // every reachable time fits a packed record
+    int variant = IL_VARIANT_AUTO;
+    int ctas_per_sm_wide = 0, ctas_per_sm_packed = 0;
     uint8_t *d_bits = nullptr;
     int32_t *d_lat = nullptr;
     unsigned long long *d_counters = nullptr;   // [4]
@@ -179,9 +183,14 @@ int64_t plan_stream_buffers(const il_profiles *pr, const int64_t *visits, int32_
     return top;
 }
 
+bool use_packed(const il_estimator *e)
+{
+    return e->can_pack && e->variant != IL_VARIANT_WIDE;
+}
+
 void free_device(il_estimator *e)
 {
-    cudaFree(e->d_arrival); cudaFree(e->d_bits); cudaFree(e->d_lat);
+    cudaFree(e->d_arrival); cudaFree(e->d_ptrace); cudaFree(e->d_bits); cudaFree(e->d_lat);
     cudaFree(e->d_counters); cudaFree(e->d_status);
     cudaFree(e->own_ws); cudaFree(e->d_cfg); cudaFree(e->d_out);
     if (e->h_counters) cudaFreeHost(e->h_counters);
@@ -203,6 +212,7 @@ int ensure_events(il_estimator *e, size_t count)
 void il::bound_view(const il_estimator *e, BoundView *out)
 {
     out->base = e->base;
+    out->packed = use_packed(e);
     out->S = e->S;
     out->n = e->n; out->n_pad = e->n_pad; out->slot_elems = e->slot_elems;
     out->smem = e->smem;
@@ -262,6 +272,9 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     for (int64_t i = 1; i < n; i++)
         if (tr->arrival_us[i] < tr->arrival_us[i - 1]) return IL_ERR_BAD_TRACE;
     if (tr->arrival_us[n - 1] > (INT64_C(1) << 62) - worst) return IL_ERR_BAD_TRACE;
+    int qbits = 5;                       // bits of a packed record that hold the query index
+    while ((INT64_C(1) << qbits) < n) qbits++;
+    const bool can_pack = tr->arrival_us[n - 1] + worst < (INT64_C(1) << (63 - qbits));
 
     int dev = 0;
     cudaDeviceProp prop;
@@ -314,6 +327,15 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
 
     IL_CUDA_E(cudaMalloc(&e->d_arrival, (size_t)n * 8));
     IL_CUDA_E(cudaMalloc(&e->d_bits, (size_t)n));
+    e->can_pack = can_pack;
+    bp.qbits = qbits;
+    if (can_pack) {
+        std::vector<uint64_t> packed((size_t)n);
+        for (int64_t i = 0; i < n; i++)
+            packed[(size_t)i] = ((uint64_t)tr->arrival_us[i] << qbits) | (uint64_t)i;
+        IL_CUDA_E(cudaMalloc(&e->d_ptrace, (size_t)n * 8));
+        IL_CUDA_E(cudaMemcpy(e->d_ptrace, packed.data(), (size_t)n * 8, cudaMemcpyHostToDevice));
+    }
     IL_CUDA_E(cudaMalloc(&e->d_lat, e->smem));
     IL_CUDA_E(cudaMalloc(&e->d_counters, 4 * sizeof(unsigned long long)));
     IL_CUDA_E(cudaMalloc(&e->d_status, sizeof(int)));
@@ -324,11 +346,13 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     else IL_CUDA_E(cudaMemset(e->d_bits, 0, (size_t)n));
     IL_CUDA_E(cudaMemcpy(e->d_lat, pr->latency_us, e->smem, cudaMemcpyHostToDevice));
 #undef IL_CUDA_E
-    bp.arrival = e->d_arrival; bp.bits = e->d_bits; bp.lat = e->d_lat;
+    bp.arrival = e->d_arrival; bp.bits = e->d_bits; bp.lat = e->d_lat; bp.ptrace = e->d_ptrace;
     bp.counters = e->d_counters; bp.status = e->d_status;
 
-    e->ctas_per_sm = des_max_ctas_per_sm(e->smem);
-    if (e->ctas_per_sm < 1) return fail(IL_ERR_CUDA);
+    e->ctas_per_sm_wide = des_max_ctas_per_sm(e->smem);
+    e->ctas_per_sm_packed = des_packed_max_ctas_per_sm(e->smem);
+    if (e->ctas_per_sm_wide < 1 || e->ctas_per_sm_packed < 1) return fail(IL_ERR_CUDA);
+    e->ctas_per_sm = use_packed(e) ? e->ctas_per_sm_packed : e->ctas_per_sm_wide;
     *out = e;
     return IL_OK;
 }
@@ -348,6 +372,14 @@ int il_set_stream(il_estimator *e, void *cuda_stream)
 {
     if (!e) return IL_ERR_INVALID_ARG;
     e->stream = static_cast<cudaStream_t>(cuda_stream);
+    return IL_OK;
+}
+
+int il_set_variant(il_estimator *e, int variant)
+{
+    if (!e || (variant != IL_VARIANT_AUTO && variant != IL_VARIANT_WIDE)) return IL_ERR_INVALID_ARG;
+    e->variant = variant;
+    e->ctas_per_sm = use_packed(e) ? e->ctas_per_sm_packed : e->ctas_per_sm_wide;
     return IL_OK;
 }
 
@@ -448,7 +480,7 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
         if (ch > 0) IL_CUDA(cudaMemsetAsync(e->d_counters, 0, sizeof(unsigned long long), st));
         const int64_t ctas = std::min<int64_t>(pl.slots / kWarpsPerCta, (cnt + kWarpsPerCta - 1) / kWarpsPerCta);
         IL_CUDA(cudaEventRecord(e->events[2 + 3 * ch], st));
-        IL_CUDA(launch_des(p, (int)ctas, e->smem, st));
+        IL_CUDA(launch_simulation(p, use_packed(e), (int)ctas, e->smem, st));
         IL_CUDA(cudaEventRecord(e->events[3 + 3 * ch], st));
         SelectParams sp;
         sp.slab = p.slab; sp.slab_stride = e->n_pad; sp.lat_or = p.lat_or;

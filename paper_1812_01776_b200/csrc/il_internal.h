@@ -16,6 +16,8 @@ struct DesParams {
     const int64_t *arrival;       // [n]
     const uint8_t *bits;          // [n]
     const int32_t *lat;           // [S][H][Bmax]
+    const uint64_t *ptrace;       // [n] packed root stream (arrival << qbits) | index; packed kernel only
+    int32_t qbits;                // bits of a packed record that hold the query index
     int32_t S, H, Bmax;
     int32_t n;                    // queries
     int32_t n_s[IL_MAX_STAGES];   // queries visiting stage s
@@ -51,6 +53,7 @@ struct SelectParams {
 // see the handle's definition.
 struct BoundView {
     DesParams base;        // bound-input part of the kernel parameters
+    bool packed;           // which simulation kernel the handle uses
     int32_t S;
     int64_t n, n_pad, slot_elems;
     size_t smem;
@@ -60,6 +63,13 @@ struct BoundView {
 void bound_view(const il_estimator *est, BoundView *out);
 
 cudaError_t launch_des(const DesParams &p, int grid, size_t smem, cudaStream_t stream);
+cudaError_t launch_des_packed(const DesParams &p, int grid, size_t smem, cudaStream_t stream);
+int des_packed_max_ctas_per_sm(size_t smem);
+inline cudaError_t launch_simulation(const DesParams &p, bool packed, int grid, size_t smem,
+                                     cudaStream_t stream)
+{
+    return packed ? launch_des_packed(p, grid, smem, stream) : launch_des(p, grid, smem, stream);
+}
 cudaError_t launch_select(const SelectParams &p, cudaStream_t stream);
 int des_max_ctas_per_sm(size_t smem);
 cudaError_t launch_int_issue(unsigned *sink, int grid, int iters, cudaStream_t stream);

@@ -87,7 +87,8 @@ extern "C" int il_estimate_device_static(il_estimator *est, const il_stage_confi
     p.slab = reinterpret_cast<int64_t *>(base + off_slab);
     p.slab_stride = v.n_pad;
     p.lat_or = reinterpret_cast<uint64_t *>(base + off_or);
-    if (launch_des(p, (int)(slots / kWarpsPerCta), v.smem, st) != cudaSuccess) return IL_ERR_CUDA;
+    if (launch_simulation(p, v.packed, (int)(slots / kWarpsPerCta), v.smem, st) != cudaSuccess)
+        return IL_ERR_CUDA;
 
     SelectParams sp;
     sp.slab = p.slab; sp.slab_stride = v.n_pad; sp.lat_or = p.lat_or;

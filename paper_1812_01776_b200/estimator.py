@@ -22,12 +22,13 @@ IL_OK = 0
 IL_ERR_INVALID_ARG, IL_ERR_BAD_TOPOLOGY, IL_ERR_BAD_PROFILE, IL_ERR_BAD_TRACE = -1, -2, -3, -4
 IL_ERR_BAD_CONFIG, IL_ERR_NOMEM, IL_ERR_CUDA, IL_ERR_ITER_LIMIT = -5, -6, -7, -8
 IL_ERR_TOO_LARGE = -9
+IL_VARIANT_AUTO, IL_VARIANT_WIDE = 0, 1
 IL_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 EXPORTS = ["il_estimator_create", "il_estimator_destroy", "il_estimate", "il_estimate_device",
            "il_set_stream", "il_workspace_bytes", "il_workspace_min_bytes", "il_set_workspace",
            "il_get_stats", "il_stage_visits", "il_strerror", "il_last_cuda_error",
-           "il_measure_int_issue", "il_estimate_device_static"]
+           "il_measure_int_issue", "il_estimate_device_static", "il_set_variant"]
 
 
 class ILError(RuntimeError):
@@ -93,6 +94,8 @@ def load_library():
     lib.il_estimate_device.argtypes = [vp, vp, i64, i64, vp, vp]
     lib.il_estimate_device_static.restype = ctypes.c_int
     lib.il_estimate_device_static.argtypes = [vp, vp, i64, i64, vp, vp]
+    lib.il_set_variant.restype = ctypes.c_int
+    lib.il_set_variant.argtypes = [vp, ctypes.c_int]
     lib.il_set_stream.restype = ctypes.c_int
     lib.il_set_stream.argtypes = [vp, vp]
     lib.il_workspace_bytes.restype = ctypes.c_int
@@ -187,6 +190,10 @@ def il_estimate_device_static(handle, d_configs: int, n: int, slo_us: int, d_out
     _check(load_library().il_estimate_device_static(handle, d_configs, int(n), int(slo_us),
                                                     d_out_p99, d_out_miss),
            "il_estimate_device_static")
+
+
+def il_set_variant(handle, variant: int) -> None:
+    _check(load_library().il_set_variant(handle, int(variant)), "il_set_variant")
 
 
 def il_set_stream(handle, cuda_stream: int) -> None:
@@ -287,6 +294,10 @@ class Estimator:
                 self._ws = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
             il_set_workspace(self._h, self._ws.data_ptr(), self._ws.numel())
         return self._ws.numel()
+
+    def set_variant(self, variant: int) -> None:
+        """IL_VARIANT_AUTO or IL_VARIANT_WIDE (see il_set_variant)."""
+        il_set_variant(self._h, variant)
 
     def use_current_stream(self) -> None:
         il_set_stream(self._h, self._torch.cuda.current_stream(self.device).cuda_stream)

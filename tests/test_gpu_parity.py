@@ -21,11 +21,12 @@ def il():
     return il_
 
 
-def gpu_run(il, w, configs=None, slo=None, host=True, ws_bytes=None):
+def gpu_run(il, w, configs=None, slo=None, host=True, ws_bytes=None, variant=0):
     import torch
     configs = w.configs if configs is None else configs
     slo = w.slo_us if slo is None else slo
     with il.Estimator.from_workload(w) as est:
+        est.set_variant(variant)
         if ws_bytes is not None:
             est.reserve_workspace(len(configs), max_bytes=ws_bytes)
         if host:
@@ -63,13 +64,14 @@ def test_hand_traces(il, case):
     assert (int(p99[0]), int(miss[0])) == (case["p99_us"], case["miss"])
 
 
+@pytest.mark.parametrize("variant", [0, 1], ids=["packed", "wide"])
 @pytest.mark.parametrize("seed", range(12))
-def test_random_small(il, oracle, seed):
+def test_random_small(il, oracle, seed, variant):
     w = workloads.random_small(seed, S=1 + seed % 6, H=3, Bmax=[4, 33, 64][seed % 3], n=700 + 37 * seed,
                                C=40, max_replicas=[3, 8, 32][seed % 3], tree=(seed % 2 == 1),
                                qps=400.0, cv=3.0, lat_lo=1, lat_hi=20000,
                                equal_stamp_every=(3 if seed % 4 == 0 else 0))
-    check(il, oracle, w, host=(seed % 2 == 0))
+    check(il, oracle, w, host=(seed % 2 == 0), variant=variant)
 
 
 def test_config1_full(il, oracle):
@@ -77,9 +79,21 @@ def test_config1_full(il, oracle):
     assert st["batches"] > 0 and st["kernel_launches"] == 2 * st["chunks"]
 
 
+@pytest.mark.parametrize("variant", [0, 1], ids=["packed", "wide"])
 @pytest.mark.parametrize("cid,n,C", [(2, 5000, 300), (3, 6001, 200), (4, 3000, 150), (5, 4097, 260)])
-def test_configs_reduced(il, oracle, cid, n, C):
-    check(il, oracle, workloads.make(cid, n_queries=n, n_candidates=C), host=False)
+def test_configs_reduced(il, oracle, cid, n, C, variant):
+    check(il, oracle, workloads.make(cid, n_queries=n, n_candidates=C), host=False, variant=variant)
+
+
+def test_times_too_large_to_pack_fall_back_to_wide_kernel(il, oracle):
+    """Arrival stamps near 2^58 leave no room for the query index in a 64-bit
+    record: the library must pick the kernel with separate time and query
+    streams on its own, with the same results as for the unshifted trace."""
+    w = workloads.make(3, n_queries=3000, n_candidates=64)
+    exp = oracle.estimate_workload(w)
+    w.arrival_us = w.arrival_us + (1 << 58)
+    p99, miss, _ = gpu_run(il, w)
+    assert np.array_equal(p99, exp[0]) and np.array_equal(miss, exp[1])
 
 
 def test_multi_chunk_small_workspace(il, oracle):
