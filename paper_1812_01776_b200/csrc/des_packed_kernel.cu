@@ -186,6 +186,86 @@ __device__ __forceinline__ int run_stage(const DesParams &p, const WarpCtx &w, c
     return nbatch;
 }
 
+// A stage whose max batch is 1.  Every batch is a single query with the same
+// service time D = latency[1], so the multi-replica FIFO queue behaves like R
+// interleaved single-server queues: query i starts at
+//     s_i = max(a_i, s_{i-R} + D)
+// and queries leave in arrival order.  Unrolled, s_i is a running maximum of
+// a_{i-jR} + j D over j, which 32 lanes evaluate for 32 consecutive queries
+// with log2(32/R) shuffle steps plus one carry from the previous 32.
+template <int KIND>
+__device__ __forceinline__ int run_stage_mb1(const DesParams &p, const WarpCtx &w, const int32_t *row,
+                                             const int R, const int n_in, const uint64_t *in,
+                                             uint64_t *out_a, uint64_t *out_b, const int bit,
+                                             const bool a_exit, const bool b_exit,
+                                             int64_t *__restrict__ slab, int &exits, uint64_t &lat_or)
+{
+    const unsigned full = 0xffffffffu;
+    const int lane = w.lane;
+    const uint32_t qmask = w.qmask;
+    const int qb = w.qbits;
+    const int64_t D = row[0];
+    const int64_t kLongAgo = -(INT64_C(1) << 62);
+    // where in the previous 32 starts the chain of this lane continues, and how many services lie between
+    const int hops = lane / R + 1;
+    const int carry_src = 32 + lane - hops * R;
+    const int64_t carry_add = (int64_t)hops * D;
+    int64_t prev = kLongAgo;            // start times of the previous 32 queries
+    int tail_a = 0, tail_b = 0;
+
+    uint64_t rec = ld_rec(in, lane, n_in);
+    for (int base = 0; base < n_in; base += 32) {
+        const uint64_t cur = rec;
+        rec = ld_rec(in, base + 32 + lane, n_in);          // next 32, off the dependent chain
+        const bool act = base + lane < n_in;
+        int64_t v = act ? (int64_t)(cur >> qb) : (INT64_C(1) << 62);
+        int64_t mul = D;
+        for (int d = R; d < 32; d <<= 1, mul <<= 1) {
+            const int64_t u = __shfl_up_sync(full, v, d);
+            if (lane >= d && u + mul > v) v = u + mul;
+        }
+        const int64_t c = __shfl_sync(full, prev, carry_src) + carry_add;
+        if (c > v) v = c;
+        prev = v;
+        const int64_t fin = v + D;
+        const uint32_t q = (uint32_t)cur & qmask;
+        const uint64_t orec = ((uint64_t)fin << qb) | q;
+        if (KIND == kForward) {
+            if (act) out_a[base + lane] = orec;
+        } else if (KIND == kExit) {
+            if (act) {
+                const int64_t l = fin - p.arrival[q];
+                slab[exits + base + lane] = l;
+                lat_or |= (uint64_t)l;
+            }
+        } else {
+            bool bitv = false;
+            if (act) bitv = (p.bits[q] >> bit) & 1;
+            const unsigned ma = __ballot_sync(full, act && !bitv);
+            const unsigned mb_ = __ballot_sync(full, act && bitv);
+            const bool to_exit = bitv ? b_exit : a_exit;
+            if (act) {
+                if (to_exit) {
+                    const unsigned me = (a_exit ? ma : 0u) | (b_exit ? mb_ : 0u);
+                    const int64_t l = fin - p.arrival[q];
+                    slab[exits + __popc(me & w.lt_mask)] = l;
+                    lat_or |= (uint64_t)l;
+                } else if (bitv) {
+                    out_b[tail_b + __popc(mb_ & w.lt_mask)] = orec;
+                } else {
+                    out_a[tail_a + __popc(ma & w.lt_mask)] = orec;
+                }
+            }
+            const int na = __popc(ma), nb = __popc(mb_);
+            exits += (a_exit ? na : 0) + (b_exit ? nb : 0);
+            tail_a += a_exit ? 0 : na;
+            tail_b += b_exit ? 0 : nb;
+        }
+    }
+    if (KIND == kExit) exits += n_in;
+    return n_in;
+}
+
 }  // namespace
 
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
@@ -244,7 +324,14 @@ des_packed_kernel(const __grid_constant__ DesParams p)
 #define IL_STAGE(WIDE_, KIND_)                                                               \
     nb = run_stage<WIDE_, KIND_>(p, w, row, mb, R, n_in, in, out_a, out_b, bit, da < 0, db < 0, \
                                  slab, exits, lat_or, p.status)
-            if (mb > 32) {
+            if (mb == 1) {
+                if (kind == kForward)
+                    nb = run_stage_mb1<kForward>(p, w, row, R, n_in, in, out_a, out_b, bit, da < 0, db < 0, slab, exits, lat_or);
+                else if (kind == kExit)
+                    nb = run_stage_mb1<kExit>(p, w, row, R, n_in, in, out_a, out_b, bit, da < 0, db < 0, slab, exits, lat_or);
+                else
+                    nb = run_stage_mb1<kBranch>(p, w, row, R, n_in, in, out_a, out_b, bit, da < 0, db < 0, slab, exits, lat_or);
+            } else if (mb > 32) {
                 if (kind == kForward) IL_STAGE(true, kForward);
                 else if (kind == kExit) IL_STAGE(true, kExit);
                 else IL_STAGE(true, kBranch);
