@@ -484,6 +484,7 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
         IL_CUDA(cudaEventRecord(e->events[3 + 3 * ch], st));
         SelectParams sp;
         sp.slab = p.slab; sp.slab_stride = e->n_pad; sp.lat_or = p.lat_or;
+        sp.arrival = e->d_arrival; sp.qbits = p.qbits; sp.packed = use_packed(e) ? 1 : 0;
         sp.n = (int32_t)e->n; sp.n_cand = cnt; sp.slo_us = slo_us;
         sp.out_p99 = d_out_p99 + lo; sp.out_miss = d_out_miss + lo;
         IL_CUDA(launch_select(sp, st));

@@ -39,8 +39,11 @@ struct DesParams {
 };
 
 struct SelectParams {
-    const int64_t *slab;          // [n_cand][slab_stride]
+    int64_t *slab;                // [n_cand][slab_stride]: latencies, or packed (finish, query) records
     int64_t slab_stride;
+    const int64_t *arrival;       // [n], to turn packed records into latencies
+    int32_t qbits;
+    int32_t packed;               // slab holds packed records (from the packed simulation kernel)
     const uint64_t *lat_or;       // [n_cand]
     int32_t n;
     int64_t n_cand;

@@ -8,6 +8,10 @@
 // far, then descends into the bucket that holds rank k.  Digits above the
 // highest set bit of any latency (known from the simulation kernel's OR) are
 // skipped.  One CTA per candidate.
+//
+// When the slab comes from the packed-record simulation kernel it holds
+// (finish time, query) records; a first sweep replaces each by
+// latency = finish - arrival[query], ORs the latencies and counts the misses.
 #include "il_internal.h"
 
 namespace il {
@@ -19,10 +23,37 @@ select_kernel(const __grid_constant__ SelectParams p)
     __shared__ unsigned long long s_prefix;
     __shared__ unsigned s_rank;
     __shared__ unsigned s_miss;
+    __shared__ unsigned long long s_or;
 
     for (int64_t c = blockIdx.x; c < p.n_cand; c += gridDim.x) {
-        const int64_t *lat = p.slab + c * p.slab_stride;
-        const uint64_t bits_used = p.lat_or[c];
+        int64_t *lat = p.slab + c * p.slab_stride;
+        unsigned miss = 0;
+        bool counted_miss = false;
+        uint64_t bits_used;
+        if (p.packed) {
+            if (threadIdx.x == 0) s_or = 0;
+            __syncthreads();
+            const uint64_t qmask = (1ull << p.qbits) - 1ull;
+            unsigned long long my_or = 0;
+            for (int i = threadIdx.x; i < p.n; i += kSelectThreads) {
+                const uint64_t rec = (uint64_t)lat[i];
+                const int64_t l = (int64_t)(rec >> p.qbits) - p.arrival[rec & qmask];
+                lat[i] = l;
+                my_or |= (unsigned long long)l;
+                miss += (l > p.slo_us);
+            }
+            counted_miss = true;
+            my_or |= __shfl_xor_sync(0xffffffffu, my_or, 16);
+            my_or |= __shfl_xor_sync(0xffffffffu, my_or, 8);
+            my_or |= __shfl_xor_sync(0xffffffffu, my_or, 4);
+            my_or |= __shfl_xor_sync(0xffffffffu, my_or, 2);
+            my_or |= __shfl_xor_sync(0xffffffffu, my_or, 1);
+            if ((threadIdx.x & 31) == 0 && my_or) atomicOr(&s_or, my_or);
+            __syncthreads();   // also orders the latency writes before the passes below
+            bits_used = s_or;
+        } else {
+            bits_used = p.lat_or[c];
+        }
         int top = 0;                                   // number of 8-bit digits that matter
         while (top < 8 && (bits_used >> (8 * top)) != 0) top++;
 
@@ -31,8 +62,6 @@ select_kernel(const __grid_constant__ SelectParams p)
             s_rank = (unsigned)((99ll * p.n + 99) / 100);   // 1-indexed rank still to find
             s_miss = 0;
         }
-        unsigned miss = 0;
-        bool counted_miss = false;
         __syncthreads();
 
         for (int d = top - 1; d >= 0; d--) {
