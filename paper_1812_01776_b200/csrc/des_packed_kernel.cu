@@ -19,17 +19,18 @@
 //     percentile kernel turns them into latencies;
 //   * a replica slot is ONE 64-bit key  (finish << q) | head-index-at-dispatch.
 //     The head index grows with every dispatch, so the key is unique and its
-//     unsigned order is exactly (finish, dispatch order): the warp-wide minimum
-//     (two redux.sync) yields at once the finish time, which lane owns the slot,
-//     and where in the input stream the batch it holds starts;
+//     unsigned order is exactly (finish, dispatch order).  The slots are kept
+//     sorted across lanes 0..R-1: the next one to be reused is lane 0, and a
+//     new batch is inserted with one shuffle, one compare and one ballot;
 //   * the next 128 arrivals sit in four registers per lane, refilled 32 at a
 //     time one rotation ahead of use, so no global load is on the serial chain;
 //     the queue count is two or three ballots and a funnel shift;
 //   * a stage with max batch 1 is a max-plus scan over 32 queries at a time
 //     (run_stage_mb1);
-//   * while arrivals find a free replica on arrival and do not share a time
-//     stamp, every batch is a single query: up to 31 such dispatches are
-//     verified and committed at once (the "run" step in run_stage).
+//   * while no arrival comes in before the previous one has been dispatched,
+//     every batch is a single query and the replicas are reused round-robin:
+//     up to 31 such dispatches are computed by a scan, verified and committed
+//     at once (the "run" step in run_stage).
 //
 // The host selects this kernel when every time the simulation can reach fits
 // in 63 - q bits.
@@ -40,7 +41,7 @@ namespace il {
 namespace {
 
 constexpr uint64_t kNeverKey = ~0ull;
-constexpr int kMinRun = 3;          // shortest run of single dispatches worth committing at once
+constexpr int kMinRun = 2;          // shortest run of single dispatches worth committing at once
 
 enum RouteKind { kForward = 0, kBranch = 1 };
 
@@ -50,8 +51,7 @@ struct WarpCtx {
     uint32_t qmask;
     int qbits;
     const uint8_t *bits;
-    uint64_t *stage_buf;     // shared memory, 32 records: ordering buffer of the run step
-    uint64_t *slot_key;      // shared memory, 32 slot keys
+    uint64_t *slot_key;      // shared memory, 32 slot keys: staging for re-ordering the slots
     uint32_t *slot_q;        // shared memory, 32 slot query ids
     int *slot_b;             // shared memory, 32 slot batch sizes
 };
@@ -93,6 +93,9 @@ __device__ __forceinline__ void append(const WarpCtx &w, Sink &sk, const uint64_
 
 // One stage of one candidate, max batch >= 2.  WIDE: max batch > 32 (the queue
 // count looks at up to 64 arrivals).  Returns the number of batches dispatched.
+//
+// Replica slots live in lanes 0..R-1, always sorted by key, so the next slot to
+// be reused is lane 0 and the one after it lane 1.
 template <bool WIDE, int KIND>
 __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, const int mb,
                                          const int R, const int n_in, const uint64_t *in, Sink &sk,
@@ -122,12 +125,11 @@ __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, c
         }
     };
 
-    // replica slots: lane r < R holds replica r.  Never-used slots get distinct
-    // keys below every real key (real finish times are >= 1, and q >= 5).
+    // Never-used slots get distinct keys below every real key (real finish
+    // times are >= 1, and q >= 5); lanes >= R never hold a slot.
     uint64_t key = (lane < R) ? (uint64_t)lane : kNeverKey;
     int sl_b = 0;            // size of the batch the slot holds (0: none)
     uint32_t sl_q = 0;       // its first query
-    bool sorted = true;      // slot keys ascend with the lane index
 
     // lookahead window: A, B, C, D hold in[base + 32 k + lane]
     int base = 0, off = 0, head = 0;
@@ -136,85 +138,100 @@ __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, c
 
     int nbatch = 0;
     int cooldown = 0, penalty = 1;   // when to try the run step again after it did not pay off
-    bool try_run = true;
+    // the slot in lane 0, known to every lane
+    uint64_t m1 = 0;
+    int pb1 = 0;
+    uint32_t pq1 = 0;
 
     while (head < n_in) {
         // ------------------------------------------------------------------
-        // Run step: how many of the next arrivals are dispatched alone, at
-        // their arrival time?  Arrival i (i-th from head, time x_i) is, given
-        // that all earlier ones of the run were, iff
-        //   (1) x_{i+1} > x_i (nobody else is queued at the dispatch instant), and
-        //   (2) fewer than R replicas are busy at x_i: with phi_i old slots free
-        //       by x_i, the phi_i-th most recent single of the run has finished,
-        //       x_{i - phi_i} + D1 <= x_i (or i < phi_i).
-        // The leading m such arrivals are committed together: their keys join
-        // the old slots' keys, the m smallest keys of the union are emitted in
-        // order and the R largest become the slots.
+        // Run step.  While every batch is a single query (service time D1),
+        // the R replicas are reused round-robin: with the old slots' finish
+        // times g_0 <= ... <= g_{R-1}, the i-th next arrival starts at
+        //     s_i = max(x_i, g_i)            (i < R)
+        //     s_i = max(x_i, s_{i-R} + D1)   (i >= R)
+        // as long as the old slots reused so far finish by s_0 + D1, and it is
+        // dispatched alone iff x_{i+1} > s_i.  The s_i are a
+        // max-plus scan over the lanes; the leading m arrivals that pass are
+        // committed at once.  Slots are popped in the order g_0.., then the new
+        // finishes, so the first m of that sequence are emitted and the last R
+        // become the slots.
         // ------------------------------------------------------------------
-        if (try_run && cooldown == 0 && __ballot_sync(full, sl_b > 1) == 0) {
+        if (cooldown == 0) {
             const int pos = off + lane;
             const uint64_t xa = __shfl_sync(full, A, pos & 31), xb = __shfl_sync(full, B, pos & 31);
             const uint64_t X = pos < 32 ? xa : xb;                  // in[head + lane]
             const uint64_t XK = X | qmask;                          // kNever stays kNever
             const uint64_t XKn = __shfl_down_sync(full, XK, 1);
-            const uint64_t XK0 = __shfl_sync(full, XK, 0);
-            // old slots free by the first arrival are free for the whole run
-            const unsigned idle0 = __ballot_sync(full, key <= XK0);
-            const unsigned busy = __ballot_sync(full, lane < R && key > XK0);
-            int phi = __popc(idle0);
-            for (unsigned bm = busy; bm; bm &= bm - 1) {
-                const uint64_t kr = __shfl_sync(full, key, __ffs(bm) - 1);
-                phi += (kr <= XK);
+            const uint64_t gk = key | qmask;
+            uint64_t v = (lane < R && gk > XK) ? gk : XK;
+            uint64_t mul = d1k;
+            for (int d = R; d < 32; d <<= 1, mul <<= 1) {
+                const uint64_t u = __shfl_up_sync(full, v, d);
+                if (lane >= d && u + mul > v && v != kNeverKey) v = u + mul;
             }
-            const uint64_t Y = __shfl_sync(full, XK, max(lane - phi, 0));
-            const bool ok = (X != kNeverKey) && (lane < 31) && (XKn > XK) &&
-                            (lane < phi || Y + d1k <= XK);
-            const int m = __ffs(~__ballot_sync(full, ok)) - 1;       // lane 31 is never ok
+            const uint64_t f0 = __shfl_sync(full, v, 0) + d1k;
+            const bool ok = (X != kNeverKey) && (lane < 31) && (XKn > v);
+            int m = __ffs(~__ballot_sync(full, ok)) - 1;             // lane 31 is never ok
+            // old slots that finish after the first new single ("late") are not
+            // reused in round-robin order: the run must end before their turn
+            const int c0 = __popc(__ballot_sync(full, lane < R && gk <= f0));   // a prefix of the lanes
+            if (c0 < R) m = min(m, c0);
             if (m >= kMinRun) {
-                const uint64_t NK = (XK - qmask) + d1k + (uint64_t)(head + lane);
-                // rank of every old key among the old keys
-                int orank = lane;
-                if (!sorted) {
-                    orank = 0;
-                    for (int r = 0; r < R; r++) orank += (__shfl_sync(full, key, r) < key);
-                }
-                // merge: o = old keys below my new key, e = new keys below my old key
-                int o = __popc(idle0), e = 0;
-                const unsigned run_mask = (1u << m) - 1u;
-                for (unsigned bm = busy; bm; bm &= bm - 1) {
-                    const int r = __ffs(bm) - 1;
-                    const uint64_t kr = __shfl_sync(full, key, r);
-                    const unsigned below = __ballot_sync(full, NK < kr) & run_mask;
-                    o += (kr < NK);
-                    if (lane == r) e = __popc(below);
-                }
-                // never-used slots hold the smallest keys and emit nothing
+                const uint64_t NK = (v - qmask) + d1k + (uint64_t)(head + lane);
+                const uint32_t xq = (uint32_t)X & qmask;
+                // emit old slots 0 .. min(m, R) - 1 in lane order; never-used ones
+                // (the lowest z lanes) hold nothing, slots with a larger batch go one by one
                 const int z = __popc(__ballot_sync(full, lane < R && sl_b == 0));
-                const int u_new = lane + o;          // union rank of my new key (lane < m)
-                const int u_old = orank + e;         // union rank of my old key (lane < R)
-                // emitted: union rank < m, at output position rank - z
-                if (lane < m && u_new < m)
-                    w.stage_buf[u_new - z] = (NK & ~(uint64_t)qmask) | ((uint32_t)X & qmask);
-                if (lane < R && sl_b == 1 && u_old < m)
-                    w.stage_buf[u_old - z] = (key & ~(uint64_t)qmask) | sl_q;
-                // kept: union rank >= m, in slot lane rank - m
-                if (lane < m && u_new >= m) {
-                    w.slot_key[u_new - m] = NK;
-                    w.slot_q[u_new - m] = (uint32_t)X & qmask;
-                    w.slot_b[u_new - m] = 1;
+                const int n_old = min(m, R);
+                const uint64_t oldrec = (key & ~(uint64_t)qmask) | sl_q;
+                unsigned multi = __ballot_sync(full, lane < n_old && sl_b > 1);
+                int p0 = min(z, n_old);
+                while (p0 < n_old) {
+                    const int nxt = multi ? __ffs(multi) - 1 : n_old;
+                    if (nxt > p0) append<KIND>(w, sk, __shfl_sync(full, oldrec, (lane + p0) & 31), nxt - p0);
+                    if (nxt < n_old) {
+                        emit(__shfl_sync(full, key, nxt), __shfl_sync(full, sl_b, nxt), __shfl_sync(full, sl_q, nxt));
+                        multi &= multi - 1;
+                    }
+                    p0 = nxt + 1;
                 }
-                if (lane < R && u_old >= m) {
-                    w.slot_key[u_old - m] = key;
-                    w.slot_q[u_old - m] = sl_q;
-                    w.slot_b[u_old - m] = sl_b;
+                // ... then the new singles 0 .. m - R - 1
+                if (m > R) append<KIND>(w, sk, (NK & ~(uint64_t)qmask) | xq, m - R);
+                if (c0 >= R) {
+                    // new slots: positions m .. m + R - 1 of the sequence (old 0..R-1, new 0..m-1)
+                    const bool take_old = m + lane < R;
+                    const int src_old = (m + lane) & 31, src_new = (m + lane - R) & 31;
+                    const uint64_t k_o = __shfl_sync(full, key, src_old), k_n = __shfl_sync(full, NK, src_new);
+                    const uint32_t q_o = __shfl_sync(full, sl_q, src_old), q_n = __shfl_sync(full, xq, src_new);
+                    const int b_o = __shfl_sync(full, sl_b, src_old);
+                    if (lane < R) {
+                        key = take_old ? k_o : k_n;
+                        sl_q = take_old ? q_o : q_n;
+                        sl_b = take_old ? b_o : 1;
+                    }
+                } else {
+                    // m <= c0 < R: kept are old m..c0-1 (all before the new ones), then the
+                    // new singles merged with the late old slots c0..R-1
+                    int above = 0, below = 0;   // late old keys below my new key / new keys below my late old key
+                    for (int r = c0; r < R; r++) {
+                        const uint64_t kr = __shfl_sync(full, key, r);
+                        const unsigned lt = __ballot_sync(full, lane < m && NK < kr);
+                        above += (kr < NK);
+                        if (lane == r) below = __popc(lt);
+                    }
+                    if (lane >= m && lane < R) {
+                        const int dst = lane < c0 ? lane - m : lane - m + below;
+                        w.slot_key[dst] = key; w.slot_q[dst] = sl_q; w.slot_b[dst] = sl_b;
+                    }
+                    if (lane < m) {
+                        const int dst = c0 - m + lane + above;
+                        w.slot_key[dst] = NK; w.slot_q[dst] = xq; w.slot_b[dst] = 1;
+                    }
+                    __syncwarp();
+                    if (lane < R) { key = w.slot_key[lane]; sl_q = w.slot_q[lane]; sl_b = w.slot_b[lane]; }
+                    __syncwarp();
                 }
-                __syncwarp();
-                const int n_emit = m - min(z, m);
-                const uint64_t rec = lane < n_emit ? w.stage_buf[lane] : 0;
-                if (lane < R) { key = w.slot_key[lane]; sl_q = w.slot_q[lane]; sl_b = w.slot_b[lane]; }
-                __syncwarp();
-                append<KIND>(w, sk, rec, n_emit);
-                sorted = true;
                 penalty = 1;
                 head += m; off += m; nbatch += m;
                 while (off >= 32) {
@@ -223,6 +240,9 @@ __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, c
                     D = ld_rec(in, base + 96 + lane, n_in);
                     off -= 32;
                 }
+                m1 = __shfl_sync(full, key, 0);
+                pb1 = __shfl_sync(full, sl_b, 0);
+                pq1 = __shfl_sync(full, sl_q, 0);
                 continue;
             }
             cooldown = penalty;
@@ -231,18 +251,16 @@ __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, c
         if (cooldown > 0) cooldown--;
 
         // ------------------------------------------------------------------
-        // Single step: one batch.
+        // Single step: one batch.  (m1, pb1, pq1) is the slot in lane 0.
         // ------------------------------------------------------------------
-        const uint32_t khi = (uint32_t)(key >> 32), klo = (uint32_t)key;
-        const uint32_t mhi = __reduce_min_sync(full, khi);
-        const uint32_t mlo = __reduce_min_sync(full, khi == mhi ? klo : 0xffffffffu);
-        const bool mine = (khi == mhi) && (klo == mlo);
-        const uint64_t mk = ((uint64_t)mhi << 32) | mlo;
-        const int pb = __reduce_add_sync(full, mine ? sl_b : 0);
+        // the slot that will be first once lane 0's is gone: lane 1, or the new batch
+        const uint64_t m2 = __shfl_sync(full, key, 1);
+        const int pb2 = __shfl_sync(full, sl_b, 1);
+        const uint32_t pq2 = __shfl_sync(full, sl_q, 1);
 
         // dispatch time as a packed threshold: (t << q) | mask
         const uint64_t a_head = __shfl_sync(full, A, off);
-        const uint64_t k1 = mk | qmask, k2 = a_head | qmask;
+        const uint64_t k1 = m1 | qmask, k2 = a_head | qmask;
         const uint64_t thr = k1 > k2 ? k1 : k2;
 
         // queue length at t, capped at mb
@@ -259,15 +277,25 @@ __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, c
             break;
         }
         const uint64_t nk = thr + ((uint64_t)(uint32_t)row[cnt - 1] << qb) + (uint64_t)head - qmask;
+        const uint32_t qh = (uint32_t)a_head & qmask;
 
-        if (pb > 0) {
-            const uint32_t pq = __reduce_add_sync(full, mine ? sl_q : 0u);
-            emit(mk, pb, pq);
-        }
-        if (mine) { key = nk; sl_b = cnt; sl_q = (uint32_t)a_head & qmask; }
-        sorted = false;
-        // a single that did not wait suggests a calm stretch: worth trying a run
-        try_run = (cnt == 1) && (k2 >= k1);
+        if (pb1 > 0) emit(m1, pb1, pq1);
+
+        // drop lane 0's slot and insert the new one at its place in the order
+        uint64_t u = __shfl_down_sync(full, key, 1);
+        const int ub = __shfl_down_sync(full, sl_b, 1);
+        const uint32_t uq = __shfl_down_sync(full, sl_q, 1);
+        if (lane == 31) u = kNeverKey;
+        const bool le = u < nk;
+        const bool here = __ballot_sync(full, le) == w.lt_mask;
+        key = le ? u : (here ? nk : key);
+        sl_b = le ? ub : (here ? cnt : sl_b);
+        sl_q = le ? uq : (here ? qh : sl_q);
+        const bool second_first = m2 < nk;
+        m1 = second_first ? m2 : nk;
+        pb1 = second_first ? pb2 : cnt;
+        pq1 = second_first ? pq2 : qh;
+
         head += cnt;
         off += cnt;
         nbatch++;
@@ -278,21 +306,13 @@ __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, c
             off -= 32;
         }
     }
-    // drain what is still in flight, in key order
+    // drain what is still in flight: slots are in key order
 #pragma unroll 1
-    for (int k = 0; k < 32; k++) {
-        const uint32_t khi = (uint32_t)(key >> 32), klo = (uint32_t)key;
-        const uint32_t mhi = __reduce_min_sync(full, khi);
-        const uint32_t mlo = __reduce_min_sync(full, khi == mhi ? klo : 0xffffffffu);
-        const uint64_t mk = ((uint64_t)mhi << 32) | mlo;
-        if (mk == kNeverKey) break;
-        const bool mine = (khi == mhi) && (klo == mlo);
-        const int pb = __reduce_add_sync(full, mine ? sl_b : 0);
-        if (pb > 0) {
-            const uint32_t pq = __reduce_add_sync(full, mine ? sl_q : 0u);
-            emit(mk, pb, pq);
-        }
-        if (mine) { key = kNeverKey; sl_b = 0; }
+    for (int r = 0; r < R; r++) {
+        const uint64_t mk = __shfl_sync(full, key, r);
+        const int pb = __shfl_sync(full, sl_b, r);
+        const uint32_t pq = __shfl_sync(full, sl_q, r);
+        if (pb > 0) emit(mk, pb, pq);
     }
     return nbatch;
 }
@@ -346,7 +366,6 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32)
 des_packed_kernel(const __grid_constant__ DesParams p)
 {
     extern __shared__ int32_t s_lat[];
-    __shared__ uint64_t s_stage[kWarpsPerCta][32];
     __shared__ uint64_t s_slot_key[kWarpsPerCta][32];
     __shared__ uint32_t s_slot_q[kWarpsPerCta][32];
     __shared__ int s_slot_b[kWarpsPerCta][32];
@@ -362,7 +381,6 @@ des_packed_kernel(const __grid_constant__ DesParams p)
     w.qbits = p.qbits;
     w.qmask = (1u << p.qbits) - 1u;
     w.bits = p.bits;
-    w.stage_buf = s_stage[wid];
     w.slot_key = s_slot_key[wid];
     w.slot_q = s_slot_q[wid];
     w.slot_b = s_slot_b[wid];
