@@ -188,3 +188,55 @@ def test_config2_full_size_sampled(il, oracle):
     k = (99 * w.n_queries + 99) // 100
     assert np.array_equal(p99 <= w.slo_us, miss <= w.n_queries - k)
     assert (p99 > 0).all() and (miss >= 0).all() and (miss <= w.n_queries).all()
+
+
+def _sampled_check(il, oracle, w, n_sample, seed, extremes):
+    """Runs every candidate of w on the GPU (device entry point, torch-owned
+    workspace as in the bench) and checks a seeded sample plus structured
+    extremes against the oracle one by one, and size-free properties on all."""
+    import torch
+    with il.Estimator.from_workload(w) as est:
+        est.reserve_workspace(w.n_candidates)
+        d = torch.from_numpy(w.configs).cuda()
+        a, b = est.estimate_device(d, w.slo_us)
+        p99, miss = a.cpu().numpy(), b.cpu().numpy()
+        st = est.stats()
+        ext = np.ascontiguousarray(extremes, dtype=np.uint8)
+        e_p99, e_miss = est.estimate(ext, w.slo_us)
+    assert st["candidates"] == w.n_candidates
+    idx = np.random.default_rng(seed).choice(w.n_candidates, size=n_sample, replace=False)
+    both = np.concatenate([w.configs[idx], ext])
+    exp = oracle.estimate_many_parallel(w.parent, w.cond_bit, w.cond_val, w.latency_us,
+                                        w.arrival_us, w.branch_bits, both, w.slo_us)
+    got_p99 = np.concatenate([p99[idx], e_p99])
+    got_miss = np.concatenate([miss[idx], e_miss])
+    bad = np.nonzero((got_p99 != exp[0]) | (got_miss != exp[1]))[0]
+    assert bad.size == 0, (w.name, bad[:5], got_p99[bad[:5]], exp[0][bad[:5]], both[bad[:2]])
+    k = (99 * w.n_queries + 99) // 100
+    assert np.array_equal(p99 <= w.slo_us, miss <= w.n_queries - k)
+    assert (p99 > 0).all() and (miss >= 0).all() and (miss <= w.n_queries).all()
+    return st
+
+
+def _extremes(S, H, mbs, Rs):
+    return np.array([[[h, mb, R, 0]] * S for h in range(H) for mb in mbs for R in Rs], np.uint8)
+
+
+def test_config3_full_size_sampled(il, oracle):
+    """65,536 candidates x 200,000 queries on the 6-stage tree."""
+    w = workloads.make(3)
+    _sampled_check(il, oracle, w, 48, 3, _extremes(6, 3, (1, 64), (1, 8)))
+
+
+def test_config5_full_size_sampled(il, oracle):
+    """1,048,576 candidates x 100,000 queries on the 8-stage tree (R up to 32, max batch up to 64)."""
+    w = workloads.make(5)
+    _sampled_check(il, oracle, w, 64, 5, _extremes(8, 4, (1, 64), (1, 32)))
+
+
+def test_config4_full_trace_candidate_subset(il, oracle):
+    """The 10-stage pipeline on the full 1,000,000-query trace.  The full sweep is
+    262,144 candidates (2.6e12 query-events, minutes of GPU time); this test runs
+    the first 8,192 candidates of the same seeded draw and checks a sample."""
+    w = workloads.make(4, n_candidates=8192)
+    _sampled_check(il, oracle, w, 24, 4, _extremes(10, 4, (1, 64), (1, 16)))
