@@ -125,7 +125,7 @@ typedef struct {
     int64_t batches;         /* batches dispatched, all candidates, all stages           */
     int64_t algorithmic_ops; /* integer operations the method needs: per batch R + max_batch + 4
                                 (replica min, queue count, table add, slot update), per query-event 3 */
-    int64_t chunks;          /* how many (simulate, select) launch pairs the call made   */
+    int64_t chunks;          /* how many (order, simulate, select) launch triples the call made */
     int64_t kernel_launches; /* kernels launched by the call                             */
     double  sim_ms;          /* device time of the simulation kernels (CUDA events)      */
     double  select_ms;       /* device time of the percentile kernels (CUDA events)      */
@@ -197,7 +197,7 @@ IL_API int il_estimate_device(il_estimator *est, const il_stage_config *d_config
  *
  * Limit: the whole batch is evaluated in one pass, with at most 32 warps
  * resident, and must fit the array:
- *     256 + 12 * slot * min(32, n rounded up to 4) + (8 * n_queries' + 8) * n
+ *     256 + 12 * slot * min(32, n rounded up to 4) + (8 * n_queries' + 12) * n
  *         <= IL_STATIC_SCRATCH_BYTES
  * where n_queries' is n_queries rounded up to 32 and slot is the number of
  * stream elements one warp keeps between stages (for a linear pipeline about

@@ -394,6 +394,7 @@ des_packed_kernel(const __grid_constant__ DesParams p)
         if (lane == 0) c = atomicAdd(&p.counters[0], 1ull);
         c = __shfl_sync(full, c, 0);
         if (c >= (unsigned long long)p.n_cand) break;
+        c = (unsigned long long)p.order[c];
 
         uint64_t *slab = reinterpret_cast<uint64_t *>(p.slab + c * p.slab_stride);
         il_stage_config my_cfg = {0, 1, 1, 0};

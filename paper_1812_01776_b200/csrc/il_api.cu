@@ -32,6 +32,7 @@ struct il_estimator {
     int64_t n_pad = 0;                 // n rounded up to 32: one slab row
     int64_t visits[IL_MAX_STAGES] = {};
     int64_t events_per_candidate = 0;
+    float span_us = 1.f;
     DesParams base = {};               // bound-input part of the kernel parameters
     size_t smem = 0;
     int64_t slot_elems = 0;
@@ -60,16 +61,21 @@ struct il_estimator {
 
 namespace {
 
+// Resident CTAs per SM are capped below the occupancy limit: on B200, 24 warps
+// per SM (6 CTAs) measured faster than 28 on the 4,096-candidate workload (each
+// warp is a long dependent chain; more resident warps only add cache pressure).
+constexpr int kMaxCtasPerSm = 6;
+
 struct Plan {
     int64_t slots = 0;       // warp slots with stream buffers
     int64_t chunk = 0;       // candidates per (simulate, select) pair
-    size_t off_time = 0, off_qid = 0, off_slab = 0, off_or = 0, total = 0;
+    size_t off_time = 0, off_qid = 0, off_slab = 0, off_or = 0, off_order = 0, total = 0;
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 size_t slot_bytes(const il_estimator *e) { return (size_t)e->slot_elems * 12; }
-size_t cand_bytes(const il_estimator *e) { return (size_t)e->n_pad * 8 + 8; }
+size_t cand_bytes(const il_estimator *e) { return (size_t)e->n_pad * 8 + 12; }
 
 int64_t full_slots(const il_estimator *e)
 {
@@ -89,6 +95,7 @@ size_t layout(const il_estimator *e, Plan &pl)
     pl.off_qid = off;  off = align_up(off + (size_t)pl.slots * e->slot_elems * 4, 256);
     pl.off_slab = off; off = align_up(off + (size_t)pl.chunk * e->n_pad * 8, 256);
     pl.off_or = off;   off = align_up(off + (size_t)pl.chunk * 8, 256);
+    pl.off_order = off; off = align_up(off + (size_t)pl.chunk * 4, 256);
     pl.total = off;
     return off;
 }
@@ -216,6 +223,7 @@ void il::bound_view(const il_estimator *e, BoundView *out)
     out->S = e->S;
     out->n = e->n; out->n_pad = e->n_pad; out->slot_elems = e->slot_elems;
     out->smem = e->smem;
+    out->span_us = e->span_us;
     out->device = e->device;
     out->stream = e->stream;
 }
@@ -288,6 +296,7 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     e->num_sms = prop.multiProcessorCount;
     e->S = S; e->H = H; e->Bmax = B; e->n = n;
     e->n_pad = (n + 31) / 32 * 32;
+    e->span_us = (float)std::max<int64_t>(1, tr->arrival_us[n - 1] - tr->arrival_us[0]);
 
     // routing table and visits per stage
     DesParams &bp = e->base;
@@ -352,7 +361,7 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     e->ctas_per_sm_wide = des_max_ctas_per_sm(e->smem);
     e->ctas_per_sm_packed = des_packed_max_ctas_per_sm(e->smem);
     if (e->ctas_per_sm_wide < 1 || e->ctas_per_sm_packed < 1) return fail(IL_ERR_CUDA);
-    e->ctas_per_sm = use_packed(e) ? e->ctas_per_sm_packed : e->ctas_per_sm_wide;
+    e->ctas_per_sm = std::min(kMaxCtasPerSm, use_packed(e) ? e->ctas_per_sm_packed : e->ctas_per_sm_wide);
     *out = e;
     return IL_OK;
 }
@@ -379,7 +388,7 @@ int il_set_variant(il_estimator *e, int variant)
 {
     if (!e || (variant != IL_VARIANT_AUTO && variant != IL_VARIANT_WIDE)) return IL_ERR_INVALID_ARG;
     e->variant = variant;
-    e->ctas_per_sm = use_packed(e) ? e->ctas_per_sm_packed : e->ctas_per_sm_wide;
+    e->ctas_per_sm = std::min(kMaxCtasPerSm, use_packed(e) ? e->ctas_per_sm_packed : e->ctas_per_sm_wide);
     return IL_OK;
 }
 
@@ -477,7 +486,15 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
         p.slab = reinterpret_cast<int64_t *>(ws + pl.off_slab);
         p.slab_stride = e->n_pad;
         p.lat_or = reinterpret_cast<uint64_t *>(ws + pl.off_or);
+        p.order = reinterpret_cast<int32_t *>(ws + pl.off_order);
+        OrderParams op;
+        op.configs = p.configs; op.n_cand = cnt; op.lat = e->d_lat;
+        op.S = e->S; op.H = e->H; op.Bmax = e->Bmax;
+        for (int s = 0; s < IL_MAX_STAGES; s++) op.n_s[s] = e->base.n_s[s];
+        op.span_us = e->span_us;
+        op.order = reinterpret_cast<int32_t *>(ws + pl.off_order);
         if (ch > 0) IL_CUDA(cudaMemsetAsync(e->d_counters, 0, sizeof(unsigned long long), st));
+        IL_CUDA(launch_order(op, st));
         const int64_t ctas = std::min<int64_t>(pl.slots / kWarpsPerCta, (cnt + kWarpsPerCta - 1) / kWarpsPerCta);
         IL_CUDA(cudaEventRecord(e->events[2 + 3 * ch], st));
         IL_CUDA(launch_simulation(p, use_packed(e), (int)ctas, e->smem, st));
@@ -489,7 +506,7 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
         sp.out_p99 = d_out_p99 + lo; sp.out_miss = d_out_miss + lo;
         IL_CUDA(launch_select(sp, st));
         IL_CUDA(cudaEventRecord(e->events[4 + 3 * ch], st));
-        launches += 2;
+        launches += 3;
     }
     IL_CUDA(cudaEventRecord(e->events[1], st));
     IL_CUDA(cudaMemcpyAsync(e->h_counters, e->d_counters, 4 * sizeof(unsigned long long),

@@ -28,6 +28,7 @@ struct DesParams {
     // this launch
     const il_stage_config *configs;  // [n_cand][S], already offset to the chunk
     int64_t n_cand;
+    const int32_t *order;         // [n_cand] candidates in the order warps should take them (costliest first)
     int64_t slot_elems;           // stream elements per warp slot
     int64_t *ws_time;             // [slots][slot_elems]
     int32_t *ws_qid;              // [slots][slot_elems]
@@ -60,6 +61,7 @@ struct BoundView {
     int32_t S;
     int64_t n, n_pad, slot_elems;
     size_t smem;
+    float span_us;
     int device;
     cudaStream_t stream;
 };
@@ -74,6 +76,19 @@ inline cudaError_t launch_simulation(const DesParams &p, bool packed, int grid, 
     return packed ? launch_des_packed(p, grid, smem, stream) : launch_des(p, grid, smem, stream);
 }
 cudaError_t launch_select(const SelectParams &p, cudaStream_t stream);
+
+// Fills order[0..n_cand) with the chunk's candidate indices, costliest first
+// (longest-processing-time-first scheduling over the warps).
+struct OrderParams {
+    const il_stage_config *configs;  // [n_cand][S]
+    int64_t n_cand;
+    const int32_t *lat;              // [S][H][Bmax]
+    int32_t S, H, Bmax;
+    int32_t n_s[IL_MAX_STAGES];
+    float span_us;                   // last arrival - first arrival (at least 1)
+    int32_t *order;                  // [n_cand] out
+};
+cudaError_t launch_order(const OrderParams &p, cudaStream_t stream);
 int des_max_ctas_per_sm(size_t smem);
 cudaError_t launch_int_issue(unsigned *sink, int grid, int iters, cudaStream_t stream);
 

@@ -65,6 +65,7 @@ extern "C" int il_estimate_device_static(il_estimator *est, const il_stage_confi
         return IL_ERR_TOO_LARGE;
     off = align_up(off + (size_t)n_cand * v.n_pad * 8, 256);
     const size_t off_or = off;   off = align_up(off + (size_t)n_cand * 8, 256);
+    const size_t off_order = off; off = align_up(off + (size_t)n_cand * 4, 256);
     if (off > IL_STATIC_SCRATCH_BYTES) return IL_ERR_TOO_LARGE;
 
     if (cudaSetDevice(v.device) != cudaSuccess) return IL_ERR_CUDA;
@@ -87,6 +88,14 @@ extern "C" int il_estimate_device_static(il_estimator *est, const il_stage_confi
     p.slab = reinterpret_cast<int64_t *>(base + off_slab);
     p.slab_stride = v.n_pad;
     p.lat_or = reinterpret_cast<uint64_t *>(base + off_or);
+    p.order = reinterpret_cast<int32_t *>(base + off_order);
+    OrderParams op;
+    op.configs = d_configs; op.n_cand = n_cand; op.lat = v.base.lat;
+    op.S = v.S; op.H = v.base.H; op.Bmax = v.base.Bmax;
+    for (int s = 0; s < IL_MAX_STAGES; s++) op.n_s[s] = v.base.n_s[s];
+    op.span_us = v.span_us;
+    op.order = reinterpret_cast<int32_t *>(base + off_order);
+    if (launch_order(op, st) != cudaSuccess) return IL_ERR_CUDA;
     if (launch_simulation(p, v.packed, (int)(slots / kWarpsPerCta), v.smem, st) != cudaSuccess)
         return IL_ERR_CUDA;
 

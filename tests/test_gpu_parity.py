@@ -76,7 +76,7 @@ def test_random_small(il, oracle, seed, variant):
 
 def test_config1_full(il, oracle):
     st = check(il, oracle, workloads.make(1))
-    assert st["batches"] > 0 and st["kernel_launches"] == 2 * st["chunks"]
+    assert st["batches"] > 0 and st["kernel_launches"] == 3 * st["chunks"]
 
 
 @pytest.mark.parametrize("variant", [0, 1], ids=["packed", "wide"])
