@@ -209,6 +209,7 @@ def run_cuda(args):
     events_per_cand = w.query_events()
 
     est = il.Estimator.from_workload(w, device=local)
+    est.set_variant(args.variant)
     ws_bytes = est.reserve_workspace(n_cand)
     stream = torch.cuda.Stream(device=dev)
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)   # > 126 MB of L2
@@ -309,7 +310,7 @@ def run_cuda(args):
                    "query_events_per_candidate": events_per_cand,
                    "l2": "256 MiB buffer written between steps; working set "
                          f"{ws_bytes / 2**30:.1f} GiB > L2",
-                   "workspace_bytes": ws_bytes, "parallelism": f"candidates sharded over {world} GPU(s)"},
+                   "workspace_bytes": ws_bytes, "kernel_variant": args.variant, "parallelism": f"candidates sharded over {world} GPU(s)"},
         "query_events_per_s": value * events_per_cand,
         "batches_per_s": batches * world * K / (total_ms * 1e-3) if batches else None,
         "mean_batch": events_per_cand * n_cand / batches if batches else None,
@@ -354,6 +355,9 @@ def main():
                          "for profiler captures, not for reported numbers")
     ap.add_argument("--queries", type=int, default=None,
                     help="trace length (default: the workload's 50,000); for profiler captures")
+    ap.add_argument("--variant", type=int, default=0,
+                    help="simulation kernel: 0 default (packed records, trace staged through shared "
+                         "memory), 1 wide streams, 2 packed records with direct trace reads")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer timing (profiler captures)")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -56,10 +56,154 @@ struct WarpCtx {
     int *slot_b;             // shared memory, 32 slot batch sizes
 };
 
-__device__ __forceinline__ uint64_t ld_rec(const uint64_t *in, int idx, int n_in)
+// ---------------------------------------------------------------------------
+// Where a stage reads its arrival stream from.
+//
+// GlobalSrc: a stream in global memory (the warp's own inter-stage buffer, or
+// the packed trace through L1/L2).
+//
+// TileSrc: the root stage's stream, i.e. the shared trace, staged through
+// shared memory once per CTA.  The trace is cut into tiles of kTileRecs
+// records; a ring of kTiles tiles is filled by bulk asynchronous copies
+// (cp.async.bulk, completion signalled on an mbarrier per ring slot) and read
+// by all warps of the CTA, each at its own pace.  A warp releases a tile when
+// its lookahead has moved past it; the warp that releases a tile last re-arms
+// the slot and issues the copy of the tile kTiles further on.  Every wait is
+// bounded: on a time-out the warp records IL_ERR_ITER_LIMIT and from then on
+// reads "no more arrivals", which ends its loops.
+// ---------------------------------------------------------------------------
+constexpr int kTileLog = 9;
+constexpr int kTileRecs = 1 << kTileLog;        // 512 records = 4 KB
+constexpr int kTiles = 4;                       // ring depth
+constexpr unsigned kTileBytes = kTileRecs * 8;
+constexpr int kWaitLimit = 1 << 24;             // polls of an mbarrier before giving up
+
+struct TileRing {
+    uint64_t tiles[kTiles][kTileRecs];          // 128-byte aligned by the declaration below
+    uint64_t full[kTiles];                      // mbarriers: "the copy into this slot has landed"
+    int released[kTiles];                       // warps that are done with the slot's current tile
+    int uses[kTiles];                           // how often the slot has been armed
+    int base_uses[kTiles];                      // `uses` at the start of the current group
+    int group_base;                             // first position (in the order array) of the group
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p)
 {
-    return idx < n_in ? in[idx] : kNeverKey;
+    return (uint32_t)__cvta_generic_to_shared(p);
 }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, int count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+
+// Waits until the slot's barrier has completed the phase with this parity.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, unsigned parity)
+{
+    for (int i = 0; i < kWaitLimit; i++)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+
+// Arms the slot's barrier for kTileBytes and starts the copy of trace tile `tile` into it.
+__device__ __forceinline__ void tile_issue(TileRing *ring, const uint64_t *ptrace, int tile)
+{
+    const int slot = tile & (kTiles - 1);
+    const uint32_t bar = smem_addr(&ring->full[slot]);
+    ring->uses[slot]++;
+    // order the CTA's earlier generic-proxy reads of the slot before the async-proxy write
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kTileBytes) : "memory");
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(smem_addr(ring->tiles[slot])), "l"(ptrace + (size_t)tile * kTileRecs), "r"(kTileBytes), "r"(bar)
+        : "memory");
+}
+
+struct GlobalSrc {
+    const uint64_t *in;
+    bool root;               // the packed trace: the query of record i is i
+    // 32 consecutive records starting at the 32-aligned index `idx0`
+    __device__ __forceinline__ uint64_t load32(int idx0, int lane, int n_in)
+    {
+        return idx0 + lane < n_in ? in[idx0 + lane] : kNeverKey;
+    }
+    __device__ __forceinline__ uint32_t query_at(int idx, uint32_t qmask) const
+    {
+        return root ? (uint32_t)idx : ((uint32_t)in[idx] & qmask);
+    }
+    __device__ __forceinline__ void finish(int, int) {}
+};
+
+struct TileSrc {
+    TileRing *ring;
+    const uint64_t *ptrace;
+    int n_tiles;
+    int cur;                 // oldest tile this warp has not released
+    int waited;              // newest tile this warp has seen land
+    bool dead;               // a wait timed out
+    int *status;
+
+    __device__ __forceinline__ void release(int tile, int lane)
+    {
+        __syncwarp();
+        if (lane == 0) {
+            const int slot = tile & (kTiles - 1);
+            if (atomicAdd(&ring->released[slot], 1) == kWarpsPerCta - 1) {
+                ring->released[slot] = 0;
+                __threadfence_block();
+                if (tile + kTiles < n_tiles) tile_issue(ring, ptrace, tile + kTiles);
+            }
+        }
+    }
+    // Waits (bounded) until tile t has landed.  Tiles must be waited for in
+    // order before they are read or released: a slot is only re-armed after all
+    // warps have released its previous tile, so waiting keeps the per-slot
+    // release counts from mixing two tiles.
+    __device__ __forceinline__ bool wait_tile(int t, int lane)
+    {
+        static_assert(kTiles == 4, "tile / kTiles is written as a shift by 2");
+        const int slot = t & (kTiles - 1);
+        const unsigned parity = (unsigned)(ring->base_uses[slot] + (t >> 2)) & 1u;
+        if (!mbar_wait_bounded(&ring->full[slot], parity)) {
+            if (lane == 0) atomicCAS(status, 0, IL_ERR_ITER_LIMIT);
+            dead = true;
+            return false;
+        }
+        waited = t;
+        return true;
+    }
+    __device__ __forceinline__ uint64_t load32(int idx0, int lane, int n_in)
+    {
+        if (idx0 >= n_in || dead) return kNeverKey;
+        const int t = idx0 >> kTileLog;
+        while (cur < t) { release(cur, lane); cur++; }
+        if (t > waited && !wait_tile(t, lane)) return kNeverKey;
+        // the trace is padded with "never" records up to a whole tile
+        return ring->tiles[t & (kTiles - 1)][(idx0 & (kTileRecs - 1)) + lane];
+    }
+    __device__ __forceinline__ uint32_t query_at(int idx, uint32_t) const { return (uint32_t)idx; }
+    // releases whatever this warp still holds, so that the ring can move on for the others
+    __device__ __forceinline__ void finish(int lane, int)
+    {
+        while (cur < n_tiles) {
+            if (cur > waited && !dead) wait_tile(cur, lane);
+            release(cur, lane);
+            cur++;
+        }
+    }
+};
 
 // Where one stage's completions go: the next stage's stream, or the slab (a
 // query that leaves), per value of the branch bit.
@@ -96,9 +240,9 @@ __device__ __forceinline__ void append(const WarpCtx &w, Sink &sk, const uint64_
 //
 // Replica slots live in lanes 0..R-1, always sorted by key, so the next slot to
 // be reused is lane 0 and the one after it lane 1.
-template <bool WIDE, int KIND>
+template <bool WIDE, int KIND, class Src>
 __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, const int mb,
-                                         const int R, const int n_in, const uint64_t *in, Sink &sk,
+                                         const int R, const int n_in, Src &src, Sink &sk,
                                          int *status)
 {
     const unsigned full = 0xffffffffu;
@@ -120,7 +264,7 @@ __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, c
         for (int j0 = 0; j0 < b; j0 += 32) {
             const int j = j0 + lane;
             uint64_t rec = 0;
-            if (j < b) rec = tbits | ((uint32_t)in[start + j] & qmask);
+            if (j < b) rec = tbits | src.query_at(start + j, qmask);
             append<KIND>(w, sk, rec, min(32, b - j0));
         }
     };
@@ -133,8 +277,8 @@ __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, c
 
     // lookahead window: A, B, C, D hold in[base + 32 k + lane]
     int base = 0, off = 0, head = 0;
-    uint64_t A = ld_rec(in, lane, n_in), B = ld_rec(in, 32 + lane, n_in),
-             C = ld_rec(in, 64 + lane, n_in), D = ld_rec(in, 96 + lane, n_in);
+    uint64_t A = src.load32(0, lane, n_in), B = src.load32(32, lane, n_in),
+             C = src.load32(64, lane, n_in), D = src.load32(96, lane, n_in);
 
     int nbatch = 0;
     int cooldown = 0, penalty = 1;   // when to try the run step again after it did not pay off
@@ -237,7 +381,7 @@ __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, c
                 while (off >= 32) {
                     A = B; B = C; C = D;
                     base += 32;
-                    D = ld_rec(in, base + 96 + lane, n_in);
+                    D = src.load32(base + 96, lane, n_in);
                     off -= 32;
                 }
                 m1 = __shfl_sync(full, key, 0);
@@ -302,7 +446,7 @@ __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, c
         while (off >= 32) {
             A = B; B = C; C = D;
             base += 32;
-            D = ld_rec(in, base + 96 + lane, n_in);
+            D = src.load32(base + 96, lane, n_in);
             off -= 32;
         }
     }
@@ -314,6 +458,7 @@ __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, c
         const uint32_t pq = __shfl_sync(full, sl_q, r);
         if (pb > 0) emit(mk, pb, pq);
     }
+    src.finish(lane, n_in);
     return nbatch;
 }
 
@@ -324,9 +469,9 @@ __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, c
 // and queries leave in arrival order.  Unrolled, s_i is a running maximum of
 // a_{i-jR} + j D over j, which 32 lanes evaluate for 32 consecutive queries
 // with log2(32/R) shuffle steps plus one carry from the previous 32.
-template <int KIND>
+template <int KIND, class Src>
 __device__ __forceinline__ int run_stage_mb1(const WarpCtx &w, const int32_t *row, const int R,
-                                             const int n_in, const uint64_t *in, Sink &sk)
+                                             const int n_in, Src &src, Sink &sk)
 {
     const unsigned full = 0xffffffffu;
     const int lane = w.lane;
@@ -340,10 +485,10 @@ __device__ __forceinline__ int run_stage_mb1(const WarpCtx &w, const int32_t *ro
     const int64_t carry_add = (int64_t)hops * D;
     int64_t prev = kLongAgo;            // start times of the previous 32 queries
 
-    uint64_t rec = ld_rec(in, lane, n_in);
+    uint64_t rec = src.load32(0, lane, n_in);
     for (int base = 0; base < n_in; base += 32) {
         const uint64_t cur = rec;
-        rec = ld_rec(in, base + 32 + lane, n_in);          // next 32, off the dependent chain
+        rec = src.load32(base + 32, lane, n_in);           // next 32, off the dependent chain
         const bool act = base + lane < n_in;
         int64_t v = act ? (int64_t)(cur >> qb) : (INT64_C(1) << 62);
         int64_t mul = D;
@@ -357,11 +502,93 @@ __device__ __forceinline__ int run_stage_mb1(const WarpCtx &w, const int32_t *ro
         const uint64_t orec = ((uint64_t)(v + D) << qb) | ((uint32_t)cur & qmask);
         append<KIND>(w, sk, orec, min(32, n_in - base));
     }
+    src.finish(lane, n_in);
     return n_in;
+}
+
+template <class Src>
+__device__ __forceinline__ int dispatch_stage(const WarpCtx &w, const int32_t *row, const int mb,
+                                              const int R, const int n_in, Src &src, Sink &sk,
+                                              int *status)
+{
+    const bool branch = sk.bit >= 0;
+    if (mb == 1)
+        return branch ? run_stage_mb1<kBranch>(w, row, R, n_in, src, sk)
+                      : run_stage_mb1<kForward>(w, row, R, n_in, src, sk);
+    if (mb > 32)
+        return branch ? run_stage<true, kBranch>(w, row, mb, R, n_in, src, sk, status)
+                      : run_stage<true, kForward>(w, row, mb, R, n_in, src, sk, status);
+    return branch ? run_stage<false, kBranch>(w, row, mb, R, n_in, src, sk, status)
+                  : run_stage<false, kForward>(w, row, mb, R, n_in, src, sk, status);
+}
+
+// Simulates candidate `c` of the chunk on this warp.  STAGED: the root stage
+// reads the trace from the CTA's tile ring (all warps of the CTA must then enter
+// together, also those without a candidate of their own: has == false).
+template <bool STAGED>
+__device__ __forceinline__ void simulate_candidate(const DesParams &p, const WarpCtx &w,
+                                                   const int32_t *s_lat, uint64_t *my_rec,
+                                                   TileRing *ring, const bool has, const int64_t c,
+                                                   unsigned long long &batches,
+                                                   unsigned long long &alg_ops)
+{
+    const unsigned full = 0xffffffffu;
+    const int lane = w.lane;
+    const int n_tiles = (p.n + kTileRecs - 1) >> kTileLog;
+    uint64_t *slab = reinterpret_cast<uint64_t *>(p.slab + (has ? c : 0) * p.slab_stride);
+    il_stage_config my_cfg = {0, 1, 1, 0};
+    if (has && lane < p.S) my_cfg = p.configs[c * p.S + lane];
+    const bool bad = lane < p.S && (my_cfg.hw >= p.H || my_cfg.max_batch < 1 ||
+                                    my_cfg.max_batch > p.Bmax || my_cfg.replicas < 1 ||
+                                    my_cfg.replicas > IL_MAX_REPLICAS);
+    const bool skip = !has || __any_sync(full, bad);
+    if (skip) {
+        if (has) {
+            if (lane == 0) atomicCAS(p.status, 0, IL_ERR_BAD_CONFIG);
+            for (int i = lane; i < p.n; i += 32) slab[i] = 0;
+        }
+        if (STAGED) {   // keep the ring moving for the other warps of the CTA
+            TileSrc src = {ring, p.ptrace, n_tiles, 0, -1, false, p.status};
+            src.finish(lane, p.n);
+        }
+        return;
+    }
+
+    int exits = 0;
+    for (int s = 0; s < p.S; s++) {
+        const int n_in = p.n_s[s];
+        if (n_in == 0) continue;
+        const int hw = __shfl_sync(full, (int)my_cfg.hw, s);
+        const int mb = __shfl_sync(full, (int)my_cfg.max_batch, s);
+        const int R = __shfl_sync(full, (int)my_cfg.replicas, s);
+        const int32_t *row = s_lat + (s * p.H + hw) * p.Bmax;
+        const int da = p.dest_a[s], db = p.dest_b[s];
+        Sink sk;
+        sk.bit = p.bit[s];
+        sk.out_a = da < 0 ? slab + exits : my_rec + p.buf_off[da];
+        sk.out_b = db < 0 ? slab + exits : my_rec + p.buf_off[db];
+        sk.tail_a = 0; sk.tail_b = 0;
+        int nb;
+        if (STAGED && s == 0) {
+            TileSrc src = {ring, p.ptrace, n_tiles, 0, -1, false, p.status};
+            nb = dispatch_stage(w, row, mb, R, n_in, src, sk, p.status);
+        } else {
+            GlobalSrc src = {s == 0 ? p.ptrace : my_rec + p.buf_off[s], s == 0};
+            nb = dispatch_stage(w, row, mb, R, n_in, src, sk, p.status);
+        }
+        // a guarded stage has at most one side that leaves the pipeline
+        if (sk.bit < 0) { if (da < 0) exits += sk.tail_a; }
+        else exits += (da < 0 ? sk.tail_a : 0) + (db < 0 ? sk.tail_b : 0);
+        batches += (unsigned)nb;
+        alg_ops += 3ull * (unsigned)n_in + (unsigned long long)nb * (unsigned)(R + mb + 4);
+        __syncwarp();   // this stage's stream writes are read by the next stage's other lanes
+    }
+    if (lane == 0 && exits != p.n) atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT);
 }
 
 }  // namespace
 
+template <bool STAGED>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
 des_packed_kernel(const __grid_constant__ DesParams p)
 {
@@ -369,8 +596,14 @@ des_packed_kernel(const __grid_constant__ DesParams p)
     __shared__ uint64_t s_slot_key[kWarpsPerCta][32];
     __shared__ uint32_t s_slot_q[kWarpsPerCta][32];
     __shared__ int s_slot_b[kWarpsPerCta][32];
+    __shared__ __align__(128) unsigned char s_ring_mem[STAGED ? sizeof(TileRing) : 16];
+    TileRing *ring = reinterpret_cast<TileRing *>(s_ring_mem);
     const int n_tab = p.S * p.H * p.Bmax;
     for (int i = threadIdx.x; i < n_tab; i += blockDim.x) s_lat[i] = p.lat[i];
+    if (STAGED && threadIdx.x == 0) {
+        for (int k = 0; k < kTiles; k++) { mbar_init(&ring->full[k], 1); ring->uses[k] = 0; ring->released[k] = 0; }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
     __syncthreads();
 
     const unsigned full = 0xffffffffu;
@@ -389,76 +622,62 @@ des_packed_kernel(const __grid_constant__ DesParams p)
     uint64_t *my_rec = reinterpret_cast<uint64_t *>(p.ws_time) + slot * p.slot_elems;
     unsigned long long batches = 0, alg_ops = 0;
 
-    for (;;) {
-        unsigned long long c = 0;
-        if (lane == 0) c = atomicAdd(&p.counters[0], 1ull);
-        c = __shfl_sync(full, c, 0);
-        if (c >= (unsigned long long)p.n_cand) break;
-        c = (unsigned long long)p.order[c];
-
-        uint64_t *slab = reinterpret_cast<uint64_t *>(p.slab + c * p.slab_stride);
-        il_stage_config my_cfg = {0, 1, 1, 0};
-        if (lane < p.S) my_cfg = p.configs[c * p.S + lane];
-        const bool bad = lane < p.S && (my_cfg.hw >= p.H || my_cfg.max_batch < 1 ||
-                                        my_cfg.max_batch > p.Bmax || my_cfg.replicas < 1 ||
-                                        my_cfg.replicas > IL_MAX_REPLICAS);
-        if (__any_sync(full, bad)) {
-            if (lane == 0) atomicCAS(p.status, 0, IL_ERR_BAD_CONFIG);
-            for (int i = lane; i < p.n; i += 32) slab[i] = 0;
-            continue;
+    if (!STAGED) {
+        // every warp on its own: take the next candidate in the order array
+        for (;;) {
+            unsigned long long c = 0;
+            if (lane == 0) c = atomicAdd(&p.counters[0], 1ull);
+            c = __shfl_sync(full, c, 0);
+            if (c >= (unsigned long long)p.n_cand) break;
+            simulate_candidate<false>(p, w, s_lat, my_rec, nullptr, true, (int64_t)p.order[c], batches, alg_ops);
         }
-
-        int exits = 0;
-        for (int s = 0; s < p.S; s++) {
-            const int n_in = p.n_s[s];
-            if (n_in == 0) continue;
-            const int hw = __shfl_sync(full, (int)my_cfg.hw, s);
-            const int mb = __shfl_sync(full, (int)my_cfg.max_batch, s);
-            const int R = __shfl_sync(full, (int)my_cfg.replicas, s);
-            const int32_t *row = s_lat + (s * p.H + hw) * p.Bmax;
-            const uint64_t *in = (s == 0) ? p.ptrace : my_rec + p.buf_off[s];
-            const int da = p.dest_a[s], db = p.dest_b[s];
-            Sink sk;
-            sk.bit = p.bit[s];
-            sk.out_a = da < 0 ? slab + exits : my_rec + p.buf_off[da];
-            sk.out_b = db < 0 ? slab + exits : my_rec + p.buf_off[db];
-            sk.tail_a = 0; sk.tail_b = 0;
-            const bool branch = sk.bit >= 0;
-            int nb;
-            if (mb == 1) {
-                nb = branch ? run_stage_mb1<kBranch>(w, row, R, n_in, in, sk)
-                            : run_stage_mb1<kForward>(w, row, R, n_in, in, sk);
-            } else if (mb > 32) {
-                nb = branch ? run_stage<true, kBranch>(w, row, mb, R, n_in, in, sk, p.status)
-                            : run_stage<true, kForward>(w, row, mb, R, n_in, in, sk, p.status);
-            } else {
-                nb = branch ? run_stage<false, kBranch>(w, row, mb, R, n_in, in, sk, p.status)
-                            : run_stage<false, kForward>(w, row, mb, R, n_in, in, sk, p.status);
+    } else {
+        // the CTA takes kWarpsPerCta consecutive positions of the order array at
+        // a time (neighbours in that order cost about the same) and its warps go
+        // through the staged trace together
+        const int n_tiles = (p.n + kTileRecs - 1) >> kTileLog;
+        for (;;) {
+            __syncthreads();      // everybody is done with the previous group's tiles
+            if (threadIdx.x == 0) {
+                const unsigned long long g = atomicAdd(&p.counters[0], (unsigned long long)kWarpsPerCta);
+                ring->group_base = g < (unsigned long long)p.n_cand ? (int)g : -1;
+                for (int k = 0; k < kTiles; k++) { ring->released[k] = 0; ring->base_uses[k] = ring->uses[k]; }
+                if (ring->group_base >= 0)
+                    for (int t = 0; t < kTiles && t < n_tiles; t++) tile_issue(ring, p.ptrace, t);
             }
-            // a guarded stage has at most one side that leaves the pipeline
-            if (!branch) { if (da < 0) exits += sk.tail_a; }
-            else exits += (da < 0 ? sk.tail_a : 0) + (db < 0 ? sk.tail_b : 0);
-            batches += (unsigned)nb;
-            alg_ops += 3ull * (unsigned)n_in + (unsigned long long)nb * (unsigned)(R + mb + 4);
-            __syncwarp();   // this stage's stream writes are read by the next stage's other lanes
+            __syncthreads();
+            const int g = ring->group_base;
+            if (g < 0) break;
+            const int64_t pos = (int64_t)g + wid;
+            const bool has = pos < p.n_cand;
+            simulate_candidate<true>(p, w, s_lat, my_rec, ring, has, has ? (int64_t)p.order[pos] : 0, batches, alg_ops);
         }
-        if (lane == 0 && exits != p.n) atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT);
+        // no copy may still be in flight into this CTA's shared memory when it exits
+        __syncthreads();
+        if (threadIdx.x == 0)
+            for (int k = 0; k < kTiles; k++)
+                if (ring->uses[k] > 0) mbar_wait_bounded(&ring->full[k], (unsigned)(ring->uses[k] - 1) & 1u);
+        __syncthreads();
     }
     if (lane == 0 && batches) { atomicAdd(&p.counters[1], batches); atomicAdd(&p.counters[2], alg_ops); }
 }
 
-cudaError_t launch_des_packed(const DesParams &p, int grid, size_t smem, cudaStream_t stream)
+cudaError_t launch_des_packed(const DesParams &p, bool staged, int grid, size_t smem, cudaStream_t stream)
 {
-    des_packed_kernel<<<grid, kWarpsPerCta * 32, smem, stream>>>(p);
+    if (staged) des_packed_kernel<true><<<grid, kWarpsPerCta * 32, smem, stream>>>(p);
+    else des_packed_kernel<false><<<grid, kWarpsPerCta * 32, smem, stream>>>(p);
     return cudaGetLastError();
 }
 
-int des_packed_max_ctas_per_sm(size_t smem)
+int des_packed_max_ctas_per_sm(bool staged, size_t smem)
 {
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, des_packed_kernel, kWarpsPerCta * 32, smem) != cudaSuccess)
-        return 0;
-    return n;
+    cudaError_t e = staged
+        ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, des_packed_kernel<true>, kWarpsPerCta * 32, smem)
+        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, des_packed_kernel<false>, kWarpsPerCta * 32, smem);
+    return e == cudaSuccess ? n : 0;
 }
+
+int trace_tile_records() { return kTileRecs; }
 
 }  // namespace il

@@ -41,7 +41,7 @@ struct il_estimator {
     uint64_t *d_ptrace = nullptr;      // packed root stream
     bool can_pack = false;             // every reachable time fits a packed record
     int variant = IL_VARIANT_AUTO;
-    int ctas_per_sm_wide = 0, ctas_per_sm_packed = 0;
+    int ctas_per_sm_wide = 0, ctas_per_sm_packed = 0, ctas_per_sm_staged = 0;
     uint8_t *d_bits = nullptr;
     int32_t *d_lat = nullptr;
     unsigned long long *d_counters = nullptr;   // [4]
@@ -195,6 +195,20 @@ bool use_packed(const il_estimator *e)
     return e->can_pack && e->variant != IL_VARIANT_WIDE;
 }
 
+int sim_kernel(const il_estimator *e)
+{
+    if (!use_packed(e)) return kSimWide;
+    return e->variant == IL_VARIANT_PACKED_DIRECT ? kSimPacked : kSimPackedStaged;
+}
+
+int ctas_for(const il_estimator *e)
+{
+    const int k = sim_kernel(e);
+    const int occ = k == kSimWide ? e->ctas_per_sm_wide
+                  : k == kSimPacked ? e->ctas_per_sm_packed : e->ctas_per_sm_staged;
+    return std::min(kMaxCtasPerSm, occ);
+}
+
 void free_device(il_estimator *e)
 {
     cudaFree(e->d_arrival); cudaFree(e->d_ptrace); cudaFree(e->d_bits); cudaFree(e->d_lat);
@@ -219,7 +233,7 @@ int ensure_events(il_estimator *e, size_t count)
 void il::bound_view(const il_estimator *e, BoundView *out)
 {
     out->base = e->base;
-    out->packed = use_packed(e);
+    out->kernel = sim_kernel(e);
     out->S = e->S;
     out->n = e->n; out->n_pad = e->n_pad; out->slot_elems = e->slot_elems;
     out->smem = e->smem;
@@ -339,11 +353,14 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     e->can_pack = can_pack;
     bp.qbits = qbits;
     if (can_pack) {
-        std::vector<uint64_t> packed((size_t)n);
+        // padded with "never" records to whole tiles, so that bulk copies always move full tiles
+        const int64_t tile = trace_tile_records();
+        const int64_t n_padded = (n + tile - 1) / tile * tile;
+        std::vector<uint64_t> packed((size_t)n_padded, ~0ull);
         for (int64_t i = 0; i < n; i++)
             packed[(size_t)i] = ((uint64_t)tr->arrival_us[i] << qbits) | (uint64_t)i;
-        IL_CUDA_E(cudaMalloc(&e->d_ptrace, (size_t)n * 8));
-        IL_CUDA_E(cudaMemcpy(e->d_ptrace, packed.data(), (size_t)n * 8, cudaMemcpyHostToDevice));
+        IL_CUDA_E(cudaMalloc(&e->d_ptrace, (size_t)n_padded * 8));
+        IL_CUDA_E(cudaMemcpy(e->d_ptrace, packed.data(), (size_t)n_padded * 8, cudaMemcpyHostToDevice));
     }
     IL_CUDA_E(cudaMalloc(&e->d_lat, e->smem));
     IL_CUDA_E(cudaMalloc(&e->d_counters, 4 * sizeof(unsigned long long)));
@@ -359,9 +376,11 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     bp.counters = e->d_counters; bp.status = e->d_status;
 
     e->ctas_per_sm_wide = des_max_ctas_per_sm(e->smem);
-    e->ctas_per_sm_packed = des_packed_max_ctas_per_sm(e->smem);
-    if (e->ctas_per_sm_wide < 1 || e->ctas_per_sm_packed < 1) return fail(IL_ERR_CUDA);
-    e->ctas_per_sm = std::min(kMaxCtasPerSm, use_packed(e) ? e->ctas_per_sm_packed : e->ctas_per_sm_wide);
+    e->ctas_per_sm_packed = des_packed_max_ctas_per_sm(false, e->smem);
+    e->ctas_per_sm_staged = des_packed_max_ctas_per_sm(true, e->smem);
+    if (e->ctas_per_sm_wide < 1 || e->ctas_per_sm_packed < 1 || e->ctas_per_sm_staged < 1)
+        return fail(IL_ERR_CUDA);
+    e->ctas_per_sm = ctas_for(e);
     *out = e;
     return IL_OK;
 }
@@ -386,9 +405,9 @@ int il_set_stream(il_estimator *e, void *cuda_stream)
 
 int il_set_variant(il_estimator *e, int variant)
 {
-    if (!e || (variant != IL_VARIANT_AUTO && variant != IL_VARIANT_WIDE)) return IL_ERR_INVALID_ARG;
+    if (!e || variant < IL_VARIANT_AUTO || variant > IL_VARIANT_PACKED_DIRECT) return IL_ERR_INVALID_ARG;
     e->variant = variant;
-    e->ctas_per_sm = std::min(kMaxCtasPerSm, use_packed(e) ? e->ctas_per_sm_packed : e->ctas_per_sm_wide);
+    e->ctas_per_sm = ctas_for(e);
     return IL_OK;
 }
 
@@ -497,7 +516,7 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
         IL_CUDA(launch_order(op, st));
         const int64_t ctas = std::min<int64_t>(pl.slots / kWarpsPerCta, (cnt + kWarpsPerCta - 1) / kWarpsPerCta);
         IL_CUDA(cudaEventRecord(e->events[2 + 3 * ch], st));
-        IL_CUDA(launch_simulation(p, use_packed(e), (int)ctas, e->smem, st));
+        IL_CUDA(launch_simulation(p, sim_kernel(e), (int)ctas, e->smem, st));
         IL_CUDA(cudaEventRecord(e->events[3 + 3 * ch], st));
         SelectParams sp;
         sp.slab = p.slab; sp.slab_stride = e->n_pad; sp.lat_or = p.lat_or;

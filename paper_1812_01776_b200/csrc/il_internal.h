@@ -57,7 +57,7 @@ struct SelectParams {
 // see the handle's definition.
 struct BoundView {
     DesParams base;        // bound-input part of the kernel parameters
-    bool packed;           // which simulation kernel the handle uses
+    int kernel;            // SimKernel the handle uses
     int32_t S;
     int64_t n, n_pad, slot_elems;
     size_t smem;
@@ -68,12 +68,16 @@ struct BoundView {
 void bound_view(const il_estimator *est, BoundView *out);
 
 cudaError_t launch_des(const DesParams &p, int grid, size_t smem, cudaStream_t stream);
-cudaError_t launch_des_packed(const DesParams &p, int grid, size_t smem, cudaStream_t stream);
-int des_packed_max_ctas_per_sm(size_t smem);
-inline cudaError_t launch_simulation(const DesParams &p, bool packed, int grid, size_t smem,
+// staged: the root stage reads the trace through a shared-memory tile ring filled by bulk copies
+cudaError_t launch_des_packed(const DesParams &p, bool staged, int grid, size_t smem, cudaStream_t stream);
+int des_packed_max_ctas_per_sm(bool staged, size_t smem);
+int trace_tile_records();     // the packed trace is padded to a multiple of this many records
+enum SimKernel { kSimWide = 0, kSimPacked = 1, kSimPackedStaged = 2 };
+inline cudaError_t launch_simulation(const DesParams &p, int kernel, int grid, size_t smem,
                                      cudaStream_t stream)
 {
-    return packed ? launch_des_packed(p, grid, smem, stream) : launch_des(p, grid, smem, stream);
+    if (kernel == kSimWide) return launch_des(p, grid, smem, stream);
+    return launch_des_packed(p, kernel == kSimPackedStaged, grid, smem, stream);
 }
 cudaError_t launch_select(const SelectParams &p, cudaStream_t stream);
 

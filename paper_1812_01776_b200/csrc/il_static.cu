@@ -96,12 +96,12 @@ extern "C" int il_estimate_device_static(il_estimator *est, const il_stage_confi
     op.span_us = v.span_us;
     op.order = reinterpret_cast<int32_t *>(base + off_order);
     if (launch_order(op, st) != cudaSuccess) return IL_ERR_CUDA;
-    if (launch_simulation(p, v.packed, (int)(slots / kWarpsPerCta), v.smem, st) != cudaSuccess)
+    if (launch_simulation(p, v.kernel, (int)(slots / kWarpsPerCta), v.smem, st) != cudaSuccess)
         return IL_ERR_CUDA;
 
     SelectParams sp;
     sp.slab = p.slab; sp.slab_stride = v.n_pad; sp.lat_or = p.lat_or;
-    sp.arrival = p.arrival; sp.qbits = p.qbits; sp.packed = v.packed ? 1 : 0;
+    sp.arrival = p.arrival; sp.qbits = p.qbits; sp.packed = v.kernel != kSimWide ? 1 : 0;
     sp.n = (int32_t)v.n; sp.n_cand = n_cand; sp.slo_us = slo_us;
     sp.out_p99 = d_out_p99; sp.out_miss = d_out_miss;
     if (launch_select(sp, st) != cudaSuccess) return IL_ERR_CUDA;
