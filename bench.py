@@ -356,8 +356,8 @@ def main():
     ap.add_argument("--queries", type=int, default=None,
                     help="trace length (default: the workload's 50,000); for profiler captures")
     ap.add_argument("--variant", type=int, default=0,
-                    help="simulation kernel: 0 default (packed records, trace staged through shared "
-                         "memory), 1 wide streams, 2 packed records with direct trace reads")
+                    help="simulation kernel: 0 default (packed records), 1 wide streams, "
+                         "2 packed records with the trace staged through shared memory")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer timing (profiler captures)")
     args = ap.parse_args()
     if args.impl == "reference":

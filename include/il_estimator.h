@@ -243,17 +243,19 @@ IL_API int il_set_workspace(il_estimator *est, void *d_workspace, size_t bytes);
  * Chooses the simulation kernel.  IL_VARIANT_AUTO (default) uses the
  * packed-record kernel whenever every time the simulation can reach (last
  * arrival + sum over stages of n * largest table entry) fits in
- * 63 - max(5, ceil(log2 n)) bits, with the shared trace staged through shared
- * memory once per CTA (bulk asynchronous copies into a ring of tiles), and the
- * kernel with separate 64-bit time and 32-bit query streams otherwise.
- * IL_VARIANT_WIDE forces the latter (it is always valid; used to test it).
- * IL_VARIANT_PACKED_DIRECT is the packed-record kernel with every warp reading
- * the trace through the caches on its own instead of the staged tiles.  All
- * give identical results.
+ * 63 - max(5, ceil(log2 n)) bits, and the kernel with separate 64-bit time and
+ * 32-bit query streams otherwise.  IL_VARIANT_WIDE forces the latter (it is
+ * always valid; used to test it).  IL_VARIANT_STAGED is the packed-record
+ * kernel with the shared trace staged through shared memory once per CTA (bulk
+ * asynchronous copies into a ring of tiles that the CTA's four warps consume
+ * together) instead of every warp reading it through L1/L2 on its own; on B200
+ * it measured slower than the default (the warps of a CTA must then move
+ * through the root stage within one ring length of each other), so it is not
+ * the default.  All variants give identical results.
  */
 #define IL_VARIANT_AUTO 0
 #define IL_VARIANT_WIDE 1
-#define IL_VARIANT_PACKED_DIRECT 2
+#define IL_VARIANT_STAGED 2
 IL_API int il_set_variant(il_estimator *est, int variant);
 
 /* Counters of the last estimate call on this handle. */

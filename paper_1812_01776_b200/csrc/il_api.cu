@@ -61,10 +61,13 @@ struct il_estimator {
 
 namespace {
 
-// Resident CTAs per SM are capped below the occupancy limit: on B200, 24 warps
-// per SM (6 CTAs) measured faster than 28 on the 4,096-candidate workload (each
-// warp is a long dependent chain; more resident warps only add cache pressure).
-constexpr int kMaxCtasPerSm = 6;
+// When a chunk fits the GPU in about one wave (at most 1.5 candidates per warp
+// slot), resident CTAs per SM are capped below the occupancy limit: on B200, 24
+// warps per SM (6 CTAs) measured faster than 28 on the 4,096-candidate workload
+// (each warp is a long dependent chain and the kernel ends with its slowest
+// warp; fewer co-resident warps let the long ones run faster).  Larger chunks
+// are throughput-bound and use every slot.
+constexpr int kOneWaveCtasPerSm = 6;
 
 struct Plan {
     int64_t slots = 0;       // warp slots with stream buffers
@@ -198,15 +201,14 @@ bool use_packed(const il_estimator *e)
 int sim_kernel(const il_estimator *e)
 {
     if (!use_packed(e)) return kSimWide;
-    return e->variant == IL_VARIANT_PACKED_DIRECT ? kSimPacked : kSimPackedStaged;
+    return e->variant == IL_VARIANT_STAGED ? kSimPackedStaged : kSimPacked;
 }
 
 int ctas_for(const il_estimator *e)
 {
     const int k = sim_kernel(e);
-    const int occ = k == kSimWide ? e->ctas_per_sm_wide
-                  : k == kSimPacked ? e->ctas_per_sm_packed : e->ctas_per_sm_staged;
-    return std::min(kMaxCtasPerSm, occ);
+    return k == kSimWide ? e->ctas_per_sm_wide
+         : k == kSimPacked ? e->ctas_per_sm_packed : e->ctas_per_sm_staged;
 }
 
 void free_device(il_estimator *e)
@@ -405,7 +407,7 @@ int il_set_stream(il_estimator *e, void *cuda_stream)
 
 int il_set_variant(il_estimator *e, int variant)
 {
-    if (!e || variant < IL_VARIANT_AUTO || variant > IL_VARIANT_PACKED_DIRECT) return IL_ERR_INVALID_ARG;
+    if (!e || variant < IL_VARIANT_AUTO || variant > IL_VARIANT_STAGED) return IL_ERR_INVALID_ARG;
     e->variant = variant;
     e->ctas_per_sm = ctas_for(e);
     return IL_OK;
@@ -514,7 +516,9 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
         op.order = reinterpret_cast<int32_t *>(ws + pl.off_order);
         if (ch > 0) IL_CUDA(cudaMemsetAsync(e->d_counters, 0, sizeof(unsigned long long), st));
         IL_CUDA(launch_order(op, st));
-        const int64_t ctas = std::min<int64_t>(pl.slots / kWarpsPerCta, (cnt + kWarpsPerCta - 1) / kWarpsPerCta);
+        int64_t ctas = std::min<int64_t>(pl.slots / kWarpsPerCta, (cnt + kWarpsPerCta - 1) / kWarpsPerCta);
+        if (2 * cnt <= 3 * full_slots(e))
+            ctas = std::min<int64_t>(ctas, (int64_t)e->num_sms * std::min(e->ctas_per_sm, kOneWaveCtasPerSm));
         IL_CUDA(cudaEventRecord(e->events[2 + 3 * ch], st));
         IL_CUDA(launch_simulation(p, sim_kernel(e), (int)ctas, e->smem, st));
         IL_CUDA(cudaEventRecord(e->events[3 + 3 * ch], st));

@@ -22,7 +22,7 @@ IL_OK = 0
 IL_ERR_INVALID_ARG, IL_ERR_BAD_TOPOLOGY, IL_ERR_BAD_PROFILE, IL_ERR_BAD_TRACE = -1, -2, -3, -4
 IL_ERR_BAD_CONFIG, IL_ERR_NOMEM, IL_ERR_CUDA, IL_ERR_ITER_LIMIT = -5, -6, -7, -8
 IL_ERR_TOO_LARGE = -9
-IL_VARIANT_AUTO, IL_VARIANT_WIDE, IL_VARIANT_PACKED_DIRECT = 0, 1, 2
+IL_VARIANT_AUTO, IL_VARIANT_WIDE, IL_VARIANT_STAGED = 0, 1, 2
 IL_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 EXPORTS = ["il_estimator_create", "il_estimator_destroy", "il_estimate", "il_estimate_device",
@@ -296,7 +296,7 @@ class Estimator:
         return self._ws.numel()
 
     def set_variant(self, variant: int) -> None:
-        """IL_VARIANT_AUTO, IL_VARIANT_WIDE or IL_VARIANT_PACKED_DIRECT (see il_set_variant)."""
+        """IL_VARIANT_AUTO, IL_VARIANT_WIDE or IL_VARIANT_STAGED (see il_set_variant)."""
         il_set_variant(self._h, variant)
 
     def use_current_stream(self) -> None:
