@@ -132,6 +132,7 @@ __device__ __forceinline__ void tile_issue(TileRing *ring, const uint64_t *ptrac
 }
 
 struct GlobalSrc {
+    static constexpr bool kRereadable = true;
     const uint64_t *in;
     bool root;               // the packed trace: the query of record i is i
     // 32 consecutive records starting at the 32-aligned index `idx0`
@@ -147,6 +148,7 @@ struct GlobalSrc {
 };
 
 struct TileSrc {
+    static constexpr bool kRereadable = false;   // released tiles are gone
     TileRing *ring;
     const uint64_t *ptrace;
     int n_tiles;
@@ -235,6 +237,17 @@ __device__ __forceinline__ void append(const WarpCtx &w, Sink &sk, const uint64_
     }
 }
 
+// Where a stage stands when the 32-bit loop (run_stage_narrow) hands it over to
+// the 64-bit loop (run_stage).
+struct StageState {
+    bool resume;         // false: start the stage from scratch
+    int head;            // arrivals consumed so far
+    int nbatch;          // batches dispatched so far
+    uint64_t key;        // this lane's slot
+    int sl_b;
+    uint32_t sl_q;
+};
+
 // One stage of one candidate, max batch >= 2.  WIDE: max batch > 32 (the queue
 // count looks at up to 64 arrivals).  Returns the number of batches dispatched.
 //
@@ -242,8 +255,8 @@ __device__ __forceinline__ void append(const WarpCtx &w, Sink &sk, const uint64_
 // be reused is lane 0 and the one after it lane 1.
 template <bool WIDE, int KIND, class Src>
 __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, const int mb,
-                                         const int R, const int n_in, Src &src, Sink &sk,
-                                         int *status)
+                                      const int R, const int n_in, Src &src, Sink &sk,
+                                      int *status, const StageState &st)
 {
     const unsigned full = 0xffffffffu;
     const int lane = w.lane;
@@ -274,18 +287,19 @@ __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, c
     uint64_t key = (lane < R) ? (uint64_t)lane : kNeverKey;
     int sl_b = 0;            // size of the batch the slot holds (0: none)
     uint32_t sl_q = 0;       // its first query
+    int head = 0, nbatch = 0;
+    if (st.resume) { key = st.key; sl_b = st.sl_b; sl_q = st.sl_q; head = st.head; nbatch = st.nbatch; }
 
     // lookahead window: A, B, C, D hold in[base + 32 k + lane]
-    int base = 0, off = 0, head = 0;
-    uint64_t A = src.load32(0, lane, n_in), B = src.load32(32, lane, n_in),
-             C = src.load32(64, lane, n_in), D = src.load32(96, lane, n_in);
+    int base = head & ~31, off = head & 31;
+    uint64_t A = src.load32(base, lane, n_in), B = src.load32(base + 32, lane, n_in),
+             C = src.load32(base + 64, lane, n_in), D = src.load32(base + 96, lane, n_in);
 
-    int nbatch = 0;
     int cooldown = 0, penalty = 1;   // when to try the run step again after it did not pay off
     // the slot in lane 0, known to every lane
-    uint64_t m1 = 0;
-    int pb1 = 0;
-    uint32_t pq1 = 0;
+    uint64_t m1 = __shfl_sync(full, key, 0);
+    int pb1 = __shfl_sync(full, sl_b, 0);
+    uint32_t pq1 = __shfl_sync(full, sl_q, 0);
 
     while (head < n_in) {
         // ------------------------------------------------------------------
@@ -462,6 +476,280 @@ __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, c
     return nbatch;
 }
 
+// ---------------------------------------------------------------------------
+// The same stage loop in 32-bit arithmetic.
+//
+// Times are kept relative to an epoch E (a 64-bit value known to every lane),
+// as unsigned 32-bit offsets below kNarrowLimit; a slot is (finish offset,
+// start index) in two registers, ordered by finish and, at equal finish, by
+// start -- since a new batch starts after every batch in flight, "<=" on the
+// finish offsets alone decides where it goes.  Everything else is the 64-bit
+// loop above, instruction for instruction at half the width.  When an offset
+// would leave the range the epoch is moved forward to the oldest time still
+// needed (the head arrival, or the finish of the oldest batch not yet handed
+// over); if that does not help (a batch or a gap in the arrivals spans more than
+// the range) the stage continues in the 64-bit loop from the state reached.
+// Needs every table entry of the row to be below kNarrowLatLimit.
+// ---------------------------------------------------------------------------
+constexpr uint32_t kNarrowLimit = 1u << 30;
+constexpr uint32_t kNarrowLatLimit = 1u << 24;     // 32 services still fit below the limit
+constexpr uint32_t kFar = 0x7fffffffu;             // an arrival beyond the range (still a real record)
+constexpr uint32_t kNever32 = 0xffffffffu;         // no record
+
+template <bool WIDE, int KIND, class Src>
+__device__ __forceinline__ int run_stage_narrow(const WarpCtx &w, const int32_t *row, const int mb,
+                                             const int R, const int n_in, Src &src, Sink &sk,
+                                             int *status)
+{
+    const unsigned full = 0xffffffffu;
+    const int lane = w.lane;
+    const uint32_t qmask = w.qmask;
+    const int qb = w.qbits;
+    const uint32_t d1 = (uint32_t)row[0];
+
+    uint64_t E = 0;                                 // epoch, set from the first arrival below
+
+    auto mkrec = [&](const uint32_t fin, const uint32_t q) -> uint64_t {
+        return ((E + fin) << qb) | q;
+    };
+    // Hands over the batch a slot held (b queries from input index `start`, finished at offset fin).
+    auto emit = [&](const uint32_t fin, const int b, const uint32_t q_first, const int start) {
+        if (b == 1) {
+            append<KIND>(w, sk, mkrec(fin, q_first), 1);
+            return;
+        }
+#pragma unroll 1
+        for (int j0 = 0; j0 < b; j0 += 32) {
+            const int j = j0 + lane;
+            uint64_t rec = 0;
+            if (j < b) rec = mkrec(fin, src.query_at(start + j, qmask));
+            append<KIND>(w, sk, rec, min(32, b - j0));
+        }
+    };
+
+    // slots, sorted over lanes 0..R-1 by (fin, sl_s); never-used slots have fin 0 and hold nothing
+    uint32_t fin = (lane < R) ? 0u : kNever32;
+    int sl_b = 0, sl_s = lane;
+    uint32_t sl_q = 0;
+
+    int base = 0, off = 0, head = 0, nbatch = 0;
+    uint32_t At, Bt, Ct, Dt, Aq, Bq, Cq, Dq;
+    auto load_win = [&](const int idx0, uint32_t &t, uint32_t &q) {
+        const uint64_t rec = src.load32(idx0, lane, n_in);
+        q = (uint32_t)rec & qmask;
+        if (rec == kNeverKey) { t = kNever32; return; }
+        const uint64_t rel = (rec >> qb) - E;       // arrivals before the epoch only occur in a backlog:
+        t = (rec >> qb) < E ? 0u                    //   "already there" is all that matters
+          : (rel >= kNarrowLimit ? kFar : (uint32_t)rel);
+    };
+    {
+        const uint64_t first = src.load32(0, lane, n_in);
+        E = __shfl_sync(full, first, 0) >> qb;
+    }
+    load_win(0, At, Aq); load_win(32, Bt, Bq); load_win(64, Ct, Cq); load_win(96, Dt, Dq);
+
+    int cooldown = 0, penalty = 1;
+    uint32_t m1 = 0; int pb1 = 0, ps1 = 0; uint32_t pq1 = 0;    // the slot in lane 0
+    bool bail = false;
+
+    // Moves the epoch forward to the oldest time still needed.  Returns false if that is no progress.
+    auto re_epoch = [&]() -> bool {
+        const uint32_t ah = __shfl_sync(full, off < 32 ? At : Bt, off & 31);
+        const uint32_t held = __reduce_min_sync(full, (lane < R && sl_b > 0) ? fin : kNever32);
+        const uint32_t delta = min(ah == kFar ? kNever32 : ah, held);
+        uint32_t d = delta;
+        if (ah == kFar && held == kNever32) {
+            // nothing in flight and the next arrival is beyond the range: jump to it
+            const uint64_t rec = src.load32(head & ~31, lane, n_in);
+            const uint64_t t = __shfl_sync(full, rec, head & 31) >> qb;
+            E = t; d = 0;
+            if (lane < R) fin = 0;
+        } else {
+            if (d == 0 || d == kNever32) return false;
+            E += d;
+            if (lane < R) fin = fin > d ? fin - d : 0u;
+        }
+        load_win(base, At, Aq); load_win(base + 32, Bt, Bq); load_win(base + 64, Ct, Cq); load_win(base + 96, Dt, Dq);
+        m1 = __shfl_sync(full, fin, 0);
+        return true;
+    };
+
+    while (head < n_in) {
+        // the head arrival must be in range to be dispatched here
+        {
+            const uint32_t ah = __shfl_sync(full, At, off);
+            if (ah >= kNarrowLimit / 2 || m1 >= kNarrowLimit / 2) {
+                if (ah == kNever32) break;      // cannot happen while head < n_in
+                if (!re_epoch()) { bail = true; break; }
+                const uint32_t ah2 = __shfl_sync(full, At, off);
+                if (ah2 >= kNarrowLimit / 2 || __shfl_sync(full, fin, 0) >= kNarrowLimit / 2) { bail = true; break; }
+            }
+        }
+        // ---------------- run step (see run_stage) ----------------
+        if (cooldown == 0) {
+            const int pos = off + lane;
+            const uint32_t xa = __shfl_sync(full, At, pos & 31), xb = __shfl_sync(full, Bt, pos & 31);
+            const uint32_t X = pos < 32 ? xa : xb;
+            const uint32_t Xn = __shfl_down_sync(full, X, 1);
+            const bool valid = X < kNarrowLimit / 2;
+            uint32_t v = (lane < R && fin > X) ? fin : X;
+            uint32_t mul = d1;
+            for (int d = R; d < 32; d <<= 1, mul <<= 1) {
+                const uint32_t u = __shfl_up_sync(full, v, d);
+                if (lane >= d && valid && u + mul > v) v = u + mul;
+            }
+            const uint32_t f0 = __shfl_sync(full, v, 0) + d1;
+            // a start beyond half the range ends the run (the epoch moves before the next step)
+            const bool ok = valid && (lane < 31) && (Xn > v) && (v < kNarrowLimit / 2);
+            int m = __ffs(~__ballot_sync(full, ok)) - 1;
+            const int c0 = __popc(__ballot_sync(full, lane < R && fin <= f0));
+            if (c0 < R) m = min(m, c0);
+            if (m >= kMinRun) {
+                const uint32_t NF = v + d1;
+                const uint32_t qa = __shfl_sync(full, Aq, pos & 31), qb2 = __shfl_sync(full, Bq, pos & 31);
+                const uint32_t xq = pos < 32 ? qa : qb2;
+                const int z = __popc(__ballot_sync(full, lane < R && sl_b == 0));
+                const int n_old = min(m, R);
+                const uint64_t oldrec = mkrec(fin, sl_q);
+                unsigned multi = __ballot_sync(full, lane < n_old && sl_b > 1);
+                int p0 = min(z, n_old);
+                while (p0 < n_old) {
+                    const int nxt = multi ? __ffs(multi) - 1 : n_old;
+                    if (nxt > p0) append<KIND>(w, sk, __shfl_sync(full, oldrec, (lane + p0) & 31), nxt - p0);
+                    if (nxt < n_old) {
+                        emit(__shfl_sync(full, fin, nxt), __shfl_sync(full, sl_b, nxt),
+                             __shfl_sync(full, sl_q, nxt), __shfl_sync(full, sl_s, nxt));
+                        multi &= multi - 1;
+                    }
+                    p0 = nxt + 1;
+                }
+                if (m > R) append<KIND>(w, sk, mkrec(NF, xq), m - R);
+                if (c0 >= R) {
+                    const bool take_old = m + lane < R;
+                    const int src_old = (m + lane) & 31, src_new = (m + lane - R) & 31;
+                    const uint32_t f_o = __shfl_sync(full, fin, src_old), f_n = __shfl_sync(full, NF, src_new);
+                    const uint32_t q_o = __shfl_sync(full, sl_q, src_old), q_n = __shfl_sync(full, xq, src_new);
+                    const int b_o = __shfl_sync(full, sl_b, src_old);
+                    const int s_o = __shfl_sync(full, sl_s, src_old);
+                    if (lane < R) {
+                        fin = take_old ? f_o : f_n;
+                        sl_q = take_old ? q_o : q_n;
+                        sl_b = take_old ? b_o : 1;
+                        sl_s = take_old ? s_o : head + src_new;
+                    }
+                } else {
+                    int above = 0, below = 0;
+                    for (int r = c0; r < R; r++) {
+                        const uint32_t fr = __shfl_sync(full, fin, r);
+                        const unsigned lt = __ballot_sync(full, lane < m && NF < fr);
+                        above += (fr <= NF);
+                        if (lane == r) below = __popc(lt);
+                    }
+                    // re-ordering through shared memory: key holds the finish offset, q and b as usual,
+                    // the start index travels in the upper half of the key word
+                    if (lane >= m && lane < R) {
+                        const int dst = lane < c0 ? lane - m : lane - m + below;
+                        w.slot_key[dst] = ((uint64_t)(uint32_t)sl_s << 32) | fin; w.slot_q[dst] = sl_q; w.slot_b[dst] = sl_b;
+                    }
+                    if (lane < m) {
+                        const int dst = c0 - m + lane + above;
+                        w.slot_key[dst] = ((uint64_t)(uint32_t)(head + lane) << 32) | NF; w.slot_q[dst] = xq; w.slot_b[dst] = 1;
+                    }
+                    __syncwarp();
+                    if (lane < R) {
+                        const uint64_t k = w.slot_key[lane];
+                        fin = (uint32_t)k; sl_s = (int)(k >> 32); sl_q = w.slot_q[lane]; sl_b = w.slot_b[lane];
+                    }
+                    __syncwarp();
+                }
+                penalty = 1;
+                head += m; off += m; nbatch += m;
+                while (off >= 32) {
+                    At = Bt; Bt = Ct; Ct = Dt; Aq = Bq; Bq = Cq; Cq = Dq;
+                    base += 32;
+                    load_win(base + 96, Dt, Dq);
+                    off -= 32;
+                }
+                m1 = __shfl_sync(full, fin, 0);
+                pb1 = __shfl_sync(full, sl_b, 0);
+                pq1 = __shfl_sync(full, sl_q, 0);
+                ps1 = __shfl_sync(full, sl_s, 0);
+                continue;
+            }
+            cooldown = penalty;
+            penalty = min(penalty * 2, 64);
+        }
+        if (cooldown > 0) cooldown--;
+
+        // ---------------- single step ----------------
+        const uint32_t m2 = __shfl_sync(full, fin, 1);
+        const int pb2 = __shfl_sync(full, sl_b, 1), ps2 = __shfl_sync(full, sl_s, 1);
+        const uint32_t pq2 = __shfl_sync(full, sl_q, 1);
+        const uint32_t a_head = __shfl_sync(full, At, off);
+        const uint32_t qh = __shfl_sync(full, Aq, off);
+        const uint32_t t = max(m1, a_head);
+        const unsigned mA = __ballot_sync(full, At <= t);
+        const unsigned mB = __ballot_sync(full, Bt <= t);
+        int cnt = __popc(__funnelshift_r(mA, mB, off));
+        if (WIDE) {
+            const unsigned mC = __ballot_sync(full, Ct <= t);
+            cnt += __popc(__funnelshift_r(mB, mC, off));
+        }
+        cnt = min(cnt, mb);
+        if (cnt < 1) {
+            if (lane == 0) atomicCAS(status, 0, IL_ERR_ITER_LIMIT);
+            break;
+        }
+        const uint32_t nf = t + (uint32_t)row[cnt - 1];      // < 2^29 + 2^24: in range
+
+        if (pb1 > 0) emit(m1, pb1, pq1, ps1);
+
+        uint32_t u = __shfl_down_sync(full, fin, 1);
+        const int ub = __shfl_down_sync(full, sl_b, 1), us = __shfl_down_sync(full, sl_s, 1);
+        const uint32_t uq = __shfl_down_sync(full, sl_q, 1);
+        if (lane == 31) u = kNever32;
+        const bool le = u <= nf;                              // equal finish: the older batch first
+        const bool here = __ballot_sync(full, le) == w.lt_mask;
+        fin = le ? u : (here ? nf : fin);
+        sl_b = le ? ub : (here ? cnt : sl_b);
+        sl_q = le ? uq : (here ? qh : sl_q);
+        sl_s = le ? us : (here ? head : sl_s);
+        const bool second_first = m2 <= nf;
+        m1 = second_first ? m2 : nf;
+        pb1 = second_first ? pb2 : cnt;
+        pq1 = second_first ? pq2 : qh;
+        ps1 = second_first ? ps2 : head;
+
+        head += cnt;
+        off += cnt;
+        nbatch++;
+        while (off >= 32) {
+            At = Bt; Bt = Ct; Ct = Dt; Aq = Bq; Bq = Cq; Cq = Dq;
+            base += 32;
+            load_win(base + 96, Dt, Dq);
+            off -= 32;
+        }
+    }
+    if (bail) {
+        // continue in 64-bit arithmetic from here
+        StageState st;
+        st.resume = true; st.head = head; st.nbatch = nbatch;
+        st.key = lane < R ? (((E + fin) << qb) | (uint32_t)sl_s) : kNeverKey;
+        if (lane < R && sl_b == 0) st.key = (uint64_t)lane;     // never-used slots keep their tiny keys
+        st.sl_b = sl_b; st.sl_q = sl_q;
+        return run_stage<WIDE, KIND>(w, row, mb, R, n_in, src, sk, status, st);
+    }
+#pragma unroll 1
+    for (int r = 0; r < R; r++) {
+        const uint32_t f = __shfl_sync(full, fin, r);
+        const int pb = __shfl_sync(full, sl_b, r), ps = __shfl_sync(full, sl_s, r);
+        const uint32_t pq = __shfl_sync(full, sl_q, r);
+        if (pb > 0) emit(f, pb, pq, ps);
+    }
+    src.finish(lane, n_in);
+    return nbatch;
+}
+
 // A stage whose max batch is 1.  Every batch is a single query with the same
 // service time D = latency[1], so the multi-replica FIFO queue behaves like R
 // interleaved single-server queues: query i starts at
@@ -515,11 +803,24 @@ __device__ __forceinline__ int dispatch_stage(const WarpCtx &w, const int32_t *r
     if (mb == 1)
         return branch ? run_stage_mb1<kBranch>(w, row, R, n_in, src, sk)
                       : run_stage_mb1<kForward>(w, row, R, n_in, src, sk);
+    // the 32-bit loop needs small table entries and a source it may read twice
+    uint32_t row_max = 0;
+    for (int b = w.lane; b < mb; b += 32) row_max = max(row_max, (uint32_t)row[b]);
+    row_max = __reduce_max_sync(0xffffffffu, row_max);
+    if (Src::kRereadable && row_max < kNarrowLatLimit) {
+        if (mb > 32)
+            return branch ? run_stage_narrow<true, kBranch>(w, row, mb, R, n_in, src, sk, status)
+                          : run_stage_narrow<true, kForward>(w, row, mb, R, n_in, src, sk, status);
+        return branch ? run_stage_narrow<false, kBranch>(w, row, mb, R, n_in, src, sk, status)
+                      : run_stage_narrow<false, kForward>(w, row, mb, R, n_in, src, sk, status);
+    }
+    StageState st;
+    st.resume = false;
     if (mb > 32)
-        return branch ? run_stage<true, kBranch>(w, row, mb, R, n_in, src, sk, status)
-                      : run_stage<true, kForward>(w, row, mb, R, n_in, src, sk, status);
-    return branch ? run_stage<false, kBranch>(w, row, mb, R, n_in, src, sk, status)
-                  : run_stage<false, kForward>(w, row, mb, R, n_in, src, sk, status);
+        return branch ? run_stage<true, kBranch>(w, row, mb, R, n_in, src, sk, status, st)
+                      : run_stage<true, kForward>(w, row, mb, R, n_in, src, sk, status, st);
+    return branch ? run_stage<false, kBranch>(w, row, mb, R, n_in, src, sk, status, st)
+                  : run_stage<false, kForward>(w, row, mb, R, n_in, src, sk, status, st);
 }
 
 // Simulates candidate `c` of the chunk on this warp.  STAGED: the root stage
