@@ -31,7 +31,14 @@ if ROOT not in sys.path:
 
 import workloads  # noqa: E402
 
-WORKLOAD_ID = 2
+WORKLOAD_ID = 2          # the benchmark workload; --workload picks another one for side measurements
+WORKLOADS = {
+    1: "config1: linear 2-stage pipeline, 2,000 Poisson arrivals (100 qps), 64 candidates",
+    2: "config2: linear 4-stage image pipeline, 50,000 gamma arrivals (200 qps, CV 4), 4,096 candidates",
+    3: "config3: 6-stage tree with one branch point, 200,000 gamma arrivals (300 qps, CV 1), 65,536 candidates",
+    4: "config4: linear 10-stage pipeline, 1,000,000 arrivals ramping 150->250 qps, 262,144 candidates",
+    5: "config5: 8-stage tree with three branch points, 100,000 gamma arrivals (500 qps, CV 2), 1,048,576 candidates",
+}
 METRIC = "candidate_configs_per_s"
 UNIT = "candidates/s"
 
@@ -159,7 +166,8 @@ def run_reference(args):
     rank, world, _ = dist_env()
     if rank != 0:
         return
-    w = workloads.make(WORKLOAD_ID)
+    w = workloads.make(args.workload, n_queries=args.queries,
+                       n_candidates=min(args.candidates or 10**9, 4096, workloads.FULL_SIZES[args.workload][1]))
     cores = os.cpu_count() or 1
     per_step = max(cores, min(w.n_candidates, 8 * cores))
     for _ in range(min(args.warmup, 1)):
@@ -167,15 +175,15 @@ def run_reference(args):
     times = [time_oracle(w, per_step, cores) for _ in range(args.steps)]
     sec = sum(times) / len(times)
     value = per_step / sec
-    sample = (f"first {per_step} of {w.n_candidates} candidates per step, full 50,000-query trace, "
+    sample = (f"first {per_step} of {workloads.FULL_SIZES[args.workload][1]} candidates per step, "
+              f"{w.n_queries}-query trace, "
               f"{cores} processes each running the single-threaded oracle on a disjoint slice")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
         "data": "synthetic",
-        "config": {"workload": "config2: linear 4-stage image pipeline, 50,000 gamma arrivals "
-                               "(200 qps, CV 4), 4,096 candidates", "sampled_candidates_per_step": per_step},
+        "config": {"workload": WORKLOADS[args.workload], "sampled_candidates_per_step": per_step},
         "query_events_per_s": value * w.query_events(),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -201,8 +209,8 @@ def run_cuda(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    per_rank = args.candidates or workloads.FULL_SIZES[WORKLOAD_ID][1]
-    w = workloads.make(WORKLOAD_ID, n_queries=args.queries, n_candidates=per_rank * world)
+    per_rank = args.candidates or workloads.FULL_SIZES[args.workload][1]
+    w = workloads.make(args.workload, n_queries=args.queries, n_candidates=per_rank * world)
     lo, hi = shard_range(w.n_candidates, rank, world)
     cfg_host = np.ascontiguousarray(w.configs[lo:hi])
     n_cand = hi - lo
@@ -295,7 +303,8 @@ def run_cuda(args):
     alu_achieved = alg_ops / sim_avg_s
     # HBM view of the same kernel: slab written once, streams written and read once, trace once per CTA wave
     n, S = w.n_queries, w.n_stages
-    stream_bytes = (events_per_cand - n) * (12 + 12)
+    rec_bytes = 12 if args.variant == 1 else 8       # wide: int64 time + int32 query; packed: one 64-bit record
+    stream_bytes = (events_per_cand - n) * 2 * rec_bytes
     hbm_bytes_per_cand = 8 * n + stream_bytes + 4 * S
     hbm_achieved = hbm_bytes_per_cand * n_cand / sim_avg_s / 1e9
 
@@ -303,9 +312,8 @@ def run_cuda(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": args.warmup, "ms_per_step": total_ms / K, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-        "config": {"workload": "config2: linear 4-stage image pipeline, 50,000 gamma arrivals "
-                               "(200 qps, CV 4), 4,096 candidates per GPU"
-                               + ("" if not (args.candidates or args.queries) else " [REDUCED for profiling]"),
+        "config": {"workload": WORKLOADS[args.workload] + " per GPU"
+                               + ("" if not (args.candidates or args.queries) else " [candidates/queries overridden]"),
                    "candidates_per_gpu": n_cand, "queries": n, "stages": S,
                    "query_events_per_candidate": events_per_cand,
                    "l2": "256 MiB buffer written between steps; working set "
@@ -318,12 +326,13 @@ def run_cuda(args):
         "kernel_ms": {"simulate": sum(sim_ms) / K, "select": sum(sel_ms) / K},
         "roofline": {"bound": "alu", "achieved": alu_achieved / 1e12, "peak": alu_peak / 1e12,
                      "unit": "Tinteger-op/s", "frac": alu_achieved / alu_peak, "traffic": None,
-                     "kernel": "des_kernel",
+                     "kernel": "des_kernel" if args.variant == 1 else "des_packed_kernel",
                      "peak_source": "integer-issue probe of this run (warp-inst/s x 32 lanes)",
                      "issue_peak_warp_inst_per_s": issue_rate},
         "roofline_hbm": {"bound": "hbm", "achieved": hbm_achieved, "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": hbm_achieved / peaks["hbm_gbs"],
-                         "peak_source": f"{peaks_kind} copy bandwidth", "kernel": "des_kernel"},
+                         "peak_source": f"{peaks_kind} copy bandwidth",
+                         "kernel": "des_kernel" if args.variant == 1 else "des_packed_kernel"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(cfg_host.nbytes),
                 "d2h_bytes_per_step": int(16 * n_cand), "matches_device_path": same},
         "gpu_launches": int(launches),
@@ -331,15 +340,17 @@ def run_cuda(args):
     }
     if world == 1 and not args.no_cpu_baseline:
         cores = os.cpu_count() or 1
-        n_sample = min(w.n_candidates, 16 * cores)
+        per_cand_s = w.query_events() / 4.5e6            # the oracle does a few million query-events/s/core
+        n_sample = int(max(cores, min(w.n_candidates, 16 * cores, 12.0 * cores / per_cand_s)))
+        n_one = int(max(1, min(64, w.n_candidates, 4.0 / per_cand_s)))
         sec = time_oracle(w, n_sample, cores)
-        sec1 = time_oracle(w, min(64, w.n_candidates), 1)
+        sec1 = time_oracle(w, n_one, 1)
         line["cpu_baseline"] = {
             "value": n_sample / sec, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"first {n_sample} of {w.n_candidates} candidates, full trace, {cores} "
-                      f"processes x single-threaded oracle; 1 core on {min(64, w.n_candidates)} candidates: "
-                      f"{min(64, w.n_candidates) / sec1:.1f} candidates/s",
-            "one_core_value": min(64, w.n_candidates) / sec1}
+                      f"processes x single-threaded oracle; 1 core on {n_one} candidates: "
+                      f"{n_one / sec1:.1f} candidates/s",
+            "one_core_value": n_one / sec1}
     print(json.dumps(line))
 
 
@@ -350,6 +361,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", type=int, default=WORKLOAD_ID, choices=[1, 2, 3, 4, 5],
+                    help="which of the five workloads (default 2, the one the metric is quoted on)")
     ap.add_argument("--candidates", type=int, default=None,
                     help="candidates per GPU (default: the workload's 4,096); smaller values are "
                          "for profiler captures, not for reported numbers")
