@@ -146,8 +146,10 @@ class ClockSampler:
 # the oracle arm (CPU); also used for the cpu_baseline object
 # ----------------------------------------------------------------------------
 
-def time_oracle(w, n_sample: int, processes: int):
-    """Times the CPU oracle, as it stands, on the first n_sample candidates."""
+def time_oracle(w, n_sample: int, processes: int, pool=None):
+    """Times the CPU oracle, as it stands, on the first n_sample candidates.
+    With a pool (already started, see oracle.make_pool) the timed region holds
+    only the simulation and the hand-over of inputs and results."""
     import oracle
     oracle.build()
     cfg = w.configs[:n_sample]
@@ -158,7 +160,7 @@ def time_oracle(w, n_sample: int, processes: int):
     else:
         oracle.estimate_many_parallel(w.parent, w.cond_bit, w.cond_val, w.latency_us,
                                       w.arrival_us, w.branch_bits, cfg, w.slo_us,
-                                      processes=processes)
+                                      processes=processes, pool=pool)
     return time.perf_counter() - t0
 
 
@@ -169,10 +171,14 @@ def run_reference(args):
     w = workloads.make(args.workload, n_queries=args.queries,
                        n_candidates=min(args.candidates or 10**9, 4096, workloads.FULL_SIZES[args.workload][1]))
     cores = os.cpu_count() or 1
+    import oracle
     per_step = max(cores, min(w.n_candidates, 8 * cores))
+    pool = oracle.make_pool(cores) if cores > 1 else None
     for _ in range(min(args.warmup, 1)):
-        time_oracle(w, cores, cores)
-    times = [time_oracle(w, per_step, cores) for _ in range(args.steps)]
+        time_oracle(w, cores, cores, pool)
+    times = [time_oracle(w, per_step, cores, pool) for _ in range(args.steps)]
+    if pool is not None:
+        pool.terminate()
     sec = sum(times) / len(times)
     value = per_step / sec
     sample = (f"first {per_step} of {workloads.FULL_SIZES[args.workload][1]} candidates per step, "
@@ -343,7 +349,11 @@ def run_cuda(args):
         per_cand_s = w.query_events() / 4.5e6            # the oracle does a few million query-events/s/core
         n_sample = int(max(cores, min(w.n_candidates, 16 * cores, 12.0 * cores / per_cand_s)))
         n_one = int(max(1, min(64, w.n_candidates, 4.0 / per_cand_s)))
-        sec = time_oracle(w, n_sample, cores)
+        import oracle
+        pool = oracle.make_pool(cores) if cores > 1 else None
+        sec = time_oracle(w, n_sample, cores, pool)
+        if pool is not None:
+            pool.terminate()
         sec1 = time_oracle(w, n_one, 1)
         line["cpu_baseline"] = {
             "value": n_sample / sec, "unit": UNIT, "cores": cores, "kind": "oracle",

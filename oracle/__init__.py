@@ -150,8 +150,25 @@ def _worker(args):
                          configs, slo_us)
 
 
+def _noop(_):
+    return os.getpid()
+
+
+def make_pool(processes: Optional[int] = None):
+    """A pool of worker processes (``spawn`` start method, so it is safe to
+    create after a CUDA context exists in the parent) that have the oracle
+    library loaded.  Pass it to estimate_many_parallel to keep process start-up
+    out of a timed region; close it with ``pool.terminate()``."""
+    import multiprocessing as mp
+    build()
+    P = max(1, processes or (os.cpu_count() or 1))
+    pool = mp.get_context("spawn").Pool(P)
+    pool.map(_noop, range(4 * P), chunksize=1)      # make every worker import this module
+    return pool
+
+
 def estimate_many_parallel(parent, cond_bit, cond_val, latency_us, arrival_us, branch_bits,
-                           configs, slo_us: int, processes: Optional[int] = None):
+                           configs, slo_us: int, processes: Optional[int] = None, pool=None):
     """Disjoint slices of the candidates on separate processes (each candidate
     is still simulated by one thread).  Uses the ``spawn`` start method so it is
     safe to call after a CUDA context exists in the parent."""
@@ -160,6 +177,13 @@ def estimate_many_parallel(parent, cond_bit, cond_val, latency_us, arrival_us, b
     configs = np.ascontiguousarray(configs, dtype=np.uint8)
     C = configs.shape[0]
     P = max(1, min(processes or (os.cpu_count() or 1), C))
+    if pool is not None:
+        n_chunks = min(C, P * 8)
+        bounds = np.linspace(0, C, n_chunks + 1).astype(np.int64)
+        jobs = [(parent, cond_bit, cond_val, latency_us, arrival_us, branch_bits,
+                 configs[bounds[i]:bounds[i + 1]], slo_us) for i in range(n_chunks)]
+        parts = pool.map(_worker, jobs, chunksize=1)
+        return (np.concatenate([p[0] for p in parts]), np.concatenate([p[1] for p in parts]))
     if P == 1:
         return estimate_many(parent, cond_bit, cond_val, latency_us, arrival_us, branch_bits,
                              configs, slo_us)
