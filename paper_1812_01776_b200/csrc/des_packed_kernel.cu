@@ -321,6 +321,8 @@ __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, c
             const uint64_t X = pos < 32 ? xa : xb;                  // in[head + lane]
             const uint64_t XK = X | qmask;                          // kNever stays kNever
             const uint64_t XKn = __shfl_down_sync(full, XK, 1);
+            // a start is never before the arrival, so arrivals that share a time stamp bound the run
+            if (__ffs(~__ballot_sync(full, X != kNeverKey && lane < 31 && XKn > XK)) - 1 < kMinRun) goto single_step;
             const uint64_t gk = key | qmask;
             uint64_t v = (lane < R && gk > XK) ? gk : XK;
             uint64_t mul = d1k;
@@ -407,7 +409,7 @@ __device__ __forceinline__ int run_stage(const WarpCtx &w, const int32_t *row, c
             penalty = min(penalty * 2, 64);
         }
         if (cooldown > 0) cooldown--;
-
+    single_step:
         // ------------------------------------------------------------------
         // Single step: one batch.  (m1, pb1, pq1) is the slot in lane 0.
         // ------------------------------------------------------------------
@@ -592,6 +594,8 @@ __device__ __forceinline__ int run_stage_narrow(const WarpCtx &w, const int32_t 
             const uint32_t X = pos < 32 ? xa : xb;
             const uint32_t Xn = __shfl_down_sync(full, X, 1);
             const bool valid = X < kNarrowLimit / 2;
+            // a start is never before the arrival, so arrivals that share a time stamp bound the run
+            if (__ffs(~__ballot_sync(full, valid && lane < 31 && Xn > X)) - 1 < kMinRun) goto single_step;
             uint32_t v = (lane < R && fin > X) ? fin : X;
             uint32_t mul = d1;
             for (int d = R; d < 32; d <<= 1, mul <<= 1) {
@@ -680,7 +684,7 @@ __device__ __forceinline__ int run_stage_narrow(const WarpCtx &w, const int32_t 
             penalty = min(penalty * 2, 64);
         }
         if (cooldown > 0) cooldown--;
-
+    single_step:
         // ---------------- single step ----------------
         const uint32_t m2 = __shfl_sync(full, fin, 1);
         const int pb2 = __shfl_sync(full, sl_b, 1), ps2 = __shfl_sync(full, sl_s, 1);
