@@ -39,6 +39,10 @@ WORKLOADS = {
     4: "config4: linear 10-stage pipeline, 1,000,000 arrivals ramping 150->250 qps, 262,144 candidates",
     5: "config5: 8-stage tree with three branch points, 100,000 gamma arrivals (500 qps, CV 2), 1,048,576 candidates",
 }
+# DRAM bytes (read + write) of des_packed_kernel per query-event, from the ncu capture summarised in
+# profiles/des_packed_kernel_config2.md (reduced case; traffic is proportional to the query-events).
+# Set to None whenever that kernel changes until the capture has been repeated.
+NCU_DRAM_BYTES_PER_QUERY_EVENT = 12.21
 METRIC = "candidate_configs_per_s"
 UNIT = "candidates/s"
 
@@ -331,7 +335,11 @@ def run_cuda(args):
         "feasible_fraction": feasible,
         "kernel_ms": {"simulate": sum(sim_ms) / K, "select": sum(sel_ms) / K},
         "roofline": {"bound": "alu", "achieved": alu_achieved / 1e12, "peak": alu_peak / 1e12,
-                     "unit": "Tinteger-op/s", "frac": alu_achieved / alu_peak, "traffic": None,
+                     "unit": "Tinteger-op/s", "frac": alu_achieved / alu_peak,
+                     "traffic": (NCU_DRAM_BYTES_PER_QUERY_EVENT * events_per_cand * n_cand
+                                 if NCU_DRAM_BYTES_PER_QUERY_EVENT and args.variant == 0 and args.workload == 2
+                                 else None),
+                     "traffic_unit": "DRAM bytes per launch (ncu capture of a reduced case, scaled by query-events)",
                      "kernel": "des_kernel" if args.variant == 1 else "des_packed_kernel",
                      "peak_source": "integer-issue probe of this run (warp-inst/s x 32 lanes)",
                      "issue_peak_warp_inst_per_s": issue_rate},
