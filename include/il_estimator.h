@@ -175,6 +175,19 @@ IL_API int il_estimate_device(il_estimator *est, const il_stage_config *d_config
                               int64_t slo_us, int64_t *d_out_p99_us, int64_t *d_out_miss);
 
 /*
+ * The Estimator's full answer for ONE configuration: the latency of every
+ * query of the trace (Section 4.2: it "returns accurate estimates of the
+ * latency for each query in the trace"; P99 and miss count are reductions of
+ * this vector).
+ *   d_config          DEVICE pointer, [S] il_stage_config (one candidate)
+ *   d_out_latency_us  DEVICE pointer, [n_queries]: latency of query i of the trace
+ * Runs one warp; meant for inspection and tests, not for throughput.  Errors
+ * as il_estimate_device.
+ */
+IL_API int il_estimate_latencies(il_estimator *est, const il_stage_config *d_config,
+                                 int64_t *d_out_latency_us);
+
+/*
  * Allocation-free variant of il_estimate_device (the paper has no counterpart;
  * this is a deployment convenience of this library).
  *

@@ -128,7 +128,7 @@ des_kernel(const __grid_constant__ DesParams p)
                         if (rt.a_exit) {
                             if (mine) {
                                 const int64_t l = tfin - p.arrival[q];
-                                slab[exits + rank] = l;
+                                slab[q] = l;   // trace order: the slab doubles as the per-query answer
                                 lat_or |= (uint64_t)l;
                             }
                             exits += __popc(ma);
@@ -143,7 +143,7 @@ des_kernel(const __grid_constant__ DesParams p)
                         if (rt.b_exit) {
                             if (mine) {
                                 const int64_t l = tfin - p.arrival[q];
-                                slab[exits + rank] = l;
+                                slab[q] = l;   // trace order: the slab doubles as the per-query answer
                                 lat_or |= (uint64_t)l;
                             }
                             exits += __popc(mb_);

@@ -244,6 +244,35 @@ void il::bound_view(const il_estimator *e, BoundView *out)
     out->stream = e->stream;
 }
 
+// The scratch buffer a call may use: the caller's (il_set_workspace) or the
+// library's own, (re)allocated here if it is too small for n_cand candidates.
+static int acquire_workspace(il_estimator *e, int64_t n_cand, char **ws_out, size_t *bytes_out)
+{
+    char *ws = static_cast<char *>(e->user_ws);
+    size_t ws_bytes = e->user_ws_bytes;
+    if (!ws) {
+        const size_t want = recommended_bytes(e, n_cand);
+        if (e->own_ws_bytes < want) {
+            size_t free_b = 0, total_b = 0;
+            IL_CUDA(cudaMemGetInfo(&free_b, &total_b));
+            const size_t grant = std::min(want, (size_t)((free_b + e->own_ws_bytes) * 0.8));
+            if (grant > e->own_ws_bytes) {
+                IL_CUDA(cudaStreamSynchronize(e->stream));
+                if (e->own_ws) { cudaFree(e->own_ws); e->own_ws = nullptr; e->own_ws_bytes = 0; }
+                if (grant < min_bytes(e)) return IL_ERR_NOMEM;
+                cudaError_t ce = cudaMalloc(&e->own_ws, grant);
+                if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; e->own_ws = nullptr; return IL_ERR_NOMEM; }
+                e->own_ws_bytes = grant;
+            }
+        }
+        ws = static_cast<char *>(e->own_ws);
+        ws_bytes = e->own_ws_bytes;
+    }
+    *ws_out = ws;
+    *bytes_out = ws_bytes;
+    return IL_OK;
+}
+
 extern "C" {
 
 const char *il_strerror(int code)
@@ -461,27 +490,10 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
     if (!d_configs || !d_out_p99 || !d_out_miss) return IL_ERR_INVALID_ARG;
     IL_CUDA(cudaSetDevice(e->device));
 
-    // workspace
-    char *ws = static_cast<char *>(e->user_ws);
-    size_t ws_bytes = e->user_ws_bytes;
-    if (!ws) {
-        const size_t want = recommended_bytes(e, n_cand);
-        if (e->own_ws_bytes < want) {
-            size_t free_b = 0, total_b = 0;
-            IL_CUDA(cudaMemGetInfo(&free_b, &total_b));
-            const size_t grant = std::min(want, (size_t)((free_b + e->own_ws_bytes) * 0.8));
-            if (grant > e->own_ws_bytes) {
-                IL_CUDA(cudaStreamSynchronize(e->stream));
-                if (e->own_ws) { cudaFree(e->own_ws); e->own_ws = nullptr; e->own_ws_bytes = 0; }
-                if (grant < min_bytes(e)) return IL_ERR_NOMEM;
-                cudaError_t ce = cudaMalloc(&e->own_ws, grant);
-                if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; e->own_ws = nullptr; return IL_ERR_NOMEM; }
-                e->own_ws_bytes = grant;
-            }
-        }
-        ws = static_cast<char *>(e->own_ws);
-        ws_bytes = e->own_ws_bytes;
-    }
+    char *ws = nullptr;
+    size_t ws_bytes = 0;
+    int wrc = acquire_workspace(e, n_cand, &ws, &ws_bytes);
+    if (wrc) return wrc;
     Plan pl;
     if (!make_plan(e, ws_bytes, n_cand, pl)) return IL_ERR_NOMEM;
 
@@ -552,6 +564,41 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
     e->stats.algorithmic_ops = (int64_t)e->h_counters[2];
     e->stats.chunks = n_chunks;
     e->stats.kernel_launches = launches;
+    return *e->h_status;
+}
+
+int il_estimate_latencies(il_estimator *e, const il_stage_config *d_config, int64_t *d_out_latency)
+{
+    if (!e || !d_config || !d_out_latency) return IL_ERR_INVALID_ARG;
+    IL_CUDA(cudaSetDevice(e->device));
+    char *ws = nullptr;
+    size_t ws_bytes = 0;
+    int rc = acquire_workspace(e, 1, &ws, &ws_bytes);
+    if (rc) return rc;
+    Plan pl;
+    if (!make_plan(e, ws_bytes, 1, pl)) return IL_ERR_NOMEM;
+    cudaStream_t st = e->stream;
+    IL_CUDA(cudaMemsetAsync(e->d_counters, 0, 4 * sizeof(unsigned long long), st));
+    IL_CUDA(cudaMemsetAsync(e->d_status, 0, sizeof(int), st));
+    DesParams p = e->base;
+    p.configs = d_config;
+    p.n_cand = 1;
+    p.slot_elems = e->slot_elems;
+    p.ws_time = reinterpret_cast<int64_t *>(ws + pl.off_time);
+    p.ws_qid = reinterpret_cast<int32_t *>(ws + pl.off_qid);
+    p.slab = reinterpret_cast<int64_t *>(ws + pl.off_slab);
+    p.slab_stride = e->n_pad;
+    p.lat_or = reinterpret_cast<uint64_t *>(ws + pl.off_or);
+    p.order = reinterpret_cast<int32_t *>(ws + pl.off_order);
+    IL_CUDA(cudaMemsetAsync(ws + pl.off_order, 0, sizeof(int32_t), st));   // the one candidate is number 0
+    const int kernel = sim_kernel(e);
+    IL_CUDA(launch_simulation(p, kernel, 1, e->smem, st));
+    if (kernel == kSimWide)   // the wide kernel writes latencies in trace order
+        IL_CUDA(cudaMemcpyAsync(d_out_latency, p.slab, (size_t)e->n * 8, cudaMemcpyDeviceToDevice, st));
+    else
+        IL_CUDA(launch_scatter_latency(p.slab, e->d_arrival, (int)e->n, p.qbits, d_out_latency, st));
+    IL_CUDA(cudaMemcpyAsync(e->h_status, e->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+    IL_CUDA(cudaStreamSynchronize(st));
     return *e->h_status;
 }
 

@@ -80,6 +80,8 @@ inline cudaError_t launch_simulation(const DesParams &p, int kernel, int grid, s
     return launch_des_packed(p, kernel == kSimPackedStaged, grid, smem, stream);
 }
 cudaError_t launch_select(const SelectParams &p, cudaStream_t stream);
+cudaError_t launch_scatter_latency(const int64_t *slab_row, const int64_t *arrival, int n, int qbits,
+                                   int64_t *out, cudaStream_t stream);
 
 // Fills order[0..n_cand) with the chunk's candidate indices, costliest first
 // (longest-processing-time-first scheduling over the warps).

@@ -103,6 +103,30 @@ select_kernel(const __grid_constant__ SelectParams p)
     }
 }
 
+// Per-query answer of one candidate: the slab row holds one (finish, query)
+// record per query, in the order the queries left the pipeline; the latency of
+// query q goes to out[q].
+__global__ void __launch_bounds__(256)
+scatter_latency_kernel(const uint64_t *__restrict__ slab_row, const int64_t *__restrict__ arrival,
+                       int n, int qbits, int64_t *__restrict__ out)
+{
+    const uint64_t qmask = (1ull << qbits) - 1ull;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        const uint64_t rec = slab_row[i];
+        const uint64_t q = rec & qmask;
+        out[q] = (int64_t)(rec >> qbits) - arrival[q];
+    }
+}
+
+cudaError_t launch_scatter_latency(const int64_t *slab_row, const int64_t *arrival, int n, int qbits,
+                                   int64_t *out, cudaStream_t stream)
+{
+    const int grid = (n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184;
+    scatter_latency_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const uint64_t *>(slab_row), arrival, n,
+                                                     qbits, out);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_select(const SelectParams &p, cudaStream_t stream)
 {
     const int grid = (int)(p.n_cand < 65535 * 16 ? p.n_cand : 65535 * 16);

@@ -28,7 +28,7 @@ IL_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 EXPORTS = ["il_estimator_create", "il_estimator_destroy", "il_estimate", "il_estimate_device",
            "il_set_stream", "il_workspace_bytes", "il_workspace_min_bytes", "il_set_workspace",
            "il_get_stats", "il_stage_visits", "il_strerror", "il_last_cuda_error",
-           "il_measure_int_issue", "il_estimate_device_static", "il_set_variant"]
+           "il_measure_int_issue", "il_estimate_device_static", "il_set_variant", "il_estimate_latencies"]
 
 
 class ILError(RuntimeError):
@@ -94,6 +94,8 @@ def load_library():
     lib.il_estimate_device.argtypes = [vp, vp, i64, i64, vp, vp]
     lib.il_estimate_device_static.restype = ctypes.c_int
     lib.il_estimate_device_static.argtypes = [vp, vp, i64, i64, vp, vp]
+    lib.il_estimate_latencies.restype = ctypes.c_int
+    lib.il_estimate_latencies.argtypes = [vp, vp, vp]
     lib.il_set_variant.restype = ctypes.c_int
     lib.il_set_variant.argtypes = [vp, ctypes.c_int]
     lib.il_set_stream.restype = ctypes.c_int
@@ -190,6 +192,11 @@ def il_estimate_device_static(handle, d_configs: int, n: int, slo_us: int, d_out
     _check(load_library().il_estimate_device_static(handle, d_configs, int(n), int(slo_us),
                                                     d_out_p99, d_out_miss),
            "il_estimate_device_static")
+
+
+def il_estimate_latencies(handle, d_config: int, d_out_latency: int) -> None:
+    """il_estimate_latencies: one candidate (device pointer) in, per-query latencies written in place."""
+    _check(load_library().il_estimate_latencies(handle, d_config, d_out_latency), "il_estimate_latencies")
 
 
 def il_set_variant(handle, variant: int) -> None:
@@ -319,6 +326,14 @@ class Estimator:
         il_estimate_device(self._h, d_configs.data_ptr(), n, slo_us, out_p99.data_ptr(),
                            out_miss.data_ptr())
         return out_p99, out_miss
+
+    def latencies(self, config: np.ndarray):
+        """Per-query latencies (int64 numpy array, trace order) of one candidate [S][4]."""
+        torch = self._torch
+        cfg = torch.from_numpy(np.ascontiguousarray(config, dtype=np.uint8).reshape(self.n_stages, 4)).to(self.device)
+        out = torch.empty(self.n_queries, dtype=torch.int64, device=self.device)
+        il_estimate_latencies(self._h, cfg.data_ptr(), out.data_ptr())
+        return out.cpu().numpy()
 
     def stats(self) -> dict:
         return il_get_stats(self._h)

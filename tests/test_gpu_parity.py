@@ -74,6 +74,33 @@ def test_random_small(il, oracle, seed, variant):
     check(il, oracle, w, host=(seed % 2 == 0), variant=variant)
 
 
+@pytest.mark.parametrize("variant", [0, 1, 2], ids=["packed", "wide", "staged"])
+@pytest.mark.parametrize("seed", [1, 4, 7, 10])
+def test_per_query_latencies(il, oracle, seed, variant):
+    """The full answer of the Estimator, query by query, against the oracle."""
+    w = workloads.random_small(seed, S=2 + seed % 5, H=3, Bmax=[4, 33, 64][seed % 3], n=900 + 31 * seed,
+                               C=6, max_replicas=[3, 8, 32][seed % 3], tree=(seed % 2 == 1),
+                               qps=400.0, cv=3.0, lat_lo=1, lat_hi=20000,
+                               equal_stamp_every=(3 if seed % 4 == 0 else 0))
+    with il.Estimator.from_workload(w) as est:
+        est.set_variant(variant)
+        for c in range(w.n_candidates):
+            got = est.latencies(w.configs[c])
+            _, _, exp = oracle.estimate_one(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us,
+                                            w.branch_bits, w.configs[c], w.slo_us, want_latency=True)
+            assert np.array_equal(got, exp), (seed, c, np.nonzero(got != exp)[0][:5])
+
+
+def test_per_query_latencies_workloads(il, oracle):
+    for cid, n in [(2, 20000), (3, 20000), (5, 20000)]:
+        w = workloads.make(cid, n_queries=n, n_candidates=4)
+        with il.Estimator.from_workload(w) as est:
+            for c in range(4):
+                _, _, exp = oracle.estimate_one(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us,
+                                                w.branch_bits, w.configs[c], w.slo_us, want_latency=True)
+                assert np.array_equal(est.latencies(w.configs[c]), exp), (cid, c)
+
+
 def test_config1_full(il, oracle):
     st = check(il, oracle, workloads.make(1))
     assert st["batches"] > 0 and st["kernel_launches"] == 3 * st["chunks"]
