@@ -39,8 +39,8 @@ WORKLOADS = {
     4: "config4: linear 10-stage pipeline, 1,000,000 arrivals ramping 150->250 qps, 262,144 candidates",
     5: "config5: 8-stage tree with three branch points, 100,000 gamma arrivals (500 qps, CV 2), 1,048,576 candidates",
 }
-# DRAM bytes (read + write) of des_packed_kernel per query-event, from the ncu capture summarised in
-# profiles/des_packed_kernel_config2.md (reduced case; traffic is proportional to the query-events).
+# DRAM bytes (read + write) of des_packed_kernel per query-event, from an ncu capture of a reduced case
+# (1,024 candidates x 20,000 queries; traffic is proportional to the query-events processed).
 # Set to None whenever that kernel changes until the capture has been repeated.
 NCU_DRAM_BYTES_PER_QUERY_EVENT = 12.21
 METRIC = "candidate_configs_per_s"
