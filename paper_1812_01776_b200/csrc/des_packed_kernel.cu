@@ -578,14 +578,12 @@ __device__ __forceinline__ int run_stage_narrow(const WarpCtx &w, const int32_t 
 
     while (head < n_in) {
         // the head arrival must be in range to be dispatched here
-        {
-            const uint32_t ah = __shfl_sync(full, At, off);
-            if (ah >= kNarrowLimit / 2 || m1 >= kNarrowLimit / 2) {
-                if (ah == kNever32) break;      // cannot happen while head < n_in
-                if (!re_epoch()) { bail = true; break; }
-                const uint32_t ah2 = __shfl_sync(full, At, off);
-                if (ah2 >= kNarrowLimit / 2 || __shfl_sync(full, fin, 0) >= kNarrowLimit / 2) { bail = true; break; }
-            }
+        uint32_t ah = __shfl_sync(full, At, off);
+        if (ah >= kNarrowLimit / 2 || m1 >= kNarrowLimit / 2) {
+            if (ah == kNever32) break;      // cannot happen while head < n_in
+            if (!re_epoch()) { bail = true; break; }
+            ah = __shfl_sync(full, At, off);
+            if (ah >= kNarrowLimit / 2 || __shfl_sync(full, fin, 0) >= kNarrowLimit / 2) { bail = true; break; }
         }
         // ---------------- run step (see run_stage) ----------------
         if (cooldown == 0) {
@@ -595,7 +593,7 @@ __device__ __forceinline__ int run_stage_narrow(const WarpCtx &w, const int32_t 
             const uint32_t Xn = __shfl_down_sync(full, X, 1);
             const bool valid = X < kNarrowLimit / 2;
             // a start is never before the arrival, so arrivals that share a time stamp bound the run
-            if (__ffs(~__ballot_sync(full, valid && lane < 31 && Xn > X)) - 1 < kMinRun) goto single_step;
+            if (__ffs(~__ballot_sync(full, valid && lane < 31 && Xn > X)) - 1 < kMinRun) { cooldown = 1; goto single_step; }
             uint32_t v = (lane < R && fin > X) ? fin : X;
             uint32_t mul = d1;
             for (int d = R; d < 32; d <<= 1, mul <<= 1) {
@@ -689,7 +687,7 @@ __device__ __forceinline__ int run_stage_narrow(const WarpCtx &w, const int32_t 
         const uint32_t m2 = __shfl_sync(full, fin, 1);
         const int pb2 = __shfl_sync(full, sl_b, 1), ps2 = __shfl_sync(full, sl_s, 1);
         const uint32_t pq2 = __shfl_sync(full, sl_q, 1);
-        const uint32_t a_head = __shfl_sync(full, At, off);
+        const uint32_t a_head = ah;
         const uint32_t qh = __shfl_sync(full, Aq, off);
         const uint32_t t = max(m1, a_head);
         const unsigned mA = __ballot_sync(full, At <= t);
