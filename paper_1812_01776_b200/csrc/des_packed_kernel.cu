@@ -41,7 +41,7 @@ namespace il {
 namespace {
 
 constexpr uint64_t kNeverKey = ~0ull;
-constexpr int kMinRun = 2;          // shortest run of single dispatches worth committing at once
+constexpr int kMinRun = 3;          // shortest run of single dispatches worth committing at once (measured: 3-4 best)
 
 enum RouteKind { kForward = 0, kBranch = 1 };
 
