@@ -42,7 +42,7 @@ WORKLOADS = {
 # DRAM bytes (read + write) of des_packed_kernel per query-event, from an ncu capture of a reduced case
 # (1,024 candidates x 20,000 queries; traffic is proportional to the query-events processed).
 # Set to None whenever that kernel changes until the capture has been repeated.
-NCU_DRAM_BYTES_PER_QUERY_EVENT = 12.21
+NCU_DRAM_BYTES_PER_QUERY_EVENT = 12.24
 METRIC = "candidate_configs_per_s"
 UNIT = "candidates/s"
 
