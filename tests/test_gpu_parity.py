@@ -101,6 +101,33 @@ def test_per_query_latencies_workloads(il, oracle):
                 assert np.array_equal(est.latencies(w.configs[c]), exp), (cid, c)
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_times_scaled_beyond_the_32_bit_loop(il, oracle, seed):
+    """Latencies of 2^24 us and more take the 64-bit stage loop of the packed
+    kernel (its run step, late-slot merge and single step included)."""
+    w = workloads.random_small(200 + seed, S=2 + seed % 4, H=2, Bmax=[4, 33, 64][seed % 3], n=900, C=30,
+                               max_replicas=[3, 8, 32][seed % 3], tree=(seed % 2 == 1), qps=400.0, cv=3.0,
+                               lat_lo=4100, lat_hi=20000, equal_stamp_every=(3 if seed % 3 == 0 else 0))
+    w.latency_us = w.latency_us * 4096            # 1.7e7 .. 8.2e7 us: above the 32-bit loop's limit
+    w.arrival_us = w.arrival_us * 4096
+    w.slo_us = w.slo_us * 4096
+    assert w.latency_us.min() >= 1 << 24
+    check(il, oracle, w)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_sparse_traces_move_the_epoch(il, oracle, seed):
+    """Gaps between arrivals far beyond 2^30 us (and, for odd seeds, services
+    long enough that batches stay in flight across them) exercise the 32-bit
+    loop's epoch moves and its hand-over to the 64-bit loop."""
+    w = workloads.random_small(300 + seed, S=2 + seed % 3, H=2, Bmax=8, n=600, C=24, max_replicas=4,
+                               tree=(seed % 2 == 0), qps=[0.0004, 0.002, 0.01][seed % 3], cv=4.0,
+                               lat_lo=1000, lat_hi=(1 << 24) - 1 if seed % 2 else 50000,
+                               equal_stamp_every=(2 if seed == 4 else 0))
+    assert np.diff(w.arrival_us).max() > (1 << 30)
+    check(il, oracle, w)
+
+
 def test_config1_full(il, oracle):
     st = check(il, oracle, workloads.make(1))
     assert st["batches"] > 0 and st["kernel_launches"] == 3 * st["chunks"]
