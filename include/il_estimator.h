@@ -188,6 +188,20 @@ IL_API int il_estimate_latencies(il_estimator *est, const il_stage_config *d_con
                                  int64_t *d_out_latency_us);
 
 /*
+ * Traffic envelope of the bound trace (Section 5: the Planner builds it for the
+ * sample trace and hands it to the Tuner): for each window length
+ * window_us[i] >= 1, the largest number of arrivals in any half-open window
+ * [t, t + window_us[i]) on the trace; the maximum arrival rate at that time
+ * scale is out_max_count[i] / window_us[i].  The paper takes the lengths from
+ * the pipeline's service time, doubling up to 60 s; the caller chooses them.
+ *   window_us       HOST pointer, [n_windows], n_windows <= 64
+ *   out_max_count   HOST pointer, [n_windows]
+ * Errors: INVALID_ARG, CUDA.
+ */
+IL_API int il_traffic_envelope(il_estimator *est, const int64_t *window_us, int32_t n_windows,
+                               int64_t *out_max_count);
+
+/*
  * Allocation-free variant of il_estimate_device (the paper has no counterpart;
  * this is a deployment convenience of this library).
  *

@@ -65,6 +65,8 @@ def _load():
         lib.orc_estimate_many.restype = ctypes.c_int
         lib.orc_estimate_many.argtypes = [ctypes.c_int32] * 3 + [p] * 4 + [ctypes.c_int64, p, p,
                                           p, ctypes.c_int64, ctypes.c_int64, p, p]
+        lib.orc_traffic_envelope.restype = ctypes.c_int
+        lib.orc_traffic_envelope.argtypes = [ctypes.c_int64, p, ctypes.c_int32, p, p]
         lib.orc_p99_miss.restype = ctypes.c_int
         lib.orc_p99_miss.argtypes = [p, ctypes.c_int64, ctypes.c_int64, p, p]
         _lib = lib
@@ -207,3 +209,17 @@ def p99_miss(latency, slo_us: int) -> Tuple[int, int]:
     if rc:
         raise OracleError(rc)
     return int(p99.value), int(miss.value)
+
+
+def traffic_envelope(arrival_us, window_us) -> np.ndarray:
+    """Largest number of arrivals in any half-open window of each given length
+    (Section 5 of the paper: the traffic envelope the Planner hands to the Tuner)."""
+    lib = _load()
+    arrival_us = np.ascontiguousarray(arrival_us, dtype=np.int64)
+    window_us = np.ascontiguousarray(window_us, dtype=np.int64)
+    out = np.zeros(window_us.shape[0], dtype=np.int64)
+    rc = lib.orc_traffic_envelope(arrival_us.shape[0], _ptr(arrival_us), window_us.shape[0],
+                                  _ptr(window_us), _ptr(out))
+    if rc:
+        raise OracleError(rc)
+    return out

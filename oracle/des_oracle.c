@@ -323,3 +323,31 @@ int orc_p99_miss(const int64_t *latency, int64_t n, int64_t slo_us,
     free(tmp);
     return ORC_OK;
 }
+
+/*
+ * Traffic envelope of the trace (Section 5, "High-Frequency Tuning"): for a
+ * window of length window_us[i], the largest number of arrivals that fall into
+ * any window of that length anywhere on the trace.  A window that maximises
+ * the count can be moved right until it starts at an arrival, so it is enough
+ * to look at the half-open windows [a_j, a_j + window_us[i]) for every arrival
+ * j.  Plain two-pointer sweep per window length.
+ */
+int orc_traffic_envelope(int64_t n, const int64_t *arrival_us, int32_t n_windows,
+                         const int64_t *window_us, int64_t *out_max_count)
+{
+    if (n < 1 || !arrival_us || n_windows < 0 || (n_windows > 0 && (!window_us || !out_max_count)))
+        return ORC_ERR_ARG;
+    for (int64_t i = 1; i < n; i++)
+        if (arrival_us[i] < arrival_us[i - 1]) return ORC_ERR_TRACE;
+    for (int32_t w = 0; w < n_windows; w++) {
+        if (window_us[w] < 1) return ORC_ERR_ARG;
+        int64_t best = 0, hi = 0;
+        for (int64_t j = 0; j < n; j++) {
+            if (hi < j) hi = j;
+            while (hi < n && arrival_us[hi] - arrival_us[j] < window_us[w]) hi++;
+            if (hi - j > best) best = hi - j;
+        }
+        out_max_count[w] = best;
+    }
+    return ORC_OK;
+}

@@ -602,6 +602,29 @@ int il_estimate_latencies(il_estimator *e, const il_stage_config *d_config, int6
     return *e->h_status;
 }
 
+int il_traffic_envelope(il_estimator *e, const int64_t *window_us, int32_t n_windows, int64_t *out_max_count)
+{
+    if (!e || n_windows < 0 || n_windows > envelope_max_windows()) return IL_ERR_INVALID_ARG;
+    if (n_windows == 0) return IL_OK;
+    if (!window_us || !out_max_count) return IL_ERR_INVALID_ARG;
+    for (int w = 0; w < n_windows; w++) if (window_us[w] < 1) return IL_ERR_INVALID_ARG;
+    IL_CUDA(cudaSetDevice(e->device));
+    // the counts fit the 4-word counter block that every estimate call clears before use
+    static_assert(sizeof(unsigned long long) * 4 >= sizeof(int) * 8, "counter block too small");
+    int host_out[64];
+    cudaStream_t st = e->stream;
+    for (int w0 = 0; w0 < n_windows; w0 += 8) {
+        const int cnt = std::min(8, n_windows - w0);
+        IL_CUDA(cudaMemsetAsync(e->d_counters, 0, 4 * sizeof(unsigned long long), st));
+        IL_CUDA(launch_envelope(e->d_arrival, (int)e->n, window_us + w0, cnt,
+                                reinterpret_cast<int *>(e->d_counters), e->num_sms, st));
+        IL_CUDA(cudaMemcpyAsync(host_out + w0, e->d_counters, cnt * sizeof(int), cudaMemcpyDeviceToHost, st));
+    }
+    IL_CUDA(cudaStreamSynchronize(st));
+    for (int w = 0; w < n_windows; w++) out_max_count[w] = host_out[w];
+    return IL_OK;
+}
+
 int il_estimate(il_estimator *e, const il_stage_config *configs, int64_t n_cand, int64_t slo_us,
                 int64_t *out_p99, int64_t *out_miss)
 {

@@ -96,6 +96,9 @@ struct OrderParams {
 };
 cudaError_t launch_order(const OrderParams &p, cudaStream_t stream);
 int des_max_ctas_per_sm(size_t smem);
+cudaError_t launch_envelope(const int64_t *d_arrival, int n, const int64_t *h_windows, int n_windows,
+                            int *d_out, int num_sms, cudaStream_t stream);
+int envelope_max_windows();
 cudaError_t launch_int_issue(unsigned *sink, int grid, int iters, cudaStream_t stream);
 
 }  // namespace il

@@ -28,7 +28,7 @@ IL_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 EXPORTS = ["il_estimator_create", "il_estimator_destroy", "il_estimate", "il_estimate_device",
            "il_set_stream", "il_workspace_bytes", "il_workspace_min_bytes", "il_set_workspace",
            "il_get_stats", "il_stage_visits", "il_strerror", "il_last_cuda_error",
-           "il_measure_int_issue", "il_estimate_device_static", "il_set_variant", "il_estimate_latencies"]
+           "il_measure_int_issue", "il_estimate_device_static", "il_set_variant", "il_estimate_latencies", "il_traffic_envelope"]
 
 
 class ILError(RuntimeError):
@@ -96,6 +96,8 @@ def load_library():
     lib.il_estimate_device_static.argtypes = [vp, vp, i64, i64, vp, vp]
     lib.il_estimate_latencies.restype = ctypes.c_int
     lib.il_estimate_latencies.argtypes = [vp, vp, vp]
+    lib.il_traffic_envelope.restype = ctypes.c_int
+    lib.il_traffic_envelope.argtypes = [vp, vp, ctypes.c_int32, vp]
     lib.il_set_variant.restype = ctypes.c_int
     lib.il_set_variant.argtypes = [vp, ctypes.c_int]
     lib.il_set_stream.restype = ctypes.c_int
@@ -197,6 +199,15 @@ def il_estimate_device_static(handle, d_configs: int, n: int, slo_us: int, d_out
 def il_estimate_latencies(handle, d_config: int, d_out_latency: int) -> None:
     """il_estimate_latencies: one candidate (device pointer) in, per-query latencies written in place."""
     _check(load_library().il_estimate_latencies(handle, d_config, d_out_latency), "il_estimate_latencies")
+
+
+def il_traffic_envelope(handle, window_us) -> np.ndarray:
+    """il_traffic_envelope: host window lengths in, host maximum counts out."""
+    window_us = np.ascontiguousarray(window_us, dtype=np.int64)
+    out = np.zeros(window_us.shape[0], dtype=np.int64)
+    _check(load_library().il_traffic_envelope(handle, window_us.ctypes.data, window_us.shape[0],
+                                              out.ctypes.data), "il_traffic_envelope")
+    return out
 
 
 def il_set_variant(handle, variant: int) -> None:
@@ -334,6 +345,10 @@ class Estimator:
         out = torch.empty(self.n_queries, dtype=torch.int64, device=self.device)
         il_estimate_latencies(self._h, cfg.data_ptr(), out.data_ptr())
         return out.cpu().numpy()
+
+    def traffic_envelope(self, window_us) -> np.ndarray:
+        """Largest number of arrivals in any window of each given length (microseconds)."""
+        return il_traffic_envelope(self._h, window_us)
 
     def stats(self) -> dict:
         return il_get_stats(self._h)

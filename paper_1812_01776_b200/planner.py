@@ -230,3 +230,31 @@ class Planner:
             if down is not None:
                 out.append(down)
         return out
+
+
+def envelope_windows(service_time_us: int, longest_us: int = 60_000_000) -> np.ndarray:
+    """Window lengths of the traffic envelope as Section 5 discretises them: the
+    smallest is the pipeline's service time, then doubling up to 60 seconds."""
+    out, w = [], max(1, int(service_time_us))
+    while w < longest_us:
+        out.append(w)
+        w *= 2
+    return np.array(out + [longest_us], dtype=np.int64)
+
+
+def tuner_handoff(planner: Planner, cfg: np.ndarray, n_queries: int, span_us: int,
+                  envelope_fn: Callable[[np.ndarray], np.ndarray]) -> dict:
+    """What the Planner gives the Tuner (Section 5, "Initialization"): the
+    traffic envelope of the sample trace, and per model the single-replica
+    throughput mu_m and the max-provisioning ratio rho_m = lambda_m / (replicas
+    x mu_m), lambda_m being the trace's mean arrival rate times the model's
+    scale factor.  envelope_fn is Estimator.traffic_envelope (or the oracle's)."""
+    windows = envelope_windows(planner.service_time(cfg))
+    counts = np.asarray(envelope_fn(windows), dtype=np.int64)
+    lam = n_queries / float(span_us)                       # queries per microsecond
+    b = cfg[:, 1].astype(np.int64)
+    lat = planner.lat[np.arange(planner.S), cfg[:, 0], b - 1].astype(np.float64)
+    mu = b / lat                                           # one replica, queries per microsecond
+    rho = lam * planner.scale / (cfg[:, 2].astype(np.float64) * mu)
+    return {"window_us": windows, "max_count": counts, "rate_per_us": counts / windows.astype(np.float64),
+            "mu_per_us": mu, "rho": rho, "scale_factor": planner.scale.copy()}

@@ -80,6 +80,21 @@ def test_planner_finds_a_plan_whenever_one_exists(oracle):
             assert res.p99_us <= slo
 
 
+def test_tuner_handoff_with_the_oracle(oracle):
+    from paper_1812_01776_b200.planner import tuner_handoff, envelope_windows
+    w, prices = small_workload()
+    slo = 60_000
+    pl = Planner(w.parent, w.latency_us, w.visits_per_stage(), prices, slo, oracle_fn(oracle, w, slo))
+    res = pl.minimize_cost()
+    span = int(w.arrival_us[-1] - w.arrival_us[0])
+    h = tuner_handoff(pl, res.config, w.n_queries, span, lambda wins: oracle.traffic_envelope(w.arrival_us, wins))
+    assert h["window_us"][0] == pl.service_time(res.config) and h["window_us"][-1] == 60_000_000
+    assert np.all(np.diff(h["window_us"]) > 0) and np.all(np.diff(h["max_count"]) >= 0)
+    assert h["max_count"][-1] == w.n_queries            # the 10 s trace fits in the 60 s window
+    assert np.all(h["rho"] > 0) and np.all(h["rho"] < 1)   # a feasible plan keeps every model below saturation
+    assert np.array_equal(envelope_windows(1000)[:3], [1000, 2000, 4000])
+
+
 @pytest.mark.gpu
 def test_planner_same_plan_on_gpu_and_oracle(oracle):
     import torch
