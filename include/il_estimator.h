@@ -283,6 +283,7 @@ IL_API int il_set_workspace(il_estimator *est, void *d_workspace, size_t bytes);
 #define IL_VARIANT_AUTO 0
 #define IL_VARIANT_WIDE 1
 #define IL_VARIANT_STAGED 2
+#define IL_VARIANT_LANES 3
 IL_API int il_set_variant(il_estimator *est, int variant);
 
 /* Counters of the last estimate call on this handle. */

@@ -8,7 +8,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libil_estimator.so")
-SOURCES = ["des_kernel.cu", "des_packed_kernel.cu", "select_kernel.cu", "order_kernel.cu", "envelope_kernel.cu", "il_api.cu", "il_static.cu"]
+SOURCES = ["des_kernel.cu", "des_packed_kernel.cu", "des_lane_kernel.cu", "select_kernel.cu", "order_kernel.cu", "envelope_kernel.cu", "il_api.cu", "il_static.cu"]
 HEADERS = [os.path.join(CSRC, "il_internal.h"), os.path.join(ROOT, "include", "il_estimator.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]

@@ -40,8 +40,12 @@ struct il_estimator {
     int64_t *d_arrival = nullptr;
     uint64_t *d_ptrace = nullptr;      // packed root stream
     bool can_pack = false;             // every reachable time fits a packed record
+    bool lane_ok = false;              // the lane kernel applies (packed records, stream offsets fit 31 bits)
     int variant = IL_VARIANT_AUTO;
-    int ctas_per_sm_wide = 0, ctas_per_sm_packed = 0, ctas_per_sm_staged = 0;
+    int ctas_per_sm_wide = 0, ctas_per_sm_packed = 0, ctas_per_sm_staged = 0, ctas_per_sm_lane = 0;
+    int64_t lane_elems = 0;            // lane kernel: stream records per candidate
+    int cpw = 1;                       // lane kernel: candidates per warp
+    size_t smem_lane = 0;
     uint8_t *d_bits = nullptr;
     int32_t *d_lat = nullptr;
     unsigned long long *d_counters = nullptr;   // [4]
@@ -77,25 +81,58 @@ struct Plan {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-size_t slot_bytes(const il_estimator *e) { return (size_t)e->slot_elems * 12; }
+bool use_packed(const il_estimator *e)
+{
+    return e->can_pack && e->variant != IL_VARIANT_WIDE;
+}
+
+int sim_kernel(const il_estimator *e)
+{
+    if (!use_packed(e)) return kSimWide;
+    if (e->variant == IL_VARIANT_LANES && e->lane_ok) return kSimLane;
+    return e->variant == IL_VARIANT_STAGED ? kSimPackedStaged : kSimPacked;
+}
+
+int ctas_for(const il_estimator *e)
+{
+    const int k = sim_kernel(e);
+    return k == kSimWide ? e->ctas_per_sm_wide
+         : k == kSimPacked ? e->ctas_per_sm_packed
+         : k == kSimLane ? e->ctas_per_sm_lane : e->ctas_per_sm_staged;
+}
+
+// A warp slot is the stream memory one resident warp works in.  The
+// warp-per-candidate kernels serve one candidate at a time from it, the lane
+// kernel cpw candidates.
+bool is_lane(const il_estimator *e) { return sim_kernel(e) == kSimLane; }
+int warps_per_cta(const il_estimator *e) { return is_lane(e) ? des_lane_warps_per_cta() : kWarpsPerCta; }
+int64_t cands_per_slot(const il_estimator *e) { return is_lane(e) ? e->cpw : 1; }
+
+size_t slot_time_bytes(const il_estimator *e)
+{
+    return is_lane(e) ? (size_t)e->cpw * e->lane_elems * 8 : (size_t)e->slot_elems * 8;
+}
+size_t slot_qid_bytes(const il_estimator *e) { return is_lane(e) ? 0 : (size_t)e->slot_elems * 4; }
+size_t slot_bytes(const il_estimator *e) { return slot_time_bytes(e) + slot_qid_bytes(e); }
 size_t cand_bytes(const il_estimator *e) { return (size_t)e->n_pad * 8 + 12; }
 
 int64_t full_slots(const il_estimator *e)
 {
-    return (int64_t)e->num_sms * e->ctas_per_sm * kWarpsPerCta;
+    return (int64_t)e->num_sms * e->ctas_per_sm * warps_per_cta(e);
 }
 
 int64_t wanted_slots(const il_estimator *e, int64_t n_cand)
 {
-    const int64_t need = (n_cand + kWarpsPerCta - 1) / kWarpsPerCta * kWarpsPerCta;
-    return std::max<int64_t>(kWarpsPerCta, std::min(full_slots(e), need));
+    const int64_t w = warps_per_cta(e), cps = cands_per_slot(e);
+    const int64_t need = ((n_cand + cps - 1) / cps + w - 1) / w * w;
+    return std::max<int64_t>(w, std::min(full_slots(e), need));
 }
 
 size_t layout(const il_estimator *e, Plan &pl)
 {
     size_t off = 0;
-    pl.off_time = off; off = align_up(off + (size_t)pl.slots * e->slot_elems * 8, 256);
-    pl.off_qid = off;  off = align_up(off + (size_t)pl.slots * e->slot_elems * 4, 256);
+    pl.off_time = off; off = align_up(off + (size_t)pl.slots * slot_time_bytes(e), 256);
+    pl.off_qid = off;  off = align_up(off + (size_t)pl.slots * slot_qid_bytes(e), 256);
     pl.off_slab = off; off = align_up(off + (size_t)pl.chunk * e->n_pad * 8, 256);
     pl.off_or = off;   off = align_up(off + (size_t)pl.chunk * 8, 256);
     pl.off_order = off; off = align_up(off + (size_t)pl.chunk * 4, 256);
@@ -108,15 +145,16 @@ size_t recommended_bytes(const il_estimator *e, int64_t n_cand)
     Plan pl;
     n_cand = std::max<int64_t>(n_cand, 1);
     pl.slots = wanted_slots(e, n_cand);
-    pl.chunk = std::max<int64_t>(std::min<int64_t>(n_cand, 8 * full_slots(e)), 2 * pl.slots);
+    pl.chunk = std::max<int64_t>(std::min<int64_t>(n_cand, 8 * full_slots(e) * cands_per_slot(e)),
+                                 2 * pl.slots * cands_per_slot(e));
     return layout(e, pl) + 1024;
 }
 
 size_t min_bytes(const il_estimator *e)
 {
     Plan pl;
-    pl.slots = kWarpsPerCta;
-    pl.chunk = 2 * kWarpsPerCta;
+    pl.slots = warps_per_cta(e);
+    pl.chunk = 2 * warps_per_cta(e);
     return layout(e, pl) + 1024;
 }
 
@@ -126,9 +164,10 @@ bool make_plan(const il_estimator *e, size_t bytes, int64_t n_cand, Plan &pl)
     if (bytes < min_bytes(e)) return false;
     const size_t usable = bytes - 1024;
     const size_t sb = slot_bytes(e), cb = cand_bytes(e);
-    int64_t slots = std::min<int64_t>(wanted_slots(e, n_cand), (int64_t)(usable / (sb + 2 * cb)));
-    slots = slots / kWarpsPerCta * kWarpsPerCta;
-    if (slots < kWarpsPerCta) return false;
+    const int64_t w = warps_per_cta(e);
+    int64_t slots = std::min<int64_t>(wanted_slots(e, n_cand), (int64_t)(usable / (sb + 2 * cands_per_slot(e) * cb)));
+    slots = slots / w * w;
+    if (slots < w) return false;
     pl.slots = slots;
     pl.chunk = std::min<int64_t>(n_cand, (int64_t)((usable - (size_t)slots * sb) / cb));
     // alignment padding may push the layout over: shrink the chunk until it fits
@@ -193,24 +232,6 @@ int64_t plan_stream_buffers(const il_profiles *pr, const int64_t *visits, int32_
     return top;
 }
 
-bool use_packed(const il_estimator *e)
-{
-    return e->can_pack && e->variant != IL_VARIANT_WIDE;
-}
-
-int sim_kernel(const il_estimator *e)
-{
-    if (!use_packed(e)) return kSimWide;
-    return e->variant == IL_VARIANT_STAGED ? kSimPackedStaged : kSimPacked;
-}
-
-int ctas_for(const il_estimator *e)
-{
-    const int k = sim_kernel(e);
-    return k == kSimWide ? e->ctas_per_sm_wide
-         : k == kSimPacked ? e->ctas_per_sm_packed : e->ctas_per_sm_staged;
-}
-
 void free_device(il_estimator *e)
 {
     cudaFree(e->d_arrival); cudaFree(e->d_ptrace); cudaFree(e->d_bits); cudaFree(e->d_lat);
@@ -235,7 +256,7 @@ int ensure_events(il_estimator *e, size_t count)
 void il::bound_view(const il_estimator *e, BoundView *out)
 {
     out->base = e->base;
-    out->kernel = sim_kernel(e);
+    out->kernel = sim_kernel(e) == kSimLane ? (int)kSimPacked : sim_kernel(e);   // its user has no lane layout
     out->S = e->S;
     out->n = e->n; out->n_pad = e->n_pad; out->slot_elems = e->slot_elems;
     out->smem = e->smem;
@@ -370,6 +391,18 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     for (int s = 0; s < S; s++) e->events_per_candidate += e->visits[s];
     e->slot_elems = std::max<int64_t>(32, plan_stream_buffers(pr, e->visits, bp.buf_off));
     for (int s = 0; s < S; s++) bp.n_s[s] = (int32_t)e->visits[s];
+    // lane kernel: every stage but the root keeps its whole arrival stream, one after the other
+    e->cpw = 32 / S;
+    e->lane_elems = 0;
+    for (int s = 1; s < S; s++) {
+        bp.lane_off[s] = (int32_t)e->lane_elems;   // below 2^31: checked next
+        e->lane_elems += (e->visits[s] + 3) / 4 * 4;
+    }
+    bp.lane_off[0] = 0;
+    const bool lane_fits = e->lane_elems < (INT64_C(1) << 31);
+    e->lane_elems = std::max<int64_t>(e->lane_elems, 4);
+    bp.lane_elems = e->lane_elems;
+    bp.cpw = e->cpw;
     bp.S = S; bp.H = H; bp.Bmax = B; bp.n = (int32_t)n;
     e->smem = (size_t)S * H * B * sizeof(int32_t);
 
@@ -382,6 +415,7 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     IL_CUDA_E(cudaMalloc(&e->d_arrival, (size_t)n * 8));
     IL_CUDA_E(cudaMalloc(&e->d_bits, (size_t)n));
     e->can_pack = can_pack;
+    e->lane_ok = can_pack && lane_fits;
     bp.qbits = qbits;
     if (can_pack) {
         // padded with "never" records to whole tiles, so that bulk copies always move full tiles
@@ -409,7 +443,10 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     e->ctas_per_sm_wide = des_max_ctas_per_sm(e->smem);
     e->ctas_per_sm_packed = des_packed_max_ctas_per_sm(false, e->smem);
     e->ctas_per_sm_staged = des_packed_max_ctas_per_sm(true, e->smem);
-    if (e->ctas_per_sm_wide < 1 || e->ctas_per_sm_packed < 1 || e->ctas_per_sm_staged < 1)
+    e->smem_lane = des_lane_smem(S * H * B);
+    e->ctas_per_sm_lane = des_lane_max_ctas_per_sm(e->smem_lane);
+    if (e->ctas_per_sm_wide < 1 || e->ctas_per_sm_packed < 1 || e->ctas_per_sm_staged < 1 ||
+        e->ctas_per_sm_lane < 1)
         return fail(IL_ERR_CUDA);
     e->ctas_per_sm = ctas_for(e);
     *out = e;
@@ -436,7 +473,7 @@ int il_set_stream(il_estimator *e, void *cuda_stream)
 
 int il_set_variant(il_estimator *e, int variant)
 {
-    if (!e || variant < IL_VARIANT_AUTO || variant > IL_VARIANT_STAGED) return IL_ERR_INVALID_ARG;
+    if (!e || variant < IL_VARIANT_AUTO || variant > IL_VARIANT_LANES) return IL_ERR_INVALID_ARG;
     e->variant = variant;
     e->ctas_per_sm = ctas_for(e);
     return IL_OK;
@@ -527,12 +564,20 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
         op.span_us = e->span_us;
         op.order = reinterpret_cast<int32_t *>(ws + pl.off_order);
         if (ch > 0) IL_CUDA(cudaMemsetAsync(e->d_counters, 0, sizeof(unsigned long long), st));
-        IL_CUDA(launch_order(op, st));
-        int64_t ctas = std::min<int64_t>(pl.slots / kWarpsPerCta, (cnt + kWarpsPerCta - 1) / kWarpsPerCta);
-        if (2 * cnt <= 3 * full_slots(e))
-            ctas = std::min<int64_t>(ctas, (int64_t)e->num_sms * std::min(e->ctas_per_sm, kOneWaveCtasPerSm));
+        const bool lane = is_lane(e);
+        const int64_t wpc = warps_per_cta(e);
+        const int64_t groups = (cnt + cands_per_slot(e) - 1) / cands_per_slot(e);
+        int64_t ctas = std::min<int64_t>(pl.slots / wpc, (groups + wpc - 1) / wpc);
+        if (lane) {
+            p.lane_ws = reinterpret_cast<uint64_t *>(ws + pl.off_time);   // warps take candidates in index order
+        } else {
+            IL_CUDA(launch_order(op, st));
+            launches++;
+            if (2 * cnt <= 3 * full_slots(e))
+                ctas = std::min<int64_t>(ctas, (int64_t)e->num_sms * std::min(e->ctas_per_sm, kOneWaveCtasPerSm));
+        }
         IL_CUDA(cudaEventRecord(e->events[2 + 3 * ch], st));
-        IL_CUDA(launch_simulation(p, sim_kernel(e), (int)ctas, e->smem, st));
+        IL_CUDA(launch_simulation(p, sim_kernel(e), (int)ctas, lane ? e->smem_lane : e->smem, st));
         IL_CUDA(cudaEventRecord(e->events[3 + 3 * ch], st));
         SelectParams sp;
         sp.slab = p.slab; sp.slab_stride = e->n_pad; sp.lat_or = p.lat_or;
@@ -541,7 +586,7 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
         sp.out_p99 = d_out_p99 + lo; sp.out_miss = d_out_miss + lo;
         IL_CUDA(launch_select(sp, st));
         IL_CUDA(cudaEventRecord(e->events[4 + 3 * ch], st));
-        launches += 3;
+        launches += 2;
     }
     IL_CUDA(cudaEventRecord(e->events[1], st));
     IL_CUDA(cudaMemcpyAsync(e->h_counters, e->d_counters, 4 * sizeof(unsigned long long),
@@ -592,7 +637,8 @@ int il_estimate_latencies(il_estimator *e, const il_stage_config *d_config, int6
     p.order = reinterpret_cast<int32_t *>(ws + pl.off_order);
     IL_CUDA(cudaMemsetAsync(ws + pl.off_order, 0, sizeof(int32_t), st));   // the one candidate is number 0
     const int kernel = sim_kernel(e);
-    IL_CUDA(launch_simulation(p, kernel, 1, e->smem, st));
+    p.lane_ws = reinterpret_cast<uint64_t *>(ws + pl.off_time);
+    IL_CUDA(launch_simulation(p, kernel, 1, kernel == kSimLane ? e->smem_lane : e->smem, st));
     if (kernel == kSimWide)   // the wide kernel writes latencies in trace order
         IL_CUDA(cudaMemcpyAsync(d_out_latency, p.slab, (size_t)e->n * 8, cudaMemcpyDeviceToDevice, st));
     else

@@ -37,6 +37,11 @@ struct DesParams {
     uint64_t *lat_or;             // [n_cand] OR of all latencies of the candidate
     unsigned long long *counters; // [0] next candidate, [1] batches dispatched, [2] algorithmic ops
     int *status;                  // first error seen by any warp (0 = none)
+    // lane-parallel kernel only (des_lane_kernel.cu)
+    uint64_t *lane_ws;            // [warp slots][cpw][lane_elems] inter-stage streams of packed records
+    int64_t lane_elems;           // stream records per candidate: every stage's arrival stream but the root's
+    int32_t lane_off[IL_MAX_STAGES]; // record offset of stage s's arrival stream inside a candidate's block
+    int32_t cpw;                  // candidates per warp, floor(32 / S)
 };
 
 struct SelectParams {
@@ -72,10 +77,16 @@ cudaError_t launch_des(const DesParams &p, int grid, size_t smem, cudaStream_t s
 cudaError_t launch_des_packed(const DesParams &p, bool staged, int grid, size_t smem, cudaStream_t stream);
 int des_packed_max_ctas_per_sm(bool staged, size_t smem);
 int trace_tile_records();     // the packed trace is padded to a multiple of this many records
-enum SimKernel { kSimWide = 0, kSimPacked = 1, kSimPackedStaged = 2 };
+// lane-parallel kernel: one lane per (candidate, stage); smem from des_lane_smem
+cudaError_t launch_des_lane(const DesParams &p, int grid, size_t smem, cudaStream_t stream);
+int des_lane_warps_per_cta();
+size_t des_lane_smem(int n_tab);
+int des_lane_max_ctas_per_sm(size_t smem);
+enum SimKernel { kSimWide = 0, kSimPacked = 1, kSimPackedStaged = 2, kSimLane = 3 };
 inline cudaError_t launch_simulation(const DesParams &p, int kernel, int grid, size_t smem,
                                      cudaStream_t stream)
 {
+    if (kernel == kSimLane) return launch_des_lane(p, grid, smem, stream);
     if (kernel == kSimWide) return launch_des(p, grid, smem, stream);
     return launch_des_packed(p, kernel == kSimPackedStaged, grid, smem, stream);
 }

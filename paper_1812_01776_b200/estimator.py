@@ -22,7 +22,7 @@ IL_OK = 0
 IL_ERR_INVALID_ARG, IL_ERR_BAD_TOPOLOGY, IL_ERR_BAD_PROFILE, IL_ERR_BAD_TRACE = -1, -2, -3, -4
 IL_ERR_BAD_CONFIG, IL_ERR_NOMEM, IL_ERR_CUDA, IL_ERR_ITER_LIMIT = -5, -6, -7, -8
 IL_ERR_TOO_LARGE = -9
-IL_VARIANT_AUTO, IL_VARIANT_WIDE, IL_VARIANT_STAGED = 0, 1, 2
+IL_VARIANT_AUTO, IL_VARIANT_WIDE, IL_VARIANT_STAGED, IL_VARIANT_LANES = 0, 1, 2, 3
 IL_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 EXPORTS = ["il_estimator_create", "il_estimator_destroy", "il_estimate", "il_estimate_device",

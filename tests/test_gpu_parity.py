@@ -64,7 +64,7 @@ def test_hand_traces(il, case):
     assert (int(p99[0]), int(miss[0])) == (case["p99_us"], case["miss"])
 
 
-@pytest.mark.parametrize("variant", [0, 1, 2], ids=["packed", "wide", "staged"])
+@pytest.mark.parametrize("variant", [0, 1, 2, 3], ids=["packed", "wide", "staged", "lanes"])
 @pytest.mark.parametrize("seed", range(12))
 def test_random_small(il, oracle, seed, variant):
     w = workloads.random_small(seed, S=1 + seed % 6, H=3, Bmax=[4, 33, 64][seed % 3], n=700 + 37 * seed,
@@ -74,7 +74,7 @@ def test_random_small(il, oracle, seed, variant):
     check(il, oracle, w, host=(seed % 2 == 0), variant=variant)
 
 
-@pytest.mark.parametrize("variant", [0, 1, 2], ids=["packed", "wide", "staged"])
+@pytest.mark.parametrize("variant", [0, 1, 2, 3], ids=["packed", "wide", "staged", "lanes"])
 @pytest.mark.parametrize("seed", [1, 4, 7, 10])
 def test_per_query_latencies(il, oracle, seed, variant):
     """The full answer of the Estimator, query by query, against the oracle."""
@@ -133,7 +133,7 @@ def test_config1_full(il, oracle):
     assert st["batches"] > 0 and st["kernel_launches"] == 3 * st["chunks"]
 
 
-@pytest.mark.parametrize("variant", [0, 1, 2], ids=["packed", "wide", "staged"])
+@pytest.mark.parametrize("variant", [0, 1, 2, 3], ids=["packed", "wide", "staged", "lanes"])
 @pytest.mark.parametrize("cid,n,C", [(2, 5000, 300), (3, 6001, 200), (4, 3000, 150), (5, 4097, 260)])
 def test_configs_reduced(il, oracle, cid, n, C, variant):
     check(il, oracle, workloads.make(cid, n_queries=n, n_candidates=C), host=False, variant=variant)
