@@ -28,13 +28,18 @@
 //     leaf, to the candidate's slab as a (finish, query) record.
 //
 // Stage s+1 reads what stage s wrote a few iterations earlier.  A lane knows
-// how far its parent has got from two words in shared memory that the parent
-// publishes every iteration: the number of records written so far, and a lower
-// bound on the time of every record still to come (its watermark).  A batch
-// that is not full and has seen all records written so far may only be closed
-// once the parent's watermark has passed the batch's dispatch time; until then
-// the lane idles for that iteration.  Parents never wait for children, so the
-// root always advances and every wait ends.
+// how far its parent has got from one word in shared memory that the parent
+// publishes every iteration: the number of records written so far, and a flag
+// once it has written all of them.  A batch that is not full is closed when the
+// next record turns out not to belong to it (or the stream has ended), so a
+// stage simply trails its parent by a few records; parents never wait for
+// children, so the root always advances and every wait ends.
+//
+// Everything a lane reads from a stream in global memory (the record it
+// examines, the record it hands on) is copied into a small per-lane staging ring
+// in shared memory by an asynchronous copy (cp.async) issued three iterations
+// before its use; one commit group per iteration, at most two groups pending, so
+// that no instruction of the loop waits for global memory.
 //
 // Records and keys are the packed 64-bit words of des_packed_kernel.cu:
 // (time << q) | query for stream records, (finish << q) | index of the batch's
@@ -47,30 +52,58 @@ namespace il {
 namespace {
 
 constexpr int kLaneWarps = 2;                  // warps per CTA
-constexpr int kRcap = IL_MAX_REPLICAS;         // ring positions of a lane's slot list
+constexpr int kRing = 32;                      // ring positions of a lane's slot list (>= IL_MAX_REPLICAS)
+constexpr uint32_t kDone = 0x80000000u;
 constexpr uint64_t kInf = ~0ull;
+constexpr int kLag = 40;        // records a stage stays behind its parent while the parent is running
+constexpr int kStage = 4;       // staging ring positions (pending groups + 2)
+constexpr int kPending = 2;     // commit groups that may still be in flight at the end of an iteration
+
+__device__ __forceinline__ void cp_async8(void *smem_dst, const void *gsrc)
+{
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // Shared memory of one warp.
 struct WarpMem {
-    uint64_t key[kRcap][32];     // slot lists, sorted by key from position lhead on (ring); [pos][lane]
-    uint32_t cnt[kRcap][32];     // batch size held by the slot (0: replica never used)
+    // Per lane a ring of batches, [pos][lane].  Positions [epos, lpos): batches whose slot has been
+    // taken over, waiting to be handed on, in key order.  Positions [lpos, tpos): the slots in use,
+    // sorted by key.
+    uint64_t key[kRing][32];     // (finish << q) | index of the batch's first arrival
+    uint32_t cnt[kRing][32];     // batch size
+    // Staging rings filled by cp.async, [position][lane]: the next records of the lane's arrival stream
+    // (position = record index mod kStage), and the records it is handing on with the finish << q of
+    // their batch (position = iteration mod kStage)
+    uint64_t stage_x[kStage][32];
+    uint64_t stage_e[kStage][32];
+    uint64_t stage_b[kStage][32];
     // Mailboxes, double-buffered by iteration parity: what iteration k publishes in buffer k & 1 is read
     // in iteration k + 1, while iteration k + 1 publishes into the other buffer; one warp barrier per
     // iteration then separates every write of a word from the reads of its previous value.
-    uint64_t wmark[2][32];       // lane's watermark: (lower bound on the time of records still to come) << q
-    uint32_t avail[2][32];       // records written so far into the lane's arrival stream (by its parent lane)
+    uint32_t avail[2][32];       // records written so far into the lane's arrival stream (by its parent
+                                 // lane); kDone set once that is all of them
 };
 
 }  // namespace
 
+// BRANCHY: some stage routes by a branch bit (otherwise every stage has one way out).
+template <bool BRANCHY>
 __global__ void __launch_bounds__(kLaneWarps * 32)
 des_lane_kernel(const __grid_constant__ DesParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    int32_t *s_lat = reinterpret_cast<int32_t *>(smem_raw);
+    // per table entry the 64-bit word (latency << q) - qmask: finish key base = dispatch key + that
+    uint64_t *s_latq = reinterpret_cast<uint64_t *>(smem_raw);
     const int n_tab = p.S * p.H * p.Bmax;
-    WarpMem *wm_all = reinterpret_cast<WarpMem *>(smem_raw + ((size_t)n_tab * 4 + 15) / 16 * 16);
-    for (int i = threadIdx.x; i < n_tab; i += blockDim.x) s_lat[i] = p.lat[i];
+    WarpMem *wm_all = reinterpret_cast<WarpMem *>(smem_raw + ((size_t)n_tab * 8 + 15) / 16 * 16);
+    const int q = p.qbits;
+    const uint64_t qmask = (1ull << q) - 1ull;
+    for (int i = threadIdx.x; i < n_tab; i += blockDim.x)
+        s_latq[i] = ((uint64_t)(uint32_t)p.lat[i] << q) - qmask;
     __syncthreads();
 
     const unsigned full = 0xffffffffu;
@@ -80,27 +113,24 @@ des_lane_kernel(const __grid_constant__ DesParams p)
     const int S = p.S, cpw = p.cpw;
     const int j = lane / S, s = lane - j * S;
     const bool lane_used = j < cpw;
-    const int q = p.qbits;
-    const uint64_t qmask = (1ull << q) - 1ull;
 
     // static facts of this lane's stage
-    int parent = -1;
     int exit_off = 0;
-    for (int u = 0; u < S; u++) {
+    for (int u = 0; u < s; u++) {
         const int a = p.dest_a[u], b2 = p.dest_b[u];
-        if (u != s && (a == s || b2 == s)) parent = u;
-        if (u < s) {
-            int kids = 0;
-            if (a >= 0) kids += p.n_s[a];
-            if (b2 >= 0 && b2 != a) kids += p.n_s[b2];
-            exit_off += p.n_s[u] - kids;
-        }
+        int kids = 0;
+        if (a >= 0) kids += p.n_s[a];
+        if (b2 >= 0 && b2 != a) kids += p.n_s[b2];
+        exit_off += p.n_s[u] - kids;
     }
-    const int par_lane = (lane_used && s > 0 && parent >= 0) ? j * S + parent : lane;
     const int da = p.dest_a[s], db = p.dest_b[s];
     const int bit = p.bit[s];
     const uint32_t n_in = lane_used ? (uint32_t)p.n_s[s] : 0u;
     const unsigned group_mask = lane_used ? (((1u << S) - 1u) << (j * S)) : 0u;
+    // mailbox of the child on either side; a lane without that child writes a word nobody reads
+    // (its own entry of a spare row would do as well: lanes j * S + child are always in range)
+    const int lane_a = (da < 0 || !lane_used) ? -1 : j * S + da;
+    const int lane_b = (db < 0 || db == da || !lane_used) ? -1 : j * S + db;
 
     const int64_t wslot = (int64_t)blockIdx.x * kLaneWarps + wid;
     uint64_t *my_block = p.lane_ws + (wslot * cpw + (lane_used ? j : 0)) * p.lane_elems;
@@ -126,148 +156,144 @@ des_lane_kernel(const __grid_constant__ DesParams p)
         }
         const bool live = has && !cand_bad && n_in > 0;
 
-        const int R = cfg.replicas, mb = cfg.max_batch;
-        const int32_t *row = s_lat + (s * p.H + cfg.hw) * p.Bmax;
+        const uint32_t R = cfg.replicas;
+        const int mb = cfg.max_batch;
+        const uint64_t *row = s_latq + (s * p.H + cfg.hw) * p.Bmax - 1;   // row[b], b = 1..Bmax
         uint64_t *out_a = da < 0 ? slab + exit_off : my_block + p.lane_off[da];
         uint64_t *out_b = db < 0 ? slab + exit_off : my_block + p.lane_off[db];
-        const int lane_a = (da < 0 || !lane_used) ? -1 : j * S + da;
-        const int lane_b = (db < 0 || db == da || !lane_used) ? -1 : j * S + db;
 
-        // slot list: R slots of never-used replicas (key 0 sorts first)
-        if (live) for (int r = 0; r < R; r++) { wm.key[r][lane] = 0; wm.cnt[r][lane] = 0; }
-        wm.avail[0][lane] = 0; wm.avail[1][lane] = 0;
-        wm.wmark[0][lane] = live ? 0 : kInf; wm.wmark[1][lane] = live ? 0 : kInf;
+        // the root's stream is complete from the start; a stage nobody visits is finished at once
+        const uint32_t avail0 = (s == 0 || !live) ? (n_in | kDone) : 0u;
+        wm.avail[0][lane] = avail0; wm.avail[1][lane] = avail0;
         __syncwarp();
 
-        uint32_t lhead = 0;          // ring position of the list's first slot
-        int lcount = R;              // slots in the list (R, or R - 1 while a batch is open)
-        int nempty = R;              // never-used slots still at the front of the list
-        uint64_t kfront = 0;         // key of the list's first slot (kInf when the list is empty)
+        uint32_t epos = 0, lpos = 0, tpos = 0;   // ring positions, see WarpMem
+        uint64_t kfront = kInf;      // key at lpos (kInf when no slot is in use)
+        uint64_t ktail = 0;          // largest key in [lpos, tpos)
         uint32_t head = 0;           // index of the open batch's first record
         int b = 0;                   // size of the open batch (0: none)
         uint64_t tk = 0;             // open batch's dispatch time as (t << q) | qmask
         uint64_t e_base = 0;         // finish << q of the batch being handed on
         uint32_t e_idx = 0;          // its next record in the arrival stream
-        int e_left = 0;              // records of it still to hand on
-        uint64_t rec_e = 0;          // in[e_idx], loaded ahead
-        uint64_t nx = 0;             // in[head + b], loaded ahead when nx_ok
-        bool nx_ok = false;
+        uint32_t e_left = 0;         // records of it not yet fetched
+        uint32_t vmask = 0;          // bit k: the record fetched k + 1 iterations ago is on its way out
+        // fetch cursor of the arrival stream: records below fx have been requested; fx1..fx3 are its
+        // values at the end of the previous three iterations, so records below fx3 have arrived
+        uint32_t fx = 0, fx1 = 0, fx2 = 0, fx3 = 0;
         uint32_t tail_a = 0, tail_b = 0;
         unsigned nb = 0;
         bool done = !live;
-        long long guard = 8ll * p.n * (S + 1) + 4096;
-        int par = 0;                 // buffer this iteration publishes into; it reads the other one
-        uint64_t w_pub = live ? 0 : kInf;
+        const unsigned long long limit = 8ull * (unsigned)p.n * (unsigned)(S + 1) + 4096ull;
+        uint32_t guard = limit > 0xffffffffull ? 0xffffffffu : (uint32_t)limit;
+        int par = 0;                 // mailbox buffer this iteration publishes into; it reads the other one
+        uint32_t av = avail0;        // mailbox word this iteration works with: the one read an iteration ago
+        uint32_t it = 0;
 
-        while (!__all_sync(full, done)) {
-            uint32_t avail = n_in;
-            uint64_t wp = kInf;
-            if (s != 0) { avail = wm.avail[par ^ 1][lane]; wp = wm.wmark[par ^ 1][par_lane]; }
+        for (;;) {
+            const uint32_t av_next = wm.avail[par ^ 1][lane];
             if (!done) {
-                // ---- emit one record of the batch being handed on
-                if (e_left > 0) {
-                    const uint32_t qid = (uint32_t)(rec_e & qmask);
-                    const uint64_t out = e_base | qid;
-                    bool to_b = false;
-                    if (bit >= 0) to_b = (p.bits[qid] >> bit) & 1;
-                    if (to_b) out_b[tail_b++] = out; else out_a[tail_a++] = out;
-                    e_idx++; e_left--;
-                    if (e_left > 0) rec_e = in[e_idx];
-                }
+                const uint32_t written = av & ~kDone;
+                const bool pdone = (av & kDone) != 0u;
+
                 // ---- examine one record of the arrival stream
                 const uint32_t i = head + (uint32_t)b;
-                bool close = false, consume = false;
-                if (i < avail) {
-                    if (!nx_ok) { nx = in[i]; nx_ok = true; }
-                    if (b > 0 && b < mb && nx <= tk) { b++; consume = true; }
-                    else close = b > 0;
-                } else if (i >= n_in) {
-                    close = b > 0;
-                } else {
-                    close = b > 0 && (b == mb || wp > tk);
-                }
+                const bool known = i < fx3;
+                const uint64_t ra = wm.stage_x[i & (kStage - 1)][lane];
+                const bool end = pdone && i >= written;
+                const bool join = known && b > 0 && b < mb && ra <= tk;
+                b += join ? 1 : 0;
+                const bool room = tpos - epos < (uint32_t)kRing;
+                const bool close = b > 0 && !join && (known || end || b == mb) && room;
                 if (close) {
-                    const uint64_t fk = (tk - qmask) + ((uint64_t)(uint32_t)row[b - 1] << q);
-                    const uint64_t key = fk | head;
-                    uint32_t pos = lhead + (uint32_t)lcount;
-                    while (pos != lhead) {
-                        const uint64_t prev = wm.key[(pos - 1) & (kRcap - 1)][lane];
-                        if (prev <= key) break;
-                        wm.key[pos & (kRcap - 1)][lane] = prev;
-                        wm.cnt[pos & (kRcap - 1)][lane] = wm.cnt[(pos - 1) & (kRcap - 1)][lane];
-                        pos--;
+                    const uint64_t key = (tk + row[b]) | head;
+                    uint32_t pos = tpos;
+                    if (tpos != lpos && key < ktail) {
+                        // a batch that finishes before one dispatched earlier: sorted insert
+#pragma unroll 1
+                        while (pos != lpos) {
+                            const uint64_t prev = wm.key[(pos - 1) & (kRing - 1)][lane];
+                            if (prev <= key) break;
+                            wm.key[pos & (kRing - 1)][lane] = prev;
+                            wm.cnt[pos & (kRing - 1)][lane] = wm.cnt[(pos - 1) & (kRing - 1)][lane];
+                            pos--;
+                        }
+                    } else {
+                        ktail = key;
                     }
-                    wm.key[pos & (kRcap - 1)][lane] = key;
-                    wm.cnt[pos & (kRcap - 1)][lane] = (uint32_t)b;
-                    if (pos == lhead) kfront = key;
-                    lcount++;
+                    wm.key[pos & (kRing - 1)][lane] = key;
+                    wm.cnt[pos & (kRing - 1)][lane] = (uint32_t)b;
+                    kfront = pos == lpos ? key : kfront;
+                    tpos++;
                     nb++;
                     head = i;
                     b = 0;
                 }
-                if (b == 0 && e_left == 0) {
-                    if (i < avail) {
-                        // open the next batch with record i; it takes over the first slot
-                        const uint32_t c0 = wm.cnt[lhead & (kRcap - 1)][lane];
-                        if (nempty > 0) nempty--;
-                        else {
-                            e_base = kfront & ~qmask;
-                            e_idx = (uint32_t)(kfront & qmask);
-                            e_left = (int)c0;
-                            rec_e = in[e_idx];
-                        }
-                        tk = max(kfront, nx) | qmask;
-                        lhead++; lcount--;
-                        kfront = lcount > 0 ? wm.key[lhead & (kRcap - 1)][lane] : kInf;
-                        b = 1;
-                        consume = true;
-                    } else if (i >= n_in) {
-                        // arrival stream exhausted: hand on what the slots still hold, in key order
-                        lhead += (uint32_t)nempty; lcount -= nempty; nempty = 0;
-                        if (lcount > 0) {
-                            const uint64_t k0 = wm.key[lhead & (kRcap - 1)][lane];
-                            e_base = k0 & ~qmask;
-                            e_idx = (uint32_t)(k0 & qmask);
-                            e_left = (int)wm.cnt[lhead & (kRcap - 1)][lane];
-                            rec_e = in[e_idx];
-                            lhead++; lcount--;
-                            kfront = lcount > 0 ? wm.key[lhead & (kRcap - 1)][lane] : kInf;
-                        } else {
-                            done = true;
-                        }
+                const bool open = known && !join && b == 0;
+                if (open) {
+                    // record i opens the next batch on the replica that is free first: one that was
+                    // never used (free from time 0) while there is one, else the slot with the smallest key
+                    uint64_t kf = 0;
+                    if (tpos - lpos == R) {
+                        kf = kfront;
+                        lpos++;
+                        kfront = lpos != tpos ? wm.key[lpos & (kRing - 1)][lane] : kInf;
                     }
+                    tk = max(kf, ra) | qmask;
+                    b = 1;
                 }
-                if (consume) {
-                    nx_ok = i + 1 < avail;
-                    if (nx_ok) nx = in[i + 1];
+                if (end && b == 0) lpos = tpos;     // stream exhausted: everything still held leaves, in key order
+
+                // ---- hand on the record requested three iterations ago
+                if (vmask & 4u) {
+                    const uint32_t sl = (it + 1u) & (kStage - 1);
+                    const uint32_t qid = (uint32_t)wm.stage_e[sl][lane] & (uint32_t)qmask;
+                    const uint64_t out = wm.stage_b[sl][lane] | qid;
+                    bool to_b = false;
+                    if (BRANCHY) to_b = bit >= 0 && ((p.bits[qid] >> bit) & 1);
+                    uint64_t *dst = to_b ? out_b + tail_b : out_a + tail_a;
+                    *dst = out;
+                    tail_b += to_b ? 1u : 0u;
+                    tail_a += to_b ? 0u : 1u;
                 }
-                // ---- publish: records written, and a lower bound on what is still to come
-                uint64_t w = kInf;
-                if (!done) {
-                    if (e_left > 0) w = e_base;
-                    else if (lcount > nempty)
-                        w = (nempty == 0 ? kfront : wm.key[(lhead + (uint32_t)nempty) & (kRcap - 1)][lane]) & ~qmask;
-                    uint64_t nxt;   // (time << q) + 1 unit that every batch still to be closed finishes at or after
-                    if (b > 0) nxt = tk + 1;
-                    else {
-                        const uint32_t i2 = head;      // b == 0: next record to open with
-                        uint64_t lb = kInf;
-                        if (i2 < avail && nx_ok) lb = nx & ~qmask;
-                        else if (i2 < n_in) lb = (i2 < avail) ? 0 : wp;
-                        nxt = lb == kInf ? kInf : lb + qmask + 1;
-                    }
-                    w = min(w, nxt);
+                // ---- request the next record to hand on
+                if (e_left == 0 && epos != lpos) {
+                    const uint64_t k = wm.key[epos & (kRing - 1)][lane];
+                    e_left = wm.cnt[epos & (kRing - 1)][lane];
+                    e_base = k & ~qmask;
+                    e_idx = (uint32_t)k & (uint32_t)qmask;
+                    epos++;
                 }
-                if (--guard < 0) { atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT); done = true; w = kInf; }
-                w_pub = w;
+                vmask = (vmask << 1) & 7u;
+                if (e_left > 0) {
+                    const uint32_t sl = it & (kStage - 1);
+                    cp_async8(&wm.stage_e[sl][lane], in + e_idx);
+                    wm.stage_b[sl][lane] = e_base;
+                    e_idx++; e_left--;
+                    vmask |= 1u;
+                }
+                // ---- request the next record to examine: up to kStage records from the one examined
+                // next, and (while the parent runs) kLag behind what it has written
+                const uint32_t i2 = head + (uint32_t)b;
+                if (fx < i2 + (uint32_t)kStage && (pdone ? fx < written : fx + (uint32_t)kLag < written)) {
+                    cp_async8(&wm.stage_x[fx & (kStage - 1)][lane], in + fx);
+                    fx++;
+                }
+                done = end && b == 0 && epos == tpos && vmask == 0u;
+                if (--guard == 0) { atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT); done = true; }
             }
+            fx3 = fx2; fx2 = fx1; fx1 = fx;
+            cp_async_commit();
+            cp_async_wait<kPending>();
             // every lane publishes every iteration (a finished lane repeats its last words)
-            wm.wmark[par][lane] = w_pub;
-            if (lane_a >= 0) wm.avail[par][lane_a] = tail_a;
-            if (lane_b >= 0) wm.avail[par][lane_b] = tail_b;
+            if (lane_a >= 0) wm.avail[par][lane_a] = tail_a | (done ? kDone : 0u);
+            if (lane_b >= 0) wm.avail[par][lane_b] = tail_b | (done ? kDone : 0u);
+            av = av_next;
             par ^= 1;
+            it++;
             __syncwarp();
+            if (__all_sync(full, done)) break;
         }
+        cp_async_wait<0>();
 
         if (live) {
             batches += nb;
@@ -290,11 +316,23 @@ des_lane_kernel(const __grid_constant__ DesParams p)
     if (lane == 0 && batches) { atomicAdd(&p.counters[1], batches); atomicAdd(&p.counters[2], alg_ops); }
 }
 
+namespace {
+bool any_branch(const DesParams &p)
+{
+    for (int s = 0; s < p.S; s++) if (p.bit[s] >= 0) return true;
+    return false;
+}
+}  // namespace
+
 cudaError_t launch_des_lane(const DesParams &p, int grid, size_t smem, cudaStream_t stream)
 {
-    cudaError_t e = cudaFuncSetAttribute(des_lane_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const bool br = any_branch(p);
+    cudaError_t e = br
+        ? cudaFuncSetAttribute(des_lane_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+        : cudaFuncSetAttribute(des_lane_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    des_lane_kernel<<<grid, kLaneWarps * 32, smem, stream>>>(p);
+    if (br) des_lane_kernel<true><<<grid, kLaneWarps * 32, smem, stream>>>(p);
+    else des_lane_kernel<false><<<grid, kLaneWarps * 32, smem, stream>>>(p);
     return cudaGetLastError();
 }
 
@@ -302,15 +340,15 @@ int des_lane_warps_per_cta() { return kLaneWarps; }
 
 size_t des_lane_smem(int n_tab)
 {
-    return ((size_t)n_tab * 4 + 15) / 16 * 16 + (size_t)kLaneWarps * sizeof(WarpMem);
+    return ((size_t)n_tab * 8 + 15) / 16 * 16 + (size_t)kLaneWarps * sizeof(WarpMem);
 }
 
 int des_lane_max_ctas_per_sm(size_t smem)
 {
     int n = 0;
-    if (cudaFuncSetAttribute(des_lane_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(des_lane_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return 0;
-    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, des_lane_kernel, kLaneWarps * 32, smem);
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, des_lane_kernel<true>, kLaneWarps * 32, smem);
     return e == cudaSuccess ? n : 0;
 }
 
