@@ -39,10 +39,10 @@ WORKLOADS = {
     4: "config4: linear 10-stage pipeline, 1,000,000 arrivals ramping 150->250 qps, 262,144 candidates",
     5: "config5: 8-stage tree with three branch points, 100,000 gamma arrivals (500 qps, CV 2), 1,048,576 candidates",
 }
-# DRAM bytes (read + write) of des_packed_kernel per query-event, from an ncu capture of a reduced case
+# DRAM bytes (read + write) of a simulation kernel per query-event, from an ncu capture of a reduced case
 # (1,024 candidates x 20,000 queries; traffic is proportional to the query-events processed).
-# Set to None whenever that kernel changes until the capture has been repeated.
-NCU_DRAM_BYTES_PER_QUERY_EVENT = 12.24
+# An entry is None whenever its kernel has changed since the capture.
+NCU_DRAM_BYTES_PER_QUERY_EVENT = {"des_packed_kernel": 12.24, "des_lane_kernel": None}
 METRIC = "candidate_configs_per_s"
 UNIT = "candidates/s"
 
@@ -228,6 +228,7 @@ def run_cuda(args):
 
     est = il.Estimator.from_workload(w, device=local)
     est.set_variant(args.variant)
+    kernel = est.kernel_name()
     ws_bytes = est.reserve_workspace(n_cand)
     stream = torch.cuda.Stream(device=dev)
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)   # > 126 MB of L2
@@ -313,7 +314,7 @@ def run_cuda(args):
     alu_achieved = alg_ops / sim_avg_s
     # HBM view of the same kernel: slab written once, streams written and read once, trace once per CTA wave
     n, S = w.n_queries, w.n_stages
-    rec_bytes = 12 if args.variant == 1 else 8       # wide: int64 time + int32 query; packed: one 64-bit record
+    rec_bytes = 12 if kernel == "des_kernel" else 8  # wide: int64 time + int32 query; else one 64-bit record
     stream_bytes = (events_per_cand - n) * 2 * rec_bytes
     hbm_bytes_per_cand = 8 * n + stream_bytes + 4 * S
     hbm_achieved = hbm_bytes_per_cand * n_cand / sim_avg_s / 1e9
@@ -328,7 +329,7 @@ def run_cuda(args):
                    "query_events_per_candidate": events_per_cand,
                    "l2": "256 MiB buffer written between steps; working set "
                          f"{ws_bytes / 2**30:.1f} GiB > L2",
-                   "workspace_bytes": ws_bytes, "kernel_variant": args.variant, "parallelism": f"candidates sharded over {world} GPU(s)"},
+                   "workspace_bytes": ws_bytes, "kernel_variant": args.variant, "kernel": kernel, "parallelism": f"candidates sharded over {world} GPU(s)"},
         "query_events_per_s": value * events_per_cand,
         "batches_per_s": batches * world * K / (total_ms * 1e-3) if batches else None,
         "mean_batch": events_per_cand * n_cand / batches if batches else None,
@@ -336,17 +337,17 @@ def run_cuda(args):
         "kernel_ms": {"simulate": sum(sim_ms) / K, "select": sum(sel_ms) / K},
         "roofline": {"bound": "alu", "achieved": alu_achieved / 1e12, "peak": alu_peak / 1e12,
                      "unit": "Tinteger-op/s", "frac": alu_achieved / alu_peak,
-                     "traffic": (NCU_DRAM_BYTES_PER_QUERY_EVENT * events_per_cand * n_cand
-                                 if NCU_DRAM_BYTES_PER_QUERY_EVENT and args.variant == 0 and args.workload == 2
+                     "traffic": (NCU_DRAM_BYTES_PER_QUERY_EVENT[kernel] * events_per_cand * n_cand
+                                 if NCU_DRAM_BYTES_PER_QUERY_EVENT.get(kernel) and args.workload == 2
                                  else None),
                      "traffic_unit": "DRAM bytes per launch (ncu capture of a reduced case, scaled by query-events)",
-                     "kernel": "des_kernel" if args.variant == 1 else "des_packed_kernel",
+                     "kernel": kernel,
                      "peak_source": "integer-issue probe of this run (warp-inst/s x 32 lanes)",
                      "issue_peak_warp_inst_per_s": issue_rate},
         "roofline_hbm": {"bound": "hbm", "achieved": hbm_achieved, "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": hbm_achieved / peaks["hbm_gbs"],
                          "peak_source": f"{peaks_kind} copy bandwidth",
-                         "kernel": "des_kernel" if args.variant == 1 else "des_packed_kernel"},
+                         "kernel": kernel},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(cfg_host.nbytes),
                 "d2h_bytes_per_step": int(16 * n_cand), "matches_device_path": same},
         "gpu_launches": int(launches),
@@ -387,8 +388,9 @@ def main():
     ap.add_argument("--queries", type=int, default=None,
                     help="trace length (default: the workload's 50,000); for profiler captures")
     ap.add_argument("--variant", type=int, default=0,
-                    help="simulation kernel: 0 default (packed records), 1 wide streams, "
-                         "2 packed records with the trace staged through shared memory")
+                    help="simulation kernel (IL_VARIANT_*): 0 the library's choice, 1 wide streams, "
+                         "2 packed records with the trace staged through shared memory, 3 lane kernel, "
+                         "4 packed records, one candidate per warp")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer timing (profiler captures)")
     args = ap.parse_args()
     if args.impl == "reference":

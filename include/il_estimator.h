@@ -267,24 +267,42 @@ IL_API int il_workspace_min_bytes(const il_estimator *est, size_t *bytes);
 IL_API int il_set_workspace(il_estimator *est, void *d_workspace, size_t bytes);
 
 /*
- * Chooses the simulation kernel.  IL_VARIANT_AUTO (default) uses the
- * packed-record kernel whenever every time the simulation can reach (last
- * arrival + sum over stages of n * largest table entry) fits in
- * 63 - max(5, ceil(log2 n)) bits, and the kernel with separate 64-bit time and
- * 32-bit query streams otherwise.  IL_VARIANT_WIDE forces the latter (it is
- * always valid; used to test it).  IL_VARIANT_STAGED is the packed-record
- * kernel with the shared trace staged through shared memory once per CTA (bulk
- * asynchronous copies into a ring of tiles that the CTA's four warps consume
- * together) instead of every warp reading it through L1/L2 on its own; on B200
- * it measured slower than the default (the warps of a CTA must then move
- * through the root stage within one ring length of each other), so it is not
- * the default.  All variants give identical results.
+ * Chooses the simulation kernel.  All variants give identical results.
+ *
+ * Records.  When every time the simulation can reach (last arrival + sum over
+ * stages of n * largest table entry) fits in 63 - q bits, q = max(5, ceil(log2 n)),
+ * a stream element is one 64-bit word (time << q) | query ("packed"); otherwise
+ * only IL_VARIANT_WIDE applies and every other choice falls back to it.
+ *
+ * IL_VARIANT_AUTO (default): the lane kernel when the inter-stage streams of one
+ *   candidate take at most 16 MiB, else the packed warp-per-candidate kernel.
+ * IL_VARIANT_LANES: one lane per (candidate, stage); the stages of a candidate
+ *   run side by side as a pipeline inside one warp, floor(32 / S) candidates per
+ *   warp.  Keeps every stage's arrival stream of every resident candidate in
+ *   the workspace.
+ * IL_VARIANT_PACKED: one candidate per warp, stages one after the other, replica
+ *   slots across the lanes, warp-level primitives for the queue count and the
+ *   slot to reuse.
+ * IL_VARIANT_STAGED: IL_VARIANT_PACKED with the shared trace staged through
+ *   shared memory once per CTA (bulk asynchronous copies into a ring of tiles
+ *   that the CTA's four warps consume together) instead of every warp reading
+ *   it through L1/L2 on its own; on B200 it measured slower (the warps of a CTA
+ *   must then move through the root stage within one ring length of each other).
+ * IL_VARIANT_WIDE: one candidate per warp with separate 64-bit time and 32-bit
+ *   query streams; always valid.
+ * il_workspace_bytes depends on the variant in force: set the variant first.
  */
 #define IL_VARIANT_AUTO 0
 #define IL_VARIANT_WIDE 1
 #define IL_VARIANT_STAGED 2
 #define IL_VARIANT_LANES 3
+#define IL_VARIANT_PACKED 4
 IL_API int il_set_variant(il_estimator *est, int variant);
+
+/* Name of the simulation kernel the handle's next estimate call will launch
+ * (the choice il_set_variant describes, resolved for the bound inputs);
+ * a static string, never NULL. */
+IL_API const char *il_kernel_name(const il_estimator *est);
 
 /* Counters of the last estimate call on this handle. */
 IL_API int il_get_stats(const il_estimator *est, il_stats *out);

@@ -81,6 +81,12 @@ struct Plan {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// The lane kernel keeps every stage's whole arrival stream per resident candidate.  Beyond this many
+// bytes per candidate too few candidates fit the device at once and the warp-per-candidate kernel,
+// which needs two streams whatever the depth, is the faster one (measured on the 10-stage, 10^6-query
+// workload: 72 MB per candidate, 0.93x).
+constexpr int64_t kLaneAutoBytes = INT64_C(16) << 20;
+
 bool use_packed(const il_estimator *e)
 {
     return e->can_pack && e->variant != IL_VARIANT_WIDE;
@@ -90,6 +96,7 @@ int sim_kernel(const il_estimator *e)
 {
     if (!use_packed(e)) return kSimWide;
     if (e->variant == IL_VARIANT_LANES && e->lane_ok) return kSimLane;
+    if (e->variant == IL_VARIANT_AUTO && e->lane_ok && e->lane_elems * 8 <= kLaneAutoBytes) return kSimLane;
     return e->variant == IL_VARIANT_STAGED ? kSimPackedStaged : kSimPacked;
 }
 
@@ -473,10 +480,21 @@ int il_set_stream(il_estimator *e, void *cuda_stream)
 
 int il_set_variant(il_estimator *e, int variant)
 {
-    if (!e || variant < IL_VARIANT_AUTO || variant > IL_VARIANT_LANES) return IL_ERR_INVALID_ARG;
+    if (!e || variant < IL_VARIANT_AUTO || variant > IL_VARIANT_PACKED) return IL_ERR_INVALID_ARG;
     e->variant = variant;
     e->ctas_per_sm = ctas_for(e);
     return IL_OK;
+}
+
+const char *il_kernel_name(const il_estimator *e)
+{
+    if (!e) return "";
+    switch (sim_kernel(e)) {
+    case kSimLane: return "des_lane_kernel";
+    case kSimPacked: return "des_packed_kernel";
+    case kSimPackedStaged: return "des_packed_kernel<staged>";
+    default: return "des_kernel";
+    }
 }
 
 int il_workspace_bytes(const il_estimator *e, int64_t n_candidates, size_t *bytes)

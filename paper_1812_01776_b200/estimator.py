@@ -22,13 +22,13 @@ IL_OK = 0
 IL_ERR_INVALID_ARG, IL_ERR_BAD_TOPOLOGY, IL_ERR_BAD_PROFILE, IL_ERR_BAD_TRACE = -1, -2, -3, -4
 IL_ERR_BAD_CONFIG, IL_ERR_NOMEM, IL_ERR_CUDA, IL_ERR_ITER_LIMIT = -5, -6, -7, -8
 IL_ERR_TOO_LARGE = -9
-IL_VARIANT_AUTO, IL_VARIANT_WIDE, IL_VARIANT_STAGED, IL_VARIANT_LANES = 0, 1, 2, 3
+IL_VARIANT_AUTO, IL_VARIANT_WIDE, IL_VARIANT_STAGED, IL_VARIANT_LANES, IL_VARIANT_PACKED = 0, 1, 2, 3, 4
 IL_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 EXPORTS = ["il_estimator_create", "il_estimator_destroy", "il_estimate", "il_estimate_device",
            "il_set_stream", "il_workspace_bytes", "il_workspace_min_bytes", "il_set_workspace",
            "il_get_stats", "il_stage_visits", "il_strerror", "il_last_cuda_error",
-           "il_measure_int_issue", "il_estimate_device_static", "il_set_variant", "il_estimate_latencies", "il_traffic_envelope"]
+           "il_measure_int_issue", "il_estimate_device_static", "il_set_variant", "il_estimate_latencies", "il_traffic_envelope", "il_kernel_name"]
 
 
 class ILError(RuntimeError):
@@ -98,6 +98,8 @@ def load_library():
     lib.il_estimate_latencies.argtypes = [vp, vp, vp]
     lib.il_traffic_envelope.restype = ctypes.c_int
     lib.il_traffic_envelope.argtypes = [vp, vp, ctypes.c_int32, vp]
+    lib.il_kernel_name.restype = ctypes.c_char_p
+    lib.il_kernel_name.argtypes = [vp]
     lib.il_set_variant.restype = ctypes.c_int
     lib.il_set_variant.argtypes = [vp, ctypes.c_int]
     lib.il_set_stream.restype = ctypes.c_int
@@ -214,6 +216,11 @@ def il_set_variant(handle, variant: int) -> None:
     _check(load_library().il_set_variant(handle, int(variant)), "il_set_variant")
 
 
+def il_kernel_name(handle) -> str:
+    """il_kernel_name: the simulation kernel the next estimate call launches."""
+    return load_library().il_kernel_name(handle).decode()
+
+
 def il_set_stream(handle, cuda_stream: int) -> None:
     _check(load_library().il_set_stream(handle, cuda_stream), "il_set_stream")
 
@@ -314,8 +321,11 @@ class Estimator:
         return self._ws.numel()
 
     def set_variant(self, variant: int) -> None:
-        """IL_VARIANT_AUTO, IL_VARIANT_WIDE or IL_VARIANT_STAGED (see il_set_variant)."""
+        """One of the IL_VARIANT_* constants (see il_set_variant in the C header)."""
         il_set_variant(self._h, variant)
+
+    def kernel_name(self) -> str:
+        return il_kernel_name(self._h)
 
     def use_current_stream(self) -> None:
         il_set_stream(self._h, self._torch.cuda.current_stream(self.device).cuda_stream)

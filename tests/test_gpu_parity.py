@@ -64,7 +64,7 @@ def test_hand_traces(il, case):
     assert (int(p99[0]), int(miss[0])) == (case["p99_us"], case["miss"])
 
 
-@pytest.mark.parametrize("variant", [0, 1, 2, 3], ids=["packed", "wide", "staged", "lanes"])
+@pytest.mark.parametrize("variant", [4, 1, 2, 3], ids=["packed", "wide", "staged", "lanes"])
 @pytest.mark.parametrize("seed", range(12))
 def test_random_small(il, oracle, seed, variant):
     w = workloads.random_small(seed, S=1 + seed % 6, H=3, Bmax=[4, 33, 64][seed % 3], n=700 + 37 * seed,
@@ -74,7 +74,7 @@ def test_random_small(il, oracle, seed, variant):
     check(il, oracle, w, host=(seed % 2 == 0), variant=variant)
 
 
-@pytest.mark.parametrize("variant", [0, 1, 2, 3], ids=["packed", "wide", "staged", "lanes"])
+@pytest.mark.parametrize("variant", [4, 1, 2, 3], ids=["packed", "wide", "staged", "lanes"])
 @pytest.mark.parametrize("seed", [1, 4, 7, 10])
 def test_per_query_latencies(il, oracle, seed, variant):
     """The full answer of the Estimator, query by query, against the oracle."""
@@ -101,8 +101,9 @@ def test_per_query_latencies_workloads(il, oracle):
                 assert np.array_equal(est.latencies(w.configs[c]), exp), (cid, c)
 
 
+@pytest.mark.parametrize("variant", [4, 0], ids=["packed", "auto"])
 @pytest.mark.parametrize("seed", range(6))
-def test_times_scaled_beyond_the_32_bit_loop(il, oracle, seed):
+def test_times_scaled_beyond_the_32_bit_loop(il, oracle, seed, variant):
     """Latencies of 2^24 us and more take the 64-bit stage loop of the packed
     kernel (its run step, late-slot merge and single step included)."""
     w = workloads.random_small(200 + seed, S=2 + seed % 4, H=2, Bmax=[4, 33, 64][seed % 3], n=900, C=30,
@@ -112,11 +113,12 @@ def test_times_scaled_beyond_the_32_bit_loop(il, oracle, seed):
     w.arrival_us = w.arrival_us * 4096
     w.slo_us = w.slo_us * 4096
     assert w.latency_us.min() >= 1 << 24
-    check(il, oracle, w)
+    check(il, oracle, w, variant=variant)
 
 
+@pytest.mark.parametrize("variant", [4, 0], ids=["packed", "auto"])
 @pytest.mark.parametrize("seed", range(6))
-def test_sparse_traces_move_the_epoch(il, oracle, seed):
+def test_sparse_traces_move_the_epoch(il, oracle, seed, variant):
     """Gaps between arrivals far beyond 2^30 us (and, for odd seeds, services
     long enough that batches stay in flight across them) exercise the 32-bit
     loop's epoch moves and its hand-over to the 64-bit loop."""
@@ -125,15 +127,16 @@ def test_sparse_traces_move_the_epoch(il, oracle, seed):
                                lat_lo=1000, lat_hi=(1 << 24) - 1 if seed % 2 else 50000,
                                equal_stamp_every=(2 if seed == 4 else 0))
     assert np.diff(w.arrival_us).max() > (1 << 30)
-    check(il, oracle, w)
+    check(il, oracle, w, variant=variant)
 
 
 def test_config1_full(il, oracle):
     st = check(il, oracle, workloads.make(1))
-    assert st["batches"] > 0 and st["kernel_launches"] == 3 * st["chunks"]
+    # the lane kernel needs no ordering pass: (simulate, select) or (order, simulate, select) per chunk
+    assert st["batches"] > 0 and st["kernel_launches"] in (2 * st["chunks"], 3 * st["chunks"])
 
 
-@pytest.mark.parametrize("variant", [0, 1, 2, 3], ids=["packed", "wide", "staged", "lanes"])
+@pytest.mark.parametrize("variant", [4, 1, 2, 3], ids=["packed", "wide", "staged", "lanes"])
 @pytest.mark.parametrize("cid,n,C", [(2, 5000, 300), (3, 6001, 200), (4, 3000, 150), (5, 4097, 260)])
 def test_configs_reduced(il, oracle, cid, n, C, variant):
     check(il, oracle, workloads.make(cid, n_queries=n, n_candidates=C), host=False, variant=variant)
@@ -150,12 +153,14 @@ def test_times_too_large_to_pack_fall_back_to_wide_kernel(il, oracle):
     assert np.array_equal(p99, exp[0]) and np.array_equal(miss, exp[1])
 
 
-def test_multi_chunk_small_workspace(il, oracle):
+@pytest.mark.parametrize("variant", [4, 3], ids=["packed", "lanes"])
+def test_multi_chunk_small_workspace(il, oracle, variant):
     """A workspace that holds only a few candidates forces many chunks."""
     w = workloads.make(2, n_queries=2000, n_candidates=100)
     with il.Estimator.from_workload(w) as est:
+        est.set_variant(variant)
         lo = il.il_workspace_min_bytes(est._h)
-    st = check(il, oracle, w, ws_bytes=lo + 40 * 2000 * 8)
+    st = check(il, oracle, w, ws_bytes=lo + 40 * 2000 * 8, variant=variant)
     assert st["chunks"] > 1
 
 
@@ -222,11 +227,12 @@ def test_repeatable_and_stream(il, oracle):
                 assert np.array_equal(b.cpu().numpy(), exp[1])
 
 
-def test_config2_full_size_sampled(il, oracle):
+@pytest.mark.parametrize("variant", [0, 4], ids=["auto", "packed"])
+def test_config2_full_size_sampled(il, oracle, variant):
     """Full trace and full candidate set in the configuration the bench times;
     a seeded sample of candidates plus structured extremes is checked one by one."""
     w = workloads.make(2)
-    p99, miss, st = gpu_run(il, w, host=False)
+    p99, miss, st = gpu_run(il, w, host=False, variant=variant)
     rng = np.random.default_rng(2)
     idx = rng.choice(w.n_candidates, size=96, replace=False)
     exp = oracle.estimate_many_parallel(w.parent, w.cond_bit, w.cond_val, w.latency_us,
@@ -234,7 +240,7 @@ def test_config2_full_size_sampled(il, oracle):
     assert np.array_equal(p99[idx], exp[0]) and np.array_equal(miss[idx], exp[1])
     # extremes: every hardware type with min/max replicas and max batch 1 / 32
     ext = np.array([[[h, mb, R, 0]] * 4 for h in range(3) for mb in (1, 32) for R in (1, 8)], np.uint8)
-    got = gpu_run(il, w, configs=ext, host=True)
+    got = gpu_run(il, w, configs=ext, host=True, variant=variant)
     exp = oracle.estimate_many_parallel(w.parent, w.cond_bit, w.cond_val, w.latency_us,
                                         w.arrival_us, w.branch_bits, ext, w.slo_us)
     assert np.array_equal(got[0], exp[0]) and np.array_equal(got[1], exp[1])
@@ -294,3 +300,26 @@ def test_config4_full_trace_candidate_subset(il, oracle):
     the first 8,192 candidates of the same seeded draw and checks a sample."""
     w = workloads.make(4, n_candidates=8192)
     _sampled_check(il, oracle, w, 24, 4, _extremes(10, 4, (1, 64), (1, 16)))
+
+
+def test_kernel_choice(il):
+    """The default picks the lane kernel while a candidate's inter-stage streams are small, the
+    warp-per-candidate packed kernel beyond, and the wide kernel when times do not fit a record."""
+    from paper_1812_01776_b200 import estimator as E
+    w = workloads.make(2, n_queries=5000, n_candidates=4)
+    with il.Estimator.from_workload(w) as est:
+        assert est.kernel_name() == "des_lane_kernel"
+        est.set_variant(E.IL_VARIANT_PACKED)
+        assert est.kernel_name() == "des_packed_kernel"
+        est.set_variant(E.IL_VARIANT_WIDE)
+        assert est.kernel_name() == "des_kernel"
+    w.arrival_us = w.arrival_us + (1 << 58)
+    with il.Estimator.from_workload(w) as est:
+        assert est.kernel_name() == "des_kernel"
+        est.set_variant(E.IL_VARIANT_LANES)
+        assert est.kernel_name() == "des_kernel"
+    w = workloads.make(4, n_candidates=2)          # 9 x 10^6 stream records per candidate
+    with il.Estimator.from_workload(w) as est:
+        assert est.kernel_name() == "des_packed_kernel"
+        est.set_variant(E.IL_VARIANT_LANES)
+        assert est.kernel_name() == "des_lane_kernel"
