@@ -125,7 +125,8 @@ typedef struct {
     int64_t batches;         /* batches dispatched, all candidates, all stages           */
     int64_t algorithmic_ops; /* integer operations the method needs: per batch R + max_batch + 4
                                 (replica min, queue count, table add, slot update), per query-event 3 */
-    int64_t chunks;          /* how many (order, simulate, select) launch triples the call made */
+    int64_t chunks;          /* how many (simulate, select) launch groups the call made (the
+                                warp-per-candidate kernels add an ordering launch to each)  */
     int64_t kernel_launches; /* kernels launched by the call                             */
     double  sim_ms;          /* device time of the simulation kernels (CUDA events)      */
     double  select_ms;       /* device time of the percentile kernels (CUDA events)      */

@@ -86,6 +86,11 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // which needs two streams whatever the depth, is the faster one (measured on the 10-stage, 10^6-query
 // workload: 72 MB per candidate, 0.93x).
 constexpr int64_t kLaneAutoBytes = INT64_C(16) << 20;
+// Resident CTAs (of two warps) per SM for the lane kernel.  Two warps per scheduler keep the issue
+// slots about as busy as more would, and every further warp lengthens all chains through the
+// shared-memory pipe: on B200, workload 2 with 16,384 candidates took 101.7 / 79.2 / 68.4 / 71.1 / 85.5 ms
+// with 2 / 3 / 4 / 5 / 7 CTAs per SM; the tree workloads did not care from 4 on.
+constexpr int kLaneCtasPerSm = 4;
 
 bool use_packed(const il_estimator *e)
 {
@@ -451,7 +456,7 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     e->ctas_per_sm_packed = des_packed_max_ctas_per_sm(false, e->smem);
     e->ctas_per_sm_staged = des_packed_max_ctas_per_sm(true, e->smem);
     e->smem_lane = des_lane_smem(S * H * B);
-    e->ctas_per_sm_lane = des_lane_max_ctas_per_sm(e->smem_lane);
+    e->ctas_per_sm_lane = std::min(des_lane_max_ctas_per_sm(e->smem_lane), kLaneCtasPerSm);
     if (e->ctas_per_sm_wide < 1 || e->ctas_per_sm_packed < 1 || e->ctas_per_sm_staged < 1 ||
         e->ctas_per_sm_lane < 1)
         return fail(IL_ERR_CUDA);
