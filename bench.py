@@ -43,6 +43,9 @@ WORKLOADS = {
 # (1,024 candidates x 20,000 queries; traffic is proportional to the query-events processed).
 # An entry is None whenever its kernel has changed since the capture.
 NCU_DRAM_BYTES_PER_QUERY_EVENT = {"des_packed_kernel": 12.24, "des_lane_kernel": 7.41}
+# Warp instructions executed per query-event (smsp__inst_executed.sum of the same captures): how many issue slots
+# the kernel spends, next to the algorithmic operation count of the roofline.
+NCU_WARP_INST_PER_QUERY_EVENT = {"des_packed_kernel": 32.9, "des_lane_kernel": 7.02}
 METRIC = "candidate_configs_per_s"
 UNIT = "candidates/s"
 
@@ -343,7 +346,10 @@ def run_cuda(args):
                      "traffic_unit": "DRAM bytes per launch (ncu capture of a reduced case, scaled by query-events)",
                      "kernel": kernel,
                      "peak_source": "integer-issue probe of this run (warp-inst/s x 32 lanes)",
-                     "issue_peak_warp_inst_per_s": issue_rate},
+                     "issue_peak_warp_inst_per_s": issue_rate,
+                     "issue_slots_used": (NCU_WARP_INST_PER_QUERY_EVENT[kernel] * events_per_cand * n_cand
+                                          / sim_avg_s / issue_rate
+                                          if NCU_WARP_INST_PER_QUERY_EVENT.get(kernel) and args.workload == 2 else None)},
         "roofline_hbm": {"bound": "hbm", "achieved": hbm_achieved, "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": hbm_achieved / peaks["hbm_gbs"],
                          "peak_source": f"{peaks_kind} copy bandwidth",

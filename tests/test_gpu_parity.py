@@ -323,3 +323,13 @@ def test_kernel_choice(il):
         assert est.kernel_name() == "des_packed_kernel"
         est.set_variant(E.IL_VARIANT_LANES)
         assert est.kernel_name() == "des_lane_kernel"
+
+
+@pytest.mark.parametrize("variant", [3, 4], ids=["lanes", "packed"])
+@pytest.mark.parametrize("S,tree", [(11, False), (13, True), (16, False), (16, True)])
+def test_deep_pipelines(il, oracle, S, tree, variant):
+    """Up to the largest stage count the interface takes (16): from 11 stages on only two candidates
+    share a warp of the lane kernel, and some of its lanes stay idle."""
+    w = workloads.random_small(400 + S + int(tree), S=S, H=2, Bmax=16, n=1500, C=21, max_replicas=6, tree=tree,
+                               qps=300.0, cv=2.0, lat_lo=200, lat_hi=9000, equal_stamp_every=(5 if tree else 0))
+    check(il, oracle, w, host=False, variant=variant)
