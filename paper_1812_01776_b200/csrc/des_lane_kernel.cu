@@ -192,6 +192,17 @@ des_lane_kernel(const __grid_constant__ DesParams p)
         for (;;) {
             const uint32_t av_next = wm.avail[par ^ 1][lane];
             if (!done) {
+                // the record to hand on in this iteration (requested three iterations ago); its branch bits
+                // are fetched here, so that the load runs under the examine step
+                const bool h_valid = (vmask & 4u) != 0u;
+                uint32_t h_qid = 0, h_bits = 0;
+                uint64_t h_base = 0;
+                if (h_valid) {
+                    const uint32_t sl = (it + 1u) & (kStage - 1);
+                    h_qid = (uint32_t)wm.stage_e[sl][lane] & (uint32_t)qmask;
+                    h_base = wm.stage_b[sl][lane];
+                    if (BRANCHY && bit >= 0) h_bits = p.bits[h_qid];
+                }
                 const uint32_t written = av & ~kDone;
                 const bool pdone = (av & kDone) != 0u;
 
@@ -243,13 +254,10 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                 }
                 if (end && b == 0) lpos = tpos;     // stream exhausted: everything still held leaves, in key order
 
-                // ---- hand on the record requested three iterations ago
-                if (vmask & 4u) {
-                    const uint32_t sl = (it + 1u) & (kStage - 1);
-                    const uint32_t qid = (uint32_t)wm.stage_e[sl][lane] & (uint32_t)qmask;
-                    const uint64_t out = wm.stage_b[sl][lane] | qid;
-                    bool to_b = false;
-                    if (BRANCHY) to_b = bit >= 0 && ((p.bits[qid] >> bit) & 1);
+                // ---- hand on the record picked up at the top of the iteration
+                if (h_valid) {
+                    const uint64_t out = h_base | h_qid;
+                    const bool to_b = BRANCHY && bit >= 0 && ((h_bits >> bit) & 1u);
                     uint64_t *dst = to_b ? out_b + tail_b : out_a + tail_a;
                     *dst = out;
                     tail_b += to_b ? 1u : 0u;
