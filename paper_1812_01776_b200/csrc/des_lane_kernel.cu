@@ -203,6 +203,16 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                     h_base = wm.stage_b[sl][lane];
                     if (BRANCHY && bit >= 0) h_bits = p.bits[h_qid];
                 }
+                // likewise the next batch to hand on, if the one in hand is used up (a batch handed over in
+                // this iteration is picked up in the next), and the table entry a close would need
+                const bool f_valid = e_left == 0 && epos != lpos;
+                uint64_t f_key = 0;
+                uint32_t f_cnt = 0;
+                if (f_valid) {
+                    f_key = wm.key[epos & (kRing - 1)][lane];
+                    f_cnt = wm.cnt[epos & (kRing - 1)][lane];
+                }
+                const uint64_t latq = row[b > 0 ? b : 1];
                 const uint32_t written = av & ~kDone;
                 const bool pdone = (av & kDone) != 0u;
 
@@ -216,7 +226,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                 const bool room = tpos - epos < (uint32_t)kRing;
                 const bool close = b > 0 && !join && (known || end || b == mb) && room;
                 if (close) {
-                    const uint64_t key = (tk + row[b]) | head;
+                    const uint64_t key = (tk + latq) | head;
                     uint32_t pos = tpos;
                     if (tpos != lpos && key < ktail) {
                         // a batch that finishes before one dispatched earlier: sorted insert
@@ -264,11 +274,10 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                     tail_a += to_b ? 0u : 1u;
                 }
                 // ---- request the next record to hand on
-                if (e_left == 0 && epos != lpos) {
-                    const uint64_t k = wm.key[epos & (kRing - 1)][lane];
-                    e_left = wm.cnt[epos & (kRing - 1)][lane];
-                    e_base = k & ~qmask;
-                    e_idx = (uint32_t)k & (uint32_t)qmask;
+                if (f_valid) {
+                    e_left = f_cnt;
+                    e_base = f_key & ~qmask;
+                    e_idx = (uint32_t)f_key & (uint32_t)qmask;
                     epos++;
                 }
                 vmask = (vmask << 1) & 7u;
