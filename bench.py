@@ -45,7 +45,7 @@ WORKLOADS = {
 NCU_DRAM_BYTES_PER_QUERY_EVENT = {"des_packed_kernel": 12.24, "des_lane_kernel": 7.41}
 # Warp instructions executed per query-event (smsp__inst_executed.sum of the same captures): how many issue slots
 # the kernel spends, next to the algorithmic operation count of the roofline.
-NCU_WARP_INST_PER_QUERY_EVENT = {"des_packed_kernel": 32.9, "des_lane_kernel": 7.02}
+NCU_WARP_INST_PER_QUERY_EVENT = {"des_packed_kernel": 32.9, "des_lane_kernel": 7.08}
 METRIC = "candidate_configs_per_s"
 UNIT = "candidates/s"
 
