@@ -195,23 +195,16 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                 // the record to hand on in this iteration (requested three iterations ago); its branch bits
                 // are fetched here, so that the load runs under the examine step
                 const bool h_valid = (vmask & 4u) != 0u;
-                uint32_t h_qid = 0, h_bits = 0;
-                uint64_t h_base = 0;
-                if (h_valid) {
-                    const uint32_t sl = (it + 1u) & (kStage - 1);
-                    h_qid = (uint32_t)wm.stage_e[sl][lane] & (uint32_t)qmask;
-                    h_base = wm.stage_b[sl][lane];
-                    if (BRANCHY && bit >= 0) h_bits = p.bits[h_qid];
-                }
+                const uint32_t h_sl = (it + 1u) & (kStage - 1);
+                const uint32_t h_qid = (uint32_t)wm.stage_e[h_sl][lane] & (uint32_t)qmask;   // unused unless h_valid
+                const uint64_t h_base = wm.stage_b[h_sl][lane];
+                uint32_t h_bits = 0;
+                if (BRANCHY && h_valid && bit >= 0) h_bits = p.bits[h_qid];
                 // likewise the next batch to hand on, if the one in hand is used up (a batch handed over in
                 // this iteration is picked up in the next), and the table entry a close would need
                 const bool f_valid = e_left == 0 && epos != lpos;
-                uint64_t f_key = 0;
-                uint32_t f_cnt = 0;
-                if (f_valid) {
-                    f_key = wm.key[epos & (kRing - 1)][lane];
-                    f_cnt = wm.cnt[epos & (kRing - 1)][lane];
-                }
+                const uint64_t f_key = wm.key[epos & (kRing - 1)][lane];                      // unused unless f_valid
+                const uint32_t f_cnt = wm.cnt[epos & (kRing - 1)][lane];
                 const uint64_t latq = row[b > 0 ? b : 1];
                 const uint32_t written = av & ~kDone;
                 const bool pdone = (av & kDone) != 0u;
