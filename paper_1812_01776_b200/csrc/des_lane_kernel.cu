@@ -206,6 +206,8 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                 const uint64_t f_key = wm.key[epos & (kRing - 1)][lane];                      // unused unless f_valid
                 const uint32_t f_cnt = wm.cnt[epos & (kRing - 1)][lane];
                 const uint64_t latq = row[b > 0 ? b : 1];
+                // key of the second slot in use, the front after a hand-over (unused unless there are two)
+                uint64_t k2 = wm.key[(lpos + 1u) & (kRing - 1)][lane];
                 const uint32_t written = av & ~kDone;
                 const bool pdone = (av & kDone) != 0u;
 
@@ -236,7 +238,8 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                     }
                     wm.key[pos & (kRing - 1)][lane] = key;
                     wm.cnt[pos & (kRing - 1)][lane] = (uint32_t)b;
-                    kfront = pos == lpos ? key : kfront;
+                    if (pos == lpos) { k2 = kfront; kfront = key; }
+                    else if (pos == lpos + 1u) k2 = key;
                     tpos++;
                     nb++;
                     head = i;
@@ -250,7 +253,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                     if (tpos - lpos == R) {
                         kf = kfront;
                         lpos++;
-                        kfront = lpos != tpos ? wm.key[lpos & (kRing - 1)][lane] : kInf;
+                        kfront = lpos != tpos ? k2 : kInf;
                     }
                     tk = max(kf, ra) | qmask;
                     b = 1;
