@@ -220,44 +220,43 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                 b += join ? 1 : 0;
                 const bool room = tpos - epos < (uint32_t)kRing;
                 const bool close = b > 0 && !join && (known || end || b == mb) && room;
-                if (close) {
-                    const uint64_t key = (tk + latq) | head;
-                    uint32_t pos = tpos;
-                    if (tpos != lpos && key < ktail) {
-                        // a batch that finishes before one dispatched earlier: sorted insert
+                // close and open as straight-line code under predicates (only the sorted insert branches),
+                // so that the hand-on and request steps below can overlap with it
+                const uint64_t key = (tk + latq) | head;
+                uint32_t pos = tpos;
+                const bool sorted_insert = close && tpos != lpos && key < ktail;
+                if (sorted_insert) {
+                    // a batch that finishes before one dispatched earlier
 #pragma unroll 1
-                        while (pos != lpos) {
-                            const uint64_t prev = wm.key[(pos - 1) & (kRing - 1)][lane];
-                            if (prev <= key) break;
-                            wm.key[pos & (kRing - 1)][lane] = prev;
-                            wm.cnt[pos & (kRing - 1)][lane] = wm.cnt[(pos - 1) & (kRing - 1)][lane];
-                            pos--;
-                        }
-                    } else {
-                        ktail = key;
+                    while (pos != lpos) {
+                        const uint64_t prev = wm.key[(pos - 1) & (kRing - 1)][lane];
+                        if (prev <= key) break;
+                        wm.key[pos & (kRing - 1)][lane] = prev;
+                        wm.cnt[pos & (kRing - 1)][lane] = wm.cnt[(pos - 1) & (kRing - 1)][lane];
+                        pos--;
                     }
+                }
+                if (close) {
                     wm.key[pos & (kRing - 1)][lane] = key;
                     wm.cnt[pos & (kRing - 1)][lane] = (uint32_t)b;
-                    if (pos == lpos) { k2 = kfront; kfront = key; }
-                    else if (pos == lpos + 1u) k2 = key;
-                    tpos++;
-                    nb++;
-                    head = i;
-                    b = 0;
                 }
+                ktail = (close && !sorted_insert) ? key : ktail;
+                const bool at_front = close && pos == lpos;
+                k2 = at_front ? kfront : ((close && pos == lpos + 1u) ? key : k2);
+                kfront = at_front ? key : kfront;
+                tpos += close ? 1u : 0u;
+                nb += close ? 1u : 0u;
+                head = close ? i : head;
+                b = close ? 0 : b;
+                // record i opens the next batch on the replica that is free first: one that was never used
+                // (free from time 0) while there is one, else the slot with the smallest key
                 const bool open = known && !join && b == 0;
-                if (open) {
-                    // record i opens the next batch on the replica that is free first: one that was
-                    // never used (free from time 0) while there is one, else the slot with the smallest key
-                    uint64_t kf = 0;
-                    if (tpos - lpos == R) {
-                        kf = kfront;
-                        lpos++;
-                        kfront = lpos != tpos ? k2 : kInf;
-                    }
-                    tk = max(kf, ra) | qmask;
-                    b = 1;
-                }
+                const bool pop = open && tpos - lpos == R;
+                const uint64_t kf = pop ? kfront : 0ull;
+                lpos += pop ? 1u : 0u;
+                kfront = pop ? (lpos != tpos ? k2 : kInf) : kfront;
+                tk = open ? (max(kf, ra) | qmask) : tk;
+                b = open ? 1 : b;
                 if (end && b == 0) lpos = tpos;     // stream exhausted: everything still held leaves, in key order
 
                 // ---- hand on the record picked up at the top of the iteration
