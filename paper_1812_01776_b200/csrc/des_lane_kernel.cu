@@ -75,6 +75,9 @@ struct WarpMem {
     // sorted by key.
     uint64_t key[kRing][32];     // (finish << q) | index of the batch's first arrival
     uint32_t cnt[kRing][32];     // batch size
+    // The lane's row of the profile, [b - 1][lane]: time of a batch of b on the stage's hardware type.
+    // One copy per lane, so that lanes with different rows or batch sizes never meet in a bank.
+    uint32_t lat[IL_MAX_BATCH][32];
     // Staging rings filled by cp.async, [position][lane]: the next records of the lane's arrival stream
     // (position = record index mod kStage), and the records it is handing on with the finish << q of
     // their batch (position = iteration mod kStage)
@@ -96,14 +99,13 @@ __global__ void __launch_bounds__(kLaneWarps * 32)
 des_lane_kernel(const __grid_constant__ DesParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    // per table entry the 64-bit word (latency << q) - qmask: finish key base = dispatch key + that
-    uint64_t *s_latq = reinterpret_cast<uint64_t *>(smem_raw);
+    int32_t *s_lat = reinterpret_cast<int32_t *>(smem_raw);      // the profile tables, [S][H][Bmax]
     const int n_tab = p.S * p.H * p.Bmax;
-    WarpMem *wm_all = reinterpret_cast<WarpMem *>(smem_raw + ((size_t)n_tab * 8 + 15) / 16 * 16);
+    WarpMem *wm_all = reinterpret_cast<WarpMem *>(smem_raw + ((size_t)n_tab * 4 + 15) / 16 * 16);
     const int q = p.qbits;
     const uint64_t qmask = (1ull << q) - 1ull;
     for (int i = threadIdx.x; i < n_tab; i += blockDim.x)
-        s_latq[i] = ((uint64_t)(uint32_t)p.lat[i] << q) - qmask;
+        s_lat[i] = p.lat[i];
     __syncthreads();
 
     const unsigned full = 0xffffffffu;
@@ -158,7 +160,10 @@ des_lane_kernel(const __grid_constant__ DesParams p)
 
         const uint32_t R = cfg.replicas;
         const int mb = cfg.max_batch;
-        const uint64_t *row = s_latq + (s * p.H + cfg.hw) * p.Bmax - 1;   // row[b], b = 1..Bmax
+        if (live) {
+            const int32_t *row = s_lat + (s * p.H + cfg.hw) * p.Bmax;
+            for (int k = 0; k < p.Bmax; k++) wm.lat[k][lane] = (uint32_t)row[k];
+        }
         uint64_t *out_a = da < 0 ? slab + exit_off : my_block + p.lane_off[da];
         uint64_t *out_b = db < 0 ? slab + exit_off : my_block + p.lane_off[db];
 
@@ -205,7 +210,8 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                 const bool f_valid = e_left == 0 && epos != lpos;
                 const uint64_t f_key = wm.key[epos & (kRing - 1)][lane];                      // unused unless f_valid
                 const uint32_t f_cnt = wm.cnt[epos & (kRing - 1)][lane];
-                const uint64_t latq = row[b > 0 ? b : 1];
+                // (latency << q) - qmask: finish key base = dispatch key + that
+                const uint64_t latq = ((uint64_t)wm.lat[b > 0 ? b - 1 : 0][lane] << q) - qmask;
                 // key of the second slot in use, the front after a hand-over (unused unless there are two)
                 uint64_t k2 = wm.key[(lpos + 1u) & (kRing - 1)][lane];
                 const uint32_t written = av & ~kDone;
@@ -357,7 +363,7 @@ int des_lane_warps_per_cta() { return kLaneWarps; }
 
 size_t des_lane_smem(int n_tab)
 {
-    return ((size_t)n_tab * 8 + 15) / 16 * 16 + (size_t)kLaneWarps * sizeof(WarpMem);
+    return ((size_t)n_tab * 4 + 15) / 16 * 16 + (size_t)kLaneWarps * sizeof(WarpMem);
 }
 
 int des_lane_max_ctas_per_sm(size_t smem)
