@@ -276,7 +276,7 @@ IL_API int il_set_workspace(il_estimator *est, void *d_workspace, size_t bytes);
  * only IL_VARIANT_WIDE applies and every other choice falls back to it.
  *
  * IL_VARIANT_AUTO (default): the lane kernel when the inter-stage streams of one
- *   candidate take at most 16 MiB, else the packed warp-per-candidate kernel.
+ *   candidate take at most 128 MiB, else the packed warp-per-candidate kernel.
  * IL_VARIANT_LANES: one lane per (candidate, stage); the stages of a candidate
  *   run side by side as a pipeline inside one warp, floor(32 / S) candidates per
  *   warp.  Keeps every stage's arrival stream of every resident candidate in

@@ -82,10 +82,11 @@ struct Plan {
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // The lane kernel keeps every stage's whole arrival stream per resident candidate.  Beyond this many
-// bytes per candidate too few candidates fit the device at once and the warp-per-candidate kernel,
-// which needs two streams whatever the depth, is the faster one (measured on the 10-stage, 10^6-query
-// workload: 72 MB per candidate, 0.93x).
-constexpr int64_t kLaneAutoBytes = INT64_C(16) << 20;
+// bytes per candidate too few candidates fit the device at once, and the warp-per-candidate kernel,
+// which needs two streams whatever the depth, takes over.  (At 72 MB per candidate, the 10-stage,
+// 10^6-query workload, a 150 GB workspace still holds 1,700 candidates and the lane kernel is 1.7x the
+// faster one.)
+constexpr int64_t kLaneAutoBytes = INT64_C(128) << 20;
 // Resident CTAs (of two warps) per SM for the lane kernel.  Two warps per scheduler keep the issue
 // slots about as busy as more would, and every further warp lengthens all chains through the
 // shared-memory pipe: on B200, workload 2 with 16,384 candidates took 101.7 / 79.2 / 68.4 / 71.1 / 85.5 ms

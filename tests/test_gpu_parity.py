@@ -250,12 +250,13 @@ def test_config2_full_size_sampled(il, oracle, variant):
     assert (p99 > 0).all() and (miss >= 0).all() and (miss <= w.n_queries).all()
 
 
-def _sampled_check(il, oracle, w, n_sample, seed, extremes):
+def _sampled_check(il, oracle, w, n_sample, seed, extremes, variant=0):
     """Runs every candidate of w on the GPU (device entry point, torch-owned
     workspace as in the bench) and checks a seeded sample plus structured
     extremes against the oracle one by one, and size-free properties on all."""
     import torch
     with il.Estimator.from_workload(w) as est:
+        est.set_variant(variant)
         est.reserve_workspace(w.n_candidates)
         d = torch.from_numpy(w.configs).cuda()
         a, b = est.estimate_device(d, w.slo_us)
@@ -294,12 +295,14 @@ def test_config5_full_size_sampled(il, oracle):
     _sampled_check(il, oracle, w, 64, 5, _extremes(8, 4, (1, 64), (1, 32)))
 
 
-def test_config4_full_trace_candidate_subset(il, oracle):
+@pytest.mark.parametrize("variant", [0, 4], ids=["auto", "packed"])
+def test_config4_full_trace_candidate_subset(il, oracle, variant):
     """The 10-stage pipeline on the full 1,000,000-query trace.  The full sweep is
     262,144 candidates (2.6e12 query-events, minutes of GPU time); this test runs
-    the first 8,192 candidates of the same seeded draw and checks a sample."""
-    w = workloads.make(4, n_candidates=8192)
-    _sampled_check(il, oracle, w, 24, 4, _extremes(10, 4, (1, 64), (1, 16)))
+    the first 8,192 candidates of the same seeded draw (4,096 on the warp-per-candidate
+    kernel) and checks a sample."""
+    w = workloads.make(4, n_candidates=8192 if variant == 0 else 4096)
+    _sampled_check(il, oracle, w, 24, 4, _extremes(10, 4, (1, 64), (1, 16)), variant=variant)
 
 
 def test_kernel_choice(il):
@@ -318,7 +321,7 @@ def test_kernel_choice(il):
         assert est.kernel_name() == "des_kernel"
         est.set_variant(E.IL_VARIANT_LANES)
         assert est.kernel_name() == "des_kernel"
-    w = workloads.make(4, n_candidates=2)          # 9 x 10^6 stream records per candidate
+    w = workloads.make(4, n_queries=2_000_000, n_candidates=2)   # 18 x 10^6 stream records per candidate
     with il.Estimator.from_workload(w) as est:
         assert est.kernel_name() == "des_packed_kernel"
         est.set_variant(E.IL_VARIANT_LANES)
