@@ -42,10 +42,10 @@ WORKLOADS = {
 # DRAM bytes (read + write) of a simulation kernel per query-event, from an ncu capture of a reduced case
 # (1,024 candidates x 20,000 queries; traffic is proportional to the query-events processed).
 # An entry is None whenever its kernel has changed since the capture.
-NCU_DRAM_BYTES_PER_QUERY_EVENT = {"des_packed_kernel": 12.24, "des_lane_kernel": 7.41}
+NCU_DRAM_BYTES_PER_QUERY_EVENT = {"des_packed_kernel": 12.24, "des_lane_kernel": 7.37}
 # Warp instructions executed per query-event (smsp__inst_executed.sum of the same captures): how many issue slots
 # the kernel spends, next to the algorithmic operation count of the roofline.
-NCU_WARP_INST_PER_QUERY_EVENT = {"des_packed_kernel": 32.9, "des_lane_kernel": 7.08}
+NCU_WARP_INST_PER_QUERY_EVENT = {"des_packed_kernel": 32.9, "des_lane_kernel": 6.53}
 METRIC = "candidate_configs_per_s"
 UNIT = "candidates/s"
 
