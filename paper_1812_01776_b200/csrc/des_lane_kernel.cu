@@ -41,6 +41,14 @@
 // before its use; one commit group per iteration, at most two groups pending, so
 // that no instruction of the loop waits for global memory.
 //
+// With few candidates a warp has a scheduler to itself and is paced by its own
+// dependency chain, so the loop body is ordered for that: whatever the end of
+// an iteration needs from shared or global memory is loaded at its top,
+// unconditionally, and the close / open steps are straight-line code under
+// predicates, so that independent work can issue while a dependent value is on
+// its way.  Each lane keeps its own copy of its stage's profile row in shared
+// memory, [batch][lane], so that table look-ups never conflict.
+//
 // Records and keys are the packed 64-bit words of des_packed_kernel.cu:
 // (time << q) | query for stream records, (finish << q) | index of the batch's
 // first arrival for replica slots, whose unsigned order is (finish, dispatch
