@@ -606,6 +606,19 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
         SelectParams sp;
         sp.slab = p.slab; sp.slab_stride = e->n_pad; sp.lat_or = p.lat_or;
         sp.arrival = e->d_arrival; sp.qbits = p.qbits; sp.packed = use_packed(e) ? 1 : 0;
+        sp.n_regions = 0;
+        if (lane) {   // where each stage's leaving queries end in a slab row (the lane kernel's layout)
+            int32_t off = 0;
+            for (int s = 0; s < e->S; s++) {
+                const int a = e->base.dest_a[s], b = e->base.dest_b[s];
+                int32_t kids = 0;
+                if (a >= 0) kids += e->base.n_s[a];
+                if (b >= 0 && b != a) kids += e->base.n_s[b];
+                const int32_t leaving = e->base.n_s[s] - kids;
+                off += leaving;
+                if (leaving > 0) sp.region_end[sp.n_regions++] = off;
+            }
+        }
         sp.n = (int32_t)e->n; sp.n_cand = cnt; sp.slo_us = slo_us;
         sp.out_p99 = d_out_p99 + lo; sp.out_miss = d_out_miss + lo;
         IL_CUDA(launch_select(sp, st));

@@ -34,7 +34,7 @@ struct DesParams {
     int32_t *ws_qid;              // [slots][slot_elems]
     int64_t *slab;                // [n_cand][slab_stride] exit latencies
     int64_t slab_stride;          // n rounded up to 32
-    uint64_t *lat_or;             // [n_cand] OR of all latencies of the candidate
+    uint64_t *lat_or;             // [n_cand] OR of all latencies of the candidate (wide kernel)
     unsigned long long *counters; // [0] next candidate, [1] batches dispatched, [2] algorithmic ops
     int *status;                  // first error seen by any warp (0 = none)
     // lane-parallel kernel only (des_lane_kernel.cu)
@@ -49,8 +49,12 @@ struct SelectParams {
     int64_t slab_stride;
     const int64_t *arrival;       // [n], to turn packed records into latencies
     int32_t qbits;
-    int32_t packed;               // slab holds packed records (from the packed simulation kernel)
-    const uint64_t *lat_or;       // [n_cand]
+    int32_t packed;               // slab holds packed records (from a packed-record simulation kernel)
+    // Packed slabs of the lane kernel: the queries that leave after stage s fill one region of the row,
+    // in finish order, so the last record of each region carries that region's largest finish time.
+    int32_t n_regions;            // 0: not known
+    int32_t region_end[IL_MAX_STAGES];   // one past the last record of each non-empty region
+    const uint64_t *lat_or;       // [n_cand]: OR of the latencies (wide kernel)
     int32_t n;
     int64_t n_cand;
     int64_t slo_us;

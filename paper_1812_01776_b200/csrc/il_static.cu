@@ -102,6 +102,7 @@ extern "C" int il_estimate_device_static(il_estimator *est, const il_stage_confi
     SelectParams sp;
     sp.slab = p.slab; sp.slab_stride = v.n_pad; sp.lat_or = p.lat_or;
     sp.arrival = p.arrival; sp.qbits = p.qbits; sp.packed = v.kernel != kSimWide ? 1 : 0;
+    sp.n_regions = 0;
     sp.n = (int32_t)v.n; sp.n_cand = n_cand; sp.slo_us = slo_us;
     sp.out_p99 = d_out_p99; sp.out_miss = d_out_miss;
     if (launch_select(sp, st) != cudaSuccess) return IL_ERR_CUDA;

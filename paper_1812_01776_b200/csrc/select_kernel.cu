@@ -9,9 +9,16 @@
 // highest set bit of any latency (known from the simulation kernel's OR) are
 // skipped.  One CTA per candidate.
 //
-// When the slab comes from the packed-record simulation kernel it holds
+// When the slab comes from a packed-record simulation kernel it holds
 // (finish time, query) records; a first sweep replaces each by
 // latency = finish - arrival[query], ORs the latencies and counts the misses.
+// When the slab's regions are known (lane kernel: one region per stage that
+// queries leave after, each in finish order), the last record of each region
+// gives the candidate's largest finish time, and largest finish - first arrival
+// bounds every latency before the sweep: if that is below 2^32 the sweep writes 32-bit latencies (into the front
+// half of the row; one barrier per 256 records keeps the writes behind the
+// reads) and histograms the top digit on the way, and the remaining passes read
+// half the bytes.
 #include "il_internal.h"
 
 namespace il {
@@ -30,6 +37,76 @@ select_kernel(const __grid_constant__ SelectParams p)
         unsigned miss = 0;
         bool counted_miss = false;
         uint64_t bits_used;
+        if (p.packed && p.n_regions > 0) {
+            uint64_t last = 0;
+#pragma unroll
+            for (int r = 0; r < IL_MAX_STAGES; r++)      // unrolled: constant indices into the parameter block
+                if (r < p.n_regions) last = max(last, (uint64_t)lat[p.region_end[r] - 1] >> p.qbits);
+            const int64_t bound64 = (int64_t)last - p.arrival[0];
+            if (bound64 < (INT64_C(1) << 32)) {
+                const uint32_t bound = bound64 > 0 ? (uint32_t)bound64 : 0u;
+                int top32 = 0;
+                while (top32 < 4 && (bound >> (8 * top32)) != 0) top32++;
+                hist[threadIdx.x] = 0;
+                if (threadIdx.x == 0) {
+                    s_prefix = 0;
+                    s_rank = (unsigned)((99ll * p.n + 99) / 100);
+                    s_miss = 0;
+                }
+                __syncthreads();
+                uint32_t *lat32 = reinterpret_cast<uint32_t *>(lat);
+                const uint64_t qmask = (1ull << p.qbits) - 1ull;
+                const int sh_top = top32 > 0 ? 8 * (top32 - 1) : 0;
+                for (int base = 0; base < p.n; base += kSelectThreads) {
+                    const int i = base + (int)threadIdx.x;
+                    uint32_t l = 0;
+                    if (i < p.n) {
+                        const uint64_t rec = (uint64_t)lat[i];
+                        l = (uint32_t)((int64_t)(rec >> p.qbits) - p.arrival[rec & qmask]);
+                        miss += ((int64_t)l > p.slo_us);
+                    }
+                    __syncthreads();        // all records of this block are read before their row space is reused
+                    if (i < p.n) {
+                        lat32[i] = l;
+                        atomicAdd(&hist[(l >> sh_top) & 0xff], 1u);
+                    }
+                }
+                __syncthreads();
+                for (int d = top32 - 1; d >= 0; d--) {
+                    const int shift = 8 * d;
+                    if (d != top32 - 1) {
+                        hist[threadIdx.x] = 0;
+                        __syncthreads();
+                        const uint32_t prefix = (uint32_t)s_prefix;
+                        const uint32_t himask = ~0u << (shift + 8);     // d <= 2 here
+                        for (int i = threadIdx.x; i < p.n; i += kSelectThreads) {
+                            const uint32_t v = lat32[i];
+                            if ((v & himask) == prefix) atomicAdd(&hist[(v >> shift) & 0xff], 1u);
+                        }
+                        __syncthreads();
+                    }
+                    if (threadIdx.x == 0) {
+                        unsigned r = s_rank, acc = 0;
+                        int b = 0;
+                        for (; b < 255; b++) {
+                            if (acc + hist[b] >= r) break;
+                            acc += hist[b];
+                        }
+                        s_rank = r - acc;
+                        s_prefix = s_prefix | ((unsigned long long)b << shift);
+                    }
+                    __syncthreads();
+                }
+                if (miss) atomicAdd(&s_miss, miss);
+                __syncthreads();
+                if (threadIdx.x == 0) {
+                    p.out_p99[c] = (int64_t)s_prefix;
+                    p.out_miss[c] = (int64_t)s_miss;
+                }
+                __syncthreads();
+                continue;
+            }
+        }
         if (p.packed) {
             if (threadIdx.x == 0) s_or = 0;
             __syncthreads();
