@@ -221,15 +221,19 @@ IL_API int il_traffic_envelope(il_estimator *est, const int64_t *window_us, int3
  * Arguments and results are those of il_estimate_device (DEVICE pointers,
  * work on the handle's stream, returns after completion, same values bit for
  * bit).  A workspace set with il_set_workspace is ignored, and il_get_stats is
- * not updated.
+ * not updated.  The call runs on the handle's device and leaves the caller's
+ * current device as it found it; after an error it has still waited for whatever
+ * it had enqueued, and il_last_cuda_error names the failing CUDA call.
  *
  * Limit: the whole batch is evaluated in one pass, with at most 32 warps
  * resident, and must fit the array:
- *     256 + 12 * slot * min(32, n rounded up to 4) + (8 * n_queries' + 12) * n
+ *     256 + r * slot * min(32, n rounded up to 4) + (8 * n_queries' + 12) * n
  *         <= IL_STATIC_SCRATCH_BYTES
- * where n_queries' is n_queries rounded up to 32 and slot is the number of
+ * where n_queries' is n_queries rounded up to 32, slot is the number of
  * stream elements one warp keeps between stages (for a linear pipeline about
- * 2 * n_queries; never more than the query-events per candidate).  A larger
+ * 2 * n_queries; never more than the query-events per candidate), and r is 8
+ * bytes per element (12 when the times are too large for packed records, see
+ * il_set_variant, or IL_VARIANT_WIDE is set).  A larger
  * request returns IL_ERR_TOO_LARGE and launches nothing; split the batch or use
  * il_estimate_device.
  *

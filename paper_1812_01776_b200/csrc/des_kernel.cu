@@ -228,6 +228,8 @@ des_kernel(const __grid_constant__ DesParams p)
 
 cudaError_t launch_des(const DesParams &p, int grid, size_t smem, cudaStream_t stream)
 {
+    cudaError_t e = cudaFuncSetAttribute(des_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
     des_kernel<<<grid, kWarpsPerCta * 32, smem, stream>>>(p);
     return cudaGetLastError();
 }
@@ -235,6 +237,8 @@ cudaError_t launch_des(const DesParams &p, int grid, size_t smem, cudaStream_t s
 int des_max_ctas_per_sm(size_t smem)
 {
     int n = 0;
+    if (cudaFuncSetAttribute(des_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, des_kernel, kWarpsPerCta * 32, smem) != cudaSuccess)
         return 0;
     return n;

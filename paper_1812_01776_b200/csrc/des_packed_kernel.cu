@@ -965,8 +965,21 @@ des_packed_kernel(const __grid_constant__ DesParams p)
     if (lane == 0 && batches) { atomicAdd(&p.counters[1], batches); atomicAdd(&p.counters[2], alg_ops); }
 }
 
+namespace {
+// Static plus dynamic shared memory passes 48 KB for the largest table shapes the interface takes
+// (16 stages x 8 hardware types x 64 batch sizes = 32 KB of tables): opt in before every use.
+cudaError_t packed_opt_in(bool staged, size_t smem)
+{
+    return staged
+        ? cudaFuncSetAttribute(des_packed_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+        : cudaFuncSetAttribute(des_packed_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+}
+}  // namespace
+
 cudaError_t launch_des_packed(const DesParams &p, bool staged, int grid, size_t smem, cudaStream_t stream)
 {
+    cudaError_t e = packed_opt_in(staged, smem);
+    if (e != cudaSuccess) return e;
     if (staged) des_packed_kernel<true><<<grid, kWarpsPerCta * 32, smem, stream>>>(p);
     else des_packed_kernel<false><<<grid, kWarpsPerCta * 32, smem, stream>>>(p);
     return cudaGetLastError();
@@ -975,6 +988,7 @@ cudaError_t launch_des_packed(const DesParams &p, bool staged, int grid, size_t 
 int des_packed_max_ctas_per_sm(bool staged, size_t smem)
 {
     int n = 0;
+    if (packed_opt_in(staged, smem) != cudaSuccess) return 0;
     cudaError_t e = staged
         ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, des_packed_kernel<true>, kWarpsPerCta * 32, smem)
         : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, des_packed_kernel<false>, kWarpsPerCta * 32, smem);

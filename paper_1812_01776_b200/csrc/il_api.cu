@@ -266,6 +266,8 @@ int ensure_events(il_estimator *e, size_t count)
 
 }  // namespace
 
+void il::set_last_cuda_error(int cuda_error) { g_last_cuda_error = cuda_error; }
+
 void il::bound_view(const il_estimator *e, BoundView *out)
 {
     out->base = e->base;
@@ -459,8 +461,10 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     e->smem_lane = des_lane_smem(S * H * B);
     e->ctas_per_sm_lane = std::min(des_lane_max_ctas_per_sm(e->smem_lane), kLaneCtasPerSm);
     if (e->ctas_per_sm_wide < 1 || e->ctas_per_sm_packed < 1 || e->ctas_per_sm_staged < 1 ||
-        e->ctas_per_sm_lane < 1)
+        e->ctas_per_sm_lane < 1) {
+        g_last_cuda_error = (int)cudaErrorLaunchOutOfResources;
         return fail(IL_ERR_CUDA);
+    }
     e->ctas_per_sm = ctas_for(e);
     *out = e;
     return IL_OK;
@@ -756,13 +760,13 @@ int il_measure_int_issue(void *cuda_stream, double *out_warp_inst_per_s, double 
     IL_CUDA(cudaGetDevice(&dev));
     IL_CUDA(cudaGetDeviceProperties(&prop, dev));
     unsigned *sink = nullptr;
-    IL_CUDA(cudaMalloc(&sink, sizeof(unsigned)));
-    cudaEvent_t a, b;
-    IL_CUDA(cudaEventCreate(&a));
-    IL_CUDA(cudaEventCreate(&b));
+    cudaEvent_t a = nullptr, b = nullptr;
+    cudaError_t ce = cudaMalloc(&sink, sizeof(unsigned));
+    if (ce == cudaSuccess) ce = cudaEventCreate(&a);
+    if (ce == cudaSuccess) ce = cudaEventCreate(&b);
     const int grid = prop.multiProcessorCount * 8;   // 8 CTAs of 8 warps per SM
     const int iters = 4096;
-    cudaError_t ce = launch_int_issue(sink, grid, 64, st);   // warm-up
+    if (ce == cudaSuccess) ce = launch_int_issue(sink, grid, 64, st);   // warm-up
     float best = 1e30f;
     for (int rep = 0; rep < 3 && ce == cudaSuccess; rep++) {
         cudaEventRecord(a, st);
@@ -773,7 +777,9 @@ int il_measure_int_issue(void *cuda_stream, double *out_warp_inst_per_s, double 
         if (ce == cudaSuccess) ce = cudaEventElapsedTime(&ms, a, b);
         best = std::min(best, ms);
     }
-    cudaEventDestroy(a); cudaEventDestroy(b); cudaFree(sink);
+    if (a) cudaEventDestroy(a);
+    if (b) cudaEventDestroy(b);
+    cudaFree(sink);
     if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return IL_ERR_CUDA; }
     // per inner step: 4 multiply-adds + 4 x (xor, add) = 12 instructions per thread
     const double inst = (double)grid * 8.0 * iters * 16.0 * 12.0;

@@ -75,6 +75,8 @@ struct BoundView {
     cudaStream_t stream;
 };
 void bound_view(const il_estimator *est, BoundView *out);
+// Records a failing CUDA call for il_last_cuda_error (thread-local).
+void set_last_cuda_error(int cuda_error);
 
 cudaError_t launch_des(const DesParams &p, int grid, size_t smem, cudaStream_t stream);
 // staged: the root stage reads the trace through a shared-memory tile ring filled by bulk copies

@@ -17,3 +17,12 @@ def oracle():
     import oracle as _oracle
     _oracle.build()
     return _oracle
+
+
+@pytest.fixture(scope="session")
+def oracle_pool(oracle):
+    """Worker processes (spawn start method, so a CUDA context in the parent is
+    no obstacle) that each run the single-threaded oracle on a slice of candidates."""
+    pool = oracle.make_pool()
+    yield pool
+    pool.terminate()

@@ -472,3 +472,22 @@ def test_rejects_bad_inputs(oracle):
         bad = w.configs[0].copy(); bad[1, col] = val
         assert code(config=bad) == -5
     assert code(branch_bits=None) == -1
+
+
+def test_grouped_arrivals_give_the_constructed_latency_multiset(oracle):
+    """Simultaneous groups of b queries, spaced apart, one replica, max batch 64: each group is one
+    batch of b at every stage, so every query of it has latency sum_s table[s][b].  The oracle must
+    reproduce that vector, and its P99 / miss must equal numpy's sort of it (rank ceil(0.99 n))."""
+    from select_cases import SELECT_CASES, grouped_workload
+    for case, (sizes, by_size, S) in SELECT_CASES.items():
+        w, want = grouped_workload(sizes, by_size, S)
+        n = want.shape[0]
+        k = (99 * n + 99) // 100
+        srt = np.sort(want)
+        _, _, lat = oracle.estimate_one(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us,
+                                        w.branch_bits, w.configs[0], 0, want_latency=True)
+        assert np.array_equal(lat, want), case
+        for slo in (int(srt[0]) - 1, int(srt[k - 1]), int(srt[-1])):
+            w.slo_us = slo
+            p99, miss = oracle.estimate_workload(w)
+            assert (int(p99[0]), int(miss[0])) == (int(srt[k - 1]), int((want > slo).sum())), (case, slo)

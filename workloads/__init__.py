@@ -311,6 +311,19 @@ def make(config_id: int, n_queries: Optional[int] = None,
                     slo_us=slo, recipe=recipe)
 
 
+def sub_batch(config_id: int, size: int, seed: int = 0, n_queries: Optional[int] = None):
+    """A seeded sample of ``size`` distinct candidates of workload ``config_id``,
+    drawn from its WHOLE candidate set (not a prefix of it), in increasing
+    candidate order.  Returns the workload restricted to the sample and the
+    sampled candidate indices."""
+    w = make(config_id, n_queries=n_queries)
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([BASE_SEED, config_id, 7, seed])))
+    idx = np.sort(rng.choice(w.n_candidates, size=min(size, w.n_candidates), replace=False))
+    w.configs = np.ascontiguousarray(w.configs[idx])
+    w.recipe.update(sub_batch=dict(size=int(idx.shape[0]), seed=seed))
+    return w, idx
+
+
 def random_small(seed: int, S: int = 3, H: int = 2, Bmax: int = 8, n: int = 200,
                  C: int = 16, max_replicas: int = 4, tree: bool = False,
                  qps: float = 200.0, cv: float = 2.0, lat_lo: int = 1, lat_hi: int = 20000,
