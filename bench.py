@@ -2,15 +2,17 @@
 """Benchmark of the batched Estimator: candidate configurations evaluated per second.
 
 One step = one pass of the whole hot path (simulation kernel + percentile
-kernel) over one batch of candidates of the image-pipeline workload
-(4 stages, 50,000 gamma arrivals at 200 qps with CV 4, 4,096 candidates).
+kernel) over one batch of candidates.  The headline workload is the largest
+one: the 10-stage pipeline on its full 1,000,000-query trace with a seeded
+16,384-candidate sample of its 262,144 candidates (drawn from the whole set).
+The same JSON line carries, under "per_workload", a short measurement of each
+of the other four workloads at full size.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
-With N > 1 (under torchrun) every rank evaluates its own 4,096-candidate slice
-of an N x 4,096 seeded candidate set against the same trace; there is no
-data-path collective, only a barrier and a max over ranks of the timings.
-Prints one JSON line on rank 0.
+With N > 1 (under torchrun) every rank evaluates its own seeded 16,384-candidate
+sample against the same trace; there is no data-path collective, only a barrier
+and a max over ranks of the timings.  Prints one JSON line on rank 0.
 """
 from __future__ import annotations
 
@@ -31,7 +33,8 @@ if ROOT not in sys.path:
 
 import workloads  # noqa: E402
 
-WORKLOAD_ID = 2          # the benchmark workload; --workload picks another one for side measurements
+WORKLOAD_ID = 4          # the headline workload (the largest); --workload picks another one
+SUB_BATCH = {4: 16384}   # workloads timed on a seeded sample of their candidates (full sweep: --candidates 0)
 WORKLOADS = {
     1: "config1: linear 2-stage pipeline, 2,000 Poisson arrivals (100 qps), 64 candidates",
     2: "config2: linear 4-stage image pipeline, 50,000 gamma arrivals (200 qps, CV 4), 4,096 candidates",
@@ -39,13 +42,21 @@ WORKLOADS = {
     4: "config4: linear 10-stage pipeline, 1,000,000 arrivals ramping 150->250 qps, 262,144 candidates",
     5: "config5: 8-stage tree with three branch points, 100,000 gamma arrivals (500 qps, CV 2), 1,048,576 candidates",
 }
-# DRAM bytes (read + write) of a simulation kernel per query-event, from an ncu capture of a reduced case
-# (1,024 candidates x 20,000 queries; traffic is proportional to the query-events processed).
-# An entry is None whenever its kernel has changed since the capture.
-NCU_DRAM_BYTES_PER_QUERY_EVENT = {"des_packed_kernel": 12.24, "des_lane_kernel": 7.37}
-# Warp instructions executed per query-event (smsp__inst_executed.sum of the same captures): how many issue slots
-# the kernel spends, next to the algorithmic operation count of the roofline.
-NCU_WARP_INST_PER_QUERY_EVENT = {"des_packed_kernel": 32.9, "des_lane_kernel": 6.53}
+# Counters of the simulation kernels from ncu captures of a reduced case (traffic and instructions grow in
+# proportion to the query-events processed).  Each entry names the SHA-256 of the kernel source it was taken
+# from; when the source in the tree differs, the figures that depend on the capture are reported as null.
+NCU_CAPTURES = {
+    "des_lane_kernel": {
+        "source": "paper_1812_01776_b200/csrc/des_lane_kernel.cu",
+        "source_sha256": "",
+        "dram_bytes_per_query_event": 7.37, "warp_inst_per_query_event": 6.53,
+        "summary": "profiles/des_lane_kernel_config2.md"},
+    "des_packed_kernel": {
+        "source": "paper_1812_01776_b200/csrc/des_packed_kernel.cu",
+        "source_sha256": "",
+        "dram_bytes_per_query_event": 12.24, "warp_inst_per_query_event": 32.9,
+        "summary": "profiles/des_packed_kernel_config2.md"},
+}
 METRIC = "candidate_configs_per_s"
 UNIT = "candidates/s"
 
@@ -54,11 +65,7 @@ UNIT = "candidates/s"
 # helpers that hold no GPU work (covered by CPU tests)
 # ----------------------------------------------------------------------------
 
-def shard_range(total: int, rank: int, world: int):
-    """Contiguous slice [lo, hi) of `total` units owned by `rank`."""
-    base, rem = divmod(total, world)
-    lo = rank * base + min(rank, rem)
-    return lo, lo + base + (1 if rank < rem else 0)
+from paper_1812_01776_b200.sharded import shard_range  # noqa: E402  (the package's sharding rule)
 
 
 def dist_env():
@@ -85,6 +92,36 @@ def reduce_sum(values, dist=None, device=None):
     t = torch.tensor(list(values), dtype=torch.float64, device=device or "cpu")
     dist.all_reduce(t, op=dist.ReduceOp.SUM)
     return t.tolist()
+
+
+def ncu_capture(kernel: str):
+    """The capture record of `kernel` if it still describes the source in the tree, else None."""
+    import hashlib
+    cap = NCU_CAPTURES.get(kernel.split("<")[0])
+    if not cap:
+        return None
+    try:
+        with open(os.path.join(ROOT, cap["source"]), "rb") as f:
+            now = hashlib.sha256(f.read()).hexdigest()
+    except OSError:
+        return None
+    return cap if now == cap["source_sha256"] else None
+
+
+def load_workload(workload_id: int, candidates, queries, seed: int = 0):
+    """The workload a step runs on and the text that names it.  candidates: None = the default
+    (a seeded sample for the workloads listed in SUB_BATCH, else the full set), 0 = the full set."""
+    full_n, full_c = workloads.FULL_SIZES[workload_id]
+    if candidates is None and queries is None and workload_id in SUB_BATCH:
+        w, _ = workloads.sub_batch(workload_id, SUB_BATCH[workload_id], seed=seed)
+        text = (f"{WORKLOADS[workload_id]}; timed on a seeded sample of {w.n_candidates:,} candidates "
+                f"drawn from the whole set, full {w.n_queries:,}-query trace")
+        return w, text
+    w = workloads.make(workload_id, n_queries=queries, n_candidates=candidates or None)
+    text = WORKLOADS[workload_id]
+    if w.n_candidates != full_c or w.n_queries != full_n:
+        text += f" [overridden: first {w.n_candidates:,} candidates, {w.n_queries:,} queries]"
+    return w, text
 
 
 def load_measured_peaks():
@@ -171,15 +208,23 @@ def time_oracle(w, n_sample: int, processes: int, pool=None):
     return time.perf_counter() - t0
 
 
+def oracle_sample(w, cores: int, seconds: float = 12.0):
+    """How many candidates of w the oracle is timed on per step: about `seconds` of work on
+    `cores` cores (it does a few million query-events per second and core), at least one per core."""
+    per_cand_s = w.query_events() / 4.5e6
+    return int(max(cores, min(w.n_candidates, seconds * cores / per_cand_s)))
+
+
 def run_reference(args):
+    """The oracle, as it stands, on the host cores: the same workload, metric and unit as the CUDA
+    arm; each step is the first oracle_sample() candidates of the batch the CUDA arm times."""
     rank, world, _ = dist_env()
     if rank != 0:
         return
-    w = workloads.make(args.workload, n_queries=args.queries,
-                       n_candidates=min(args.candidates or 10**9, 4096, workloads.FULL_SIZES[args.workload][1]))
+    w, text = load_workload(args.workload, args.candidates, args.queries)
     cores = os.cpu_count() or 1
     import oracle
-    per_step = max(cores, min(w.n_candidates, 8 * cores))
+    per_step = oracle_sample(w, cores, seconds=6.0)
     pool = oracle.make_pool(cores) if cores > 1 else None
     for _ in range(min(args.warmup, 1)):
         time_oracle(w, cores, cores, pool)
@@ -188,7 +233,7 @@ def run_reference(args):
         pool.terminate()
     sec = sum(times) / len(times)
     value = per_step / sec
-    sample = (f"first {per_step} of {workloads.FULL_SIZES[args.workload][1]} candidates per step, "
+    sample = (f"first {per_step} of the {w.n_candidates} candidates of the batch per step, "
               f"{w.n_queries}-query trace, "
               f"{cores} processes each running the single-threaded oracle on a disjoint slice")
     line = {
@@ -196,7 +241,7 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
         "data": "synthetic",
-        "config": {"workload": WORKLOADS[args.workload], "sampled_candidates_per_step": per_step},
+        "config": workload_config(w, text, world),
         "query_events_per_s": value * w.query_events(),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -205,50 +250,36 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def workload_config(w, text: str, world: int):
+    """The `config` object: names the workload only, so that both arms print the same one."""
+    return {"workload": text + (" per GPU" if world > 1 else ""),
+            "candidates_per_gpu": w.n_candidates, "queries": w.n_queries, "stages": w.n_stages,
+            "query_events_per_candidate": w.query_events(),
+            "l2": "256 MiB buffer written between steps (L2 is 126 MB)",
+            "parallelism": f"candidates sharded over {world} GPU(s), no data-path collective"}
+
+
 # ----------------------------------------------------------------------------
 # the CUDA arm
 # ----------------------------------------------------------------------------
 
-def run_cuda(args):
-    import torch
-    import torch.distributed as dist
-    import paper_1812_01776_b200 as il
-
-    rank, world, local = dist_env()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the Estimator")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-
-    per_rank = args.candidates or workloads.FULL_SIZES[args.workload][1]
-    w = workloads.make(args.workload, n_queries=args.queries, n_candidates=per_rank * world)
-    lo, hi = shard_range(w.n_candidates, rank, world)
-    cfg_host = np.ascontiguousarray(w.configs[lo:hi])
-    n_cand = hi - lo
+def measure(il, torch, w, dev, stream, flush, steps, warmup, e2e_steps, variant, issue_rate, peaks,
+            barrier=lambda: None, sampler=None):
+    """Times `steps` device-resident steps (after `warmup`) and `e2e_steps` host-buffer steps of
+    workload w on this rank's GPU.  Returns the per-workload record; times are per-rank."""
+    n_cand = w.n_candidates
+    cfg_host = np.ascontiguousarray(w.configs)
     events_per_cand = w.query_events()
-
-    est = il.Estimator.from_workload(w, device=local)
-    est.set_variant(args.variant)
+    est = il.Estimator.from_workload(w, device=dev.index)
+    est.set_variant(variant)
     kernel = est.kernel_name()
     ws_bytes = est.reserve_workspace(n_cand)
-    stream = torch.cuda.Stream(device=dev)
-    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)   # > 126 MB of L2
     cfg_pinned = torch.from_numpy(cfg_host).pin_memory()
-    out_pinned = torch.empty((2, n_cand), dtype=torch.int64).pin_memory()
-
     with torch.cuda.stream(stream):
         est.use_current_stream()
         d_cfg = cfg_pinned.to(dev, non_blocking=True)
         d_p99 = torch.empty(n_cand, dtype=torch.int64, device=dev)
         d_miss = torch.empty(n_cand, dtype=torch.int64, device=dev)
-
-        def barrier():
-            torch.cuda.synchronize(dev)
-            if world > 1:
-                dist.barrier()
-            torch.cuda.synchronize(dev)
 
         def one_step():
             """Device-resident step, timed on the library's stream; returns ms and stats."""
@@ -271,99 +302,175 @@ def run_cuda(args):
             b.synchronize()
             return a.elapsed_time(b), p99, miss
 
-        for _ in range(args.warmup):
+        for _ in range(warmup):
             one_step()
         barrier()
-        sampler = ClockSampler(local)
-        if rank == 0:
+        if sampler is not None:
             sampler.start()
-        step_ms, sim_ms, sel_ms, launches, batches, alg_ops = [], [], [], 0, 0, 0
-        for _ in range(args.steps):
+        step_ms, sim_ms, sel_ms, launches = [], [], [], 0
+        st = {}
+        for _ in range(steps):
             ms, st = one_step()
             step_ms.append(ms); sim_ms.append(st["sim_ms"]); sel_ms.append(st["select_ms"])
-            launches += st["kernel_launches"]; batches = st["batches"]; alg_ops = st["algorithmic_ops"]
+            launches += st["kernel_launches"]
         barrier()
-        clocks = sampler.stop() if rank == 0 else {}
-        total_ms = sum(step_ms)
-
-        # end to end through host buffers
+        clocks = sampler.stop() if sampler is not None else None
         one_step_e2e()
         barrier()
         e2e_ms = []
-        for _ in range(1 if args.no_e2e else args.steps):
+        p99_h = miss_h = None
+        for _ in range(e2e_steps):
             ms, p99_h, miss_h = one_step_e2e()
             e2e_ms.append(ms)
         barrier()
-        e2e_total = sum(e2e_ms)
         same = bool(np.array_equal(p99_h, d_p99.cpu().numpy()) and np.array_equal(miss_h, d_miss.cpu().numpy()))
         feasible = float((p99_h <= w.slo_us).mean())
+    est.close()
 
-        issue_rate, _ = il.il_measure_int_issue(stream.cuda_stream)
+    n, S = w.n_queries, w.n_stages
+    sim_s = statistics.mean(sim_ms) * 1e-3
+    sel_s = statistics.mean(sel_ms) * 1e-3
+    total_events = events_per_cand * n_cand
+    rec_bytes = 12 if kernel == "des_kernel" else 8  # separate time/query streams, else one 64-bit record
+    slab_bytes = 8 * n * n_cand                       # written once by the simulation, read once by the select
+    stream_bytes = (events_per_cand - n) * 2 * rec_bytes * n_cand   # written once, read once
+    cap = ncu_capture(kernel)
+    alu_peak = issue_rate * 32.0
+    rec = {
+        "candidates": n_cand, "queries": n, "stages": S, "query_events_per_candidate": events_per_cand,
+        "kernel": kernel, "workspace_bytes": ws_bytes, "steps": steps, "warmup": warmup,
+        "ms_per_step": {"mean": statistics.mean(step_ms), "median": statistics.median(step_ms),
+                        "best": min(step_ms)},
+        "step_ms_sum": sum(step_ms), "e2e_ms_sum": sum(e2e_ms), "e2e_steps": e2e_steps,
+        "candidates_per_s": n_cand / (statistics.mean(step_ms) * 1e-3),
+        "candidates_per_s_best": n_cand / (min(step_ms) * 1e-3),
+        "query_events_per_s": total_events / (statistics.mean(step_ms) * 1e-3),
+        "batches": st.get("batches"), "mean_batch": total_events / st["batches"] if st.get("batches") else None,
+        "stage_runs_simulated": st.get("stage_runs"), "stage_runs_of_the_method": n_cand * S,
+        "feasible_fraction": feasible,
+        "kernel_ms": {"simulate": statistics.mean(sim_ms), "select": statistics.mean(sel_ms)},
+        "gpu_launches": int(launches),
+        "e2e": {"candidates_per_s": n_cand * e2e_steps / (sum(e2e_ms) * 1e-3),
+                "h2d_bytes_per_step": int(cfg_host.nbytes), "d2h_bytes_per_step": int(16 * n_cand),
+                "matches_device_path": same},
+        "roofline": {"bound": "alu", "achieved": st["algorithmic_ops"] / sim_s / 1e12, "peak": alu_peak / 1e12,
+                     "unit": "Tinteger-op/s", "frac": st["algorithmic_ops"] / sim_s / alu_peak,
+                     "traffic": cap["dram_bytes_per_query_event"] * total_events if cap else None,
+                     "traffic_unit": "DRAM bytes per launch (ncu capture of a reduced case, scaled by query-events)",
+                     "capture": ({"summary": cap["summary"], "source_sha256": cap["source_sha256"]} if cap else
+                                 "none that matches the kernel source in the tree"),
+                     "kernel": kernel,
+                     "peak_source": "integer-issue probe of this run (warp-inst/s x 32 lanes)",
+                     "issue_peak_warp_inst_per_s": issue_rate,
+                     "issue_slots_used": (cap["warp_inst_per_query_event"] * total_events / sim_s / issue_rate
+                                          if cap else None)},
+        "roofline_hbm": {"bound": "hbm", "kernel": kernel, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "achieved": (slab_bytes + stream_bytes) / sim_s / 1e9,
+                         "frac": (slab_bytes + stream_bytes) / sim_s / 1e9 / peaks["hbm_gbs"],
+                         "bytes": "latency slab written once + every inter-stage stream record written once "
+                                  "and read once (the streams are this design's, not the method's)",
+                         "slab_only_achieved": slab_bytes / sim_s / 1e9,
+                         "slab_only_frac": slab_bytes / sim_s / 1e9 / peaks["hbm_gbs"]},
+        "roofline_select": {"bound": "hbm", "kernel": "select_kernel", "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                            "achieved": slab_bytes / sel_s / 1e9 if sel_s > 0 else None,
+                            "frac": slab_bytes / sel_s / 1e9 / peaks["hbm_gbs"] if sel_s > 0 else None,
+                            "bytes": "8 n per candidate, read once"},
+    }
+    if clocks is not None:
+        rec["clocks"] = clocks
+    return rec
 
-    total_ms, e2e_total = reduce_max([total_ms, e2e_total], dist if world > 1 else None, dev)
+
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    import paper_1812_01776_b200 as il
+
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the Estimator")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    peaks, peaks_kind = load_measured_peaks()
+    stream = torch.cuda.Stream(device=dev)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)   # > 126 MB of L2
+    issue_rate, _ = il.il_measure_int_issue(stream.cuda_stream)
+    torch.cuda.synchronize(dev)
+
+    # every rank takes its own seeded sample (or, for a workload timed in full, its own slice)
+    if args.candidates is None and args.queries is None and args.workload in SUB_BATCH:
+        w, text = load_workload(args.workload, None, None, seed=rank)
+    else:
+        w, text = load_workload(args.workload, (args.candidates or workloads.FULL_SIZES[args.workload][1]) * world
+                                if args.candidates != 0 else 0, args.queries)
+        lo, hi = shard_range(w.n_candidates, rank, world)
+        w.configs = np.ascontiguousarray(w.configs[lo:hi])
+    e2e_steps = 1 if args.no_e2e else max(1, min(args.steps, args.e2e_steps))
+    main = measure(il, torch, w, dev, stream, flush, args.steps, args.warmup, e2e_steps, args.variant,
+                   issue_rate, peaks, barrier, ClockSampler(local) if rank == 0 else None)
+    total_ms, e2e_total = reduce_max([main["step_ms_sum"], main["e2e_ms_sum"]], dist if world > 1 else None, dev)
+
+    per_workload = []
+    if world == 1 and not args.no_per_workload:
+        for wid in (1, 2, 3, 5):
+            if wid == args.workload:
+                continue
+            wk, tk = load_workload(wid, None, None)
+            r = measure(il, torch, wk, dev, stream, flush, 3, 2, 1, args.variant, issue_rate, peaks)
+            r["workload"] = tk
+            for k in ("step_ms_sum", "e2e_ms_sum"):
+                r.pop(k)
+            per_workload.append(r)
     if world > 1:
         dist.destroy_process_group()
     if rank != 0:
         return
 
     K = args.steps
+    n_cand = w.n_candidates
     cand_total = n_cand * world
     value = cand_total * K / (total_ms * 1e-3)
-    e2e_value = cand_total * (1 if args.no_e2e else K) / (e2e_total * 1e-3)
-    peaks, peaks_kind = load_measured_peaks()
-    sim_avg_s = (sum(sim_ms) / K) * 1e-3
-    # integer-issue roofline of the simulation kernel (the dominant one)
-    alu_peak = issue_rate * 32.0                     # thread-level integer ops/s, measured in this run
-    alu_achieved = alg_ops / sim_avg_s
-    # HBM view of the same kernel: slab written once, streams written and read once, trace once per CTA wave
-    n, S = w.n_queries, w.n_stages
-    rec_bytes = 12 if kernel == "des_kernel" else 8  # wide: int64 time + int32 query; else one 64-bit record
-    stream_bytes = (events_per_cand - n) * 2 * rec_bytes
-    hbm_bytes_per_cand = 8 * n + stream_bytes + 4 * S
-    hbm_achieved = hbm_bytes_per_cand * n_cand / sim_avg_s / 1e9
-
+    e2e_value = cand_total * e2e_steps / (e2e_total * 1e-3)
+    cfg = workload_config(w, text, world)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": args.warmup, "ms_per_step": total_ms / K, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-        "config": {"workload": WORKLOADS[args.workload] + " per GPU"
-                               + ("" if not (args.candidates or args.queries) else " [candidates/queries overridden]"),
-                   "candidates_per_gpu": n_cand, "queries": n, "stages": S,
-                   "query_events_per_candidate": events_per_cand,
-                   "l2": "256 MiB buffer written between steps; working set "
-                         f"{ws_bytes / 2**30:.1f} GiB > L2",
-                   "workspace_bytes": ws_bytes, "kernel_variant": args.variant, "kernel": kernel, "parallelism": f"candidates sharded over {world} GPU(s)"},
-        "query_events_per_s": value * events_per_cand,
-        "batches_per_s": batches * world * K / (total_ms * 1e-3) if batches else None,
-        "mean_batch": events_per_cand * n_cand / batches if batches else None,
-        "feasible_fraction": feasible,
-        "kernel_ms": {"simulate": sum(sim_ms) / K, "select": sum(sel_ms) / K},
-        "roofline": {"bound": "alu", "achieved": alu_achieved / 1e12, "peak": alu_peak / 1e12,
-                     "unit": "Tinteger-op/s", "frac": alu_achieved / alu_peak,
-                     "traffic": (NCU_DRAM_BYTES_PER_QUERY_EVENT[kernel] * events_per_cand * n_cand
-                                 if NCU_DRAM_BYTES_PER_QUERY_EVENT.get(kernel) and args.workload == 2
-                                 else None),
-                     "traffic_unit": "DRAM bytes per launch (ncu capture of a reduced case, scaled by query-events)",
-                     "kernel": kernel,
-                     "peak_source": "integer-issue probe of this run (warp-inst/s x 32 lanes)",
-                     "issue_peak_warp_inst_per_s": issue_rate,
-                     "issue_slots_used": (NCU_WARP_INST_PER_QUERY_EVENT[kernel] * events_per_cand * n_cand
-                                          / sim_avg_s / issue_rate
-                                          if NCU_WARP_INST_PER_QUERY_EVENT.get(kernel) and args.workload == 2 else None)},
-        "roofline_hbm": {"bound": "hbm", "achieved": hbm_achieved, "peak": peaks["hbm_gbs"],
-                         "unit": "GB/s", "frac": hbm_achieved / peaks["hbm_gbs"],
-                         "peak_source": f"{peaks_kind} copy bandwidth",
-                         "kernel": kernel},
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(cfg_host.nbytes),
-                "d2h_bytes_per_step": int(16 * n_cand), "matches_device_path": same},
-        "gpu_launches": int(launches),
-        "clocks": clocks,
+        "config": cfg,
+        "launch": {"workspace_bytes": main["workspace_bytes"], "kernel_variant": args.variant,
+                   "kernel": main["kernel"]},
+        "ms_per_step_stats": main["ms_per_step"],
+        "query_events_per_s": value * main["query_events_per_candidate"],
+        "batches_per_s": main["batches"] * world / (total_ms / K * 1e-3) if main["batches"] else None,
+        "mean_batch": main["mean_batch"],
+        "stage_runs_simulated": main["stage_runs_simulated"],
+        "stage_runs_of_the_method": main["stage_runs_of_the_method"],
+        "feasible_fraction": main["feasible_fraction"],
+        "kernel_ms": main["kernel_ms"],
+        "roofline": main["roofline"],
+        "roofline_hbm": dict(main["roofline_hbm"], peak_source=f"{peaks_kind} copy bandwidth"),
+        "roofline_select": dict(main["roofline_select"], peak_source=f"{peaks_kind} copy bandwidth"),
+        "e2e": {"value": e2e_value, "unit": UNIT, "steps": e2e_steps,
+                "h2d_bytes_per_step": main["e2e"]["h2d_bytes_per_step"],
+                "d2h_bytes_per_step": main["e2e"]["d2h_bytes_per_step"],
+                "matches_device_path": main["e2e"]["matches_device_path"]},
+        "gpu_launches": main["gpu_launches"],
+        "clocks": main.get("clocks", {}),
+        "per_workload": per_workload,
     }
     if world == 1 and not args.no_cpu_baseline:
         cores = os.cpu_count() or 1
-        per_cand_s = w.query_events() / 4.5e6            # the oracle does a few million query-events/s/core
-        n_sample = int(max(cores, min(w.n_candidates, 16 * cores, 12.0 * cores / per_cand_s)))
-        n_one = int(max(1, min(64, w.n_candidates, 4.0 / per_cand_s)))
+        n_sample = oracle_sample(w, cores)
+        n_one = int(max(1, min(64, w.n_candidates, 4.0 / (w.query_events() / 4.5e6))))
         import oracle
         pool = oracle.make_pool(cores) if cores > 1 else None
         sec = time_oracle(w, n_sample, cores, pool)
@@ -372,7 +479,7 @@ def run_cuda(args):
         sec1 = time_oracle(w, n_one, 1)
         line["cpu_baseline"] = {
             "value": n_sample / sec, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"first {n_sample} of {w.n_candidates} candidates, full trace, {cores} "
+            "sample": f"first {n_sample} of the {w.n_candidates} candidates of the batch, full trace, {cores} "
                       f"processes x single-threaded oracle; 1 core on {n_one} candidates: "
                       f"{n_one / sec1:.1f} candidates/s",
             "one_core_value": n_one / sec1}
@@ -387,17 +494,20 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", type=int, default=WORKLOAD_ID, choices=[1, 2, 3, 4, 5],
-                    help="which of the five workloads (default 2, the one the metric is quoted on)")
+                    help="which of the five workloads the headline numbers are taken on (default 4, the largest)")
     ap.add_argument("--candidates", type=int, default=None,
-                    help="candidates per GPU (default: the workload's 4,096); smaller values are "
-                         "for profiler captures, not for reported numbers")
+                    help="candidates per GPU: the first N of the workload's draw (0: all of them); default: the "
+                         "full set, or for workload 4 a seeded sample of 16,384 drawn from the whole set")
     ap.add_argument("--queries", type=int, default=None,
-                    help="trace length (default: the workload's 50,000); for profiler captures")
+                    help="trace length (default: the workload's own); shorter traces are for profiler captures")
     ap.add_argument("--variant", type=int, default=0,
                     help="simulation kernel (IL_VARIANT_*): 0 the library's choice, 1 wide streams, "
                          "2 packed records with the trace staged through shared memory, 3 lane kernel, "
                          "4 packed records, one candidate per warp")
-    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer timing (profiler captures)")
+    ap.add_argument("--no-e2e", action="store_true", help="one host-buffer step only (profiler captures)")
+    ap.add_argument("--e2e-steps", type=int, default=5, help="host-buffer steps timed (at most --steps)")
+    ap.add_argument("--no-per-workload", action="store_true",
+                    help="skip the short measurements of the other workloads")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -131,6 +131,15 @@ typedef struct {
     double  sim_ms;          /* device time of the simulation kernels (CUDA events)      */
     double  select_ms;       /* device time of the percentile kernels (CUDA events)      */
     double  total_ms;        /* device time of all stream work of the call               */
+    int64_t fallback_candidates; /* candidates the lane kernel gave up on (stream ring overflow) and the
+                                warp-per-candidate kernel evaluated instead; results are the same     */
+    int64_t stage_runs;      /* (stage, candidate) simulations carried out: candidates * S unless
+                                candidates with a common configuration prefix shared them            */
+    int64_t error_detail;    /* diagnostic for IL_ERR_ITER_LIMIT: which device check gave up (bit 0: the
+                                lane kernel's iteration bound, bit 1: its count of leaving queries, bit 3:
+                                the warp-per-candidate kernel's count of leaving queries); 0 otherwise */
+    int64_t early_exits;     /* il_feasible*: candidates dropped before the end of the trace because more
+                                queries had missed the objective than the P99 rule allows             */
 } il_stats;
 
 /*
@@ -174,6 +183,29 @@ IL_API int il_estimate(il_estimator *est, const il_stage_config *configs, int64_
  */
 IL_API int il_estimate_device(il_estimator *est, const il_stage_config *d_configs, int64_t n,
                               int64_t slo_us, int64_t *d_out_p99_us, int64_t *d_out_miss);
+
+/*
+ * Feasibility only (Section 4.3: the one question the Planner asks in Algorithms 1 and 2,
+ * "Feasible(pipeline, slo)": does the configuration meet the objective at P99?).
+ *   out_feasible[c] = 1  iff  the k-th smallest latency of candidate c is <= slo_us, k = ceil(0.99 n),
+ *                        equivalently iff at most n - k queries have latency > slo_us;  else 0.
+ * Exactly the answer out_p99_us[c] <= slo_us of il_estimate, but cheaper to get: the lane kernel
+ * compares each query with the objective as it leaves the pipeline, writes no latencies and runs no
+ * percentile pass, and drops a candidate as soon as more than n - k of its queries have missed the
+ * objective (an overloaded candidate is decided within the first few per cent of the trace;
+ * il_stats.early_exits counts them).  A feasible candidate is simulated to the end, so its answer is
+ * exact too.  The warp-per-candidate kernels have no early exit: with them this call computes P99
+ * and compares.
+ *   il_feasible         configs HOST [n][S], out_feasible HOST [n] bytes; candidates validated on the host
+ *   il_feasible_device  DEVICE pointers; an invalid candidate makes the call return BAD_CONFIG
+ * Work on the handle's stream; returns after completion.  Errors as il_estimate / il_estimate_device.
+ * If the lane kernel gives candidates up on stream ring overflow (see il_set_variant), they are
+ * evaluated by the warp-per-candidate kernel in the same call, which then allocates temporaries.
+ */
+IL_API int il_feasible(il_estimator *est, const il_stage_config *configs, int64_t n, int64_t slo_us,
+                       uint8_t *out_feasible);
+IL_API int il_feasible_device(il_estimator *est, const il_stage_config *d_configs, int64_t n, int64_t slo_us,
+                              uint8_t *d_out_feasible);
 
 /*
  * The Estimator's full answer for ONE configuration: the latency of every
@@ -279,12 +311,16 @@ IL_API int il_set_workspace(il_estimator *est, void *d_workspace, size_t bytes);
  * a stream element is one 64-bit word (time << q) | query ("packed"); otherwise
  * only IL_VARIANT_WIDE applies and every other choice falls back to it.
  *
- * IL_VARIANT_AUTO (default): the lane kernel when the inter-stage streams of one
- *   candidate take at most 128 MiB, else the packed warp-per-candidate kernel.
+ * IL_VARIANT_AUTO (default): the lane kernel.
  * IL_VARIANT_LANES: one lane per (candidate, stage); the stages of a candidate
  *   run side by side as a pipeline inside one warp, floor(32 / S) candidates per
- *   warp.  Keeps every stage's arrival stream of every resident candidate in
- *   the workspace.
+ *   warp.  A stage's arrival stream lives in a ring of at most 8,192 records, so
+ *   the scratch per resident candidate does not grow with the trace; a parent
+ *   stage waits when it would overrun its child's ring.  A candidate in which one
+ *   batch stays in flight while more than a ring of later records passes through
+ *   the other replicas of its stage cannot be finished that way: it is
+ *   evaluated by the IL_VARIANT_PACKED kernel in the same call
+ *   (il_stats.fallback_candidates counts them).
  * IL_VARIANT_PACKED: one candidate per warp, stages one after the other, replica
  *   slots across the lanes, warp-level primitives for the queue count and the
  *   slot to reuse.
@@ -303,6 +339,19 @@ IL_API int il_set_workspace(il_estimator *est, void *d_workspace, size_t bytes);
 #define IL_VARIANT_LANES 3
 #define IL_VARIANT_PACKED 4
 IL_API int il_set_variant(il_estimator *est, int variant);
+
+/*
+ * Hooks for the library's own tests; not for production use.
+ *   IL_KNOB_LANE_RING_LOG2  value 6..24: largest ring length (log2 records) of the lane kernel's
+ *                           streams (default 13).  Small rings force the overflow path.
+ *   IL_KNOB_ITER_LIMIT      value >= 0: iteration bound of the simulation kernels' loops; 0 restores
+ *                           the bound each loop derives from its input.  A small bound makes a call
+ *                           return IL_ERR_ITER_LIMIT; the handle stays usable.
+ * Set a knob before il_workspace_bytes / il_set_workspace: sizes depend on the ring length.
+ */
+#define IL_KNOB_LANE_RING_LOG2 1
+#define IL_KNOB_ITER_LIMIT 2
+IL_API int il_set_test_knob(il_estimator *est, int knob, int64_t value);
 
 /* Name of the simulation kernel the handle's next estimate call will launch
  * (the choice il_set_variant describes, resolved for the bound inputs);

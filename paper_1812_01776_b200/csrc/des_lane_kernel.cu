@@ -49,6 +49,33 @@
 // its way.  Each lane keeps its own copy of its stage's profile row in shared
 // memory, [batch][lane], so that table look-ups never conflict.
 //
+// Stream memory.  A stage's arrival stream lives in a RING of K records (K a
+// power of two chosen by the host), not in a buffer of its full length, so the
+// scratch a resident candidate needs does not grow with the trace.  A lane still
+// needs every record from the first one of its oldest batch in flight (whose
+// records it re-reads when the batch leaves) up to the one it examines, so the
+// parent may run at most K records ahead of that point: each lane publishes,
+// now and then, the index below which it needs nothing any more, and a parent
+// that would overrun a child's ring holds its hand-on step until the child has
+// moved on (simulated times do not depend on the order in which lanes take their
+// steps).  Leaves write to the slab and never wait, so every wait ends -- except
+// when one batch stays in flight while more than K later records pass through
+// the other replicas of its stage: then parent and child wait for each other.
+// The child detects that (ring full, nothing left to examine or hand on, no
+// progress), marks the candidate in the overflow array and ends the candidate's
+// lanes; the host evaluates marked candidates with the warp-per-candidate
+// kernel, which has no such limit.  With K >= the longest stream (RING = false)
+// none of this code is compiled in.
+//
+// Scheduling.  The floor(32 / S) groups of a warp are independent of each other:
+// when all lanes of a group have finished their candidate, the group takes the
+// next candidate from a global work counter (looked at every eighth iteration)
+// while the other groups carry on, so a warp never idles behind its slowest
+// candidate.  In the feasibility-only instantiation (Section 4.3, "Feasible")
+// the leaves compare each leaving query with the objective instead of writing
+// it to the slab, and a group drops its candidate as soon as more queries have
+// missed the objective than the P99 rule allows.
+//
 // Records and keys are the packed 64-bit words of des_packed_kernel.cu:
 // (time << q) | query for stream records, (finish << q) | index of the batch's
 // first arrival for replica slots, whose unsigned order is (finish, dispatch
@@ -63,6 +90,8 @@ constexpr int kLaneWarps = 2;                  // warps per CTA
 constexpr int kRing = 32;                      // ring positions of a lane's slot list (>= IL_MAX_REPLICAS)
 constexpr uint32_t kDone = 0x80000000u;
 constexpr uint64_t kInf = ~0ull;
+constexpr uint32_t kAbort = 0xffffffffu;      // ring mailbox: the candidate is given up (ring overflow)
+constexpr uint32_t kRingSlack = 4;            // records a parent may have under way when it checks for room
 constexpr int kLag = 40;        // records a stage stays behind its parent while the parent is running
 constexpr int kStage = 4;       // staging ring positions (pending groups + 2)
 constexpr int kPending = 2;     // commit groups that may still be in flight at the end of an iteration
@@ -97,12 +126,22 @@ struct WarpMem {
     // iteration then separates every write of a word from the reads of its previous value.
     uint32_t avail[2][32];       // records written so far into the lane's arrival stream (by its parent
                                  // lane); kDone set once that is all of them
+    // Ring streams only: index below which the lane needs no record of its arrival stream any more
+    // (its parent may overwrite those ring positions), or kAbort.  Grows monotonically; a reader that
+    // sees an older value only waits longer.
+    uint32_t freed[32];
+    // Feasibility only: queries of the group's candidate that have missed the objective so far, [group]
+    uint32_t miss[32];
 };
 
 }  // namespace
 
 // BRANCHY: some stage routes by a branch bit (otherwise every stage has one way out).
-template <bool BRANCHY>
+// RING: the stream rings are shorter than the longest stream, so positions wrap and parents wait for room.
+// FEAS: feasibility only (Section 4.3, "Feasible"): leaving queries are compared with the objective as
+//       they leave, nothing is written to a slab, and a candidate is dropped as soon as more queries
+//       have missed the objective than the P99 rule allows.
+template <bool BRANCHY, bool RING, bool FEAS>
 __global__ void __launch_bounds__(kLaneWarps * 32)
 des_lane_kernel(const __grid_constant__ DesParams p)
 {
@@ -137,6 +176,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
     const int bit = p.bit[s];
     const uint32_t n_in = lane_used ? (uint32_t)p.n_s[s] : 0u;
     const unsigned group_mask = lane_used ? (((1u << S) - 1u) << (j * S)) : 0u;
+    const int root_lane = lane_used ? j * S : 0;
     // mailbox of the child on either side; a lane without that child writes a word nobody reads
     // (its own entry of a spare row would do as well: lanes j * S + child are always in range)
     const int lane_a = (da < 0 || !lane_used) ? -1 : j * S + da;
@@ -145,206 +185,341 @@ des_lane_kernel(const __grid_constant__ DesParams p)
     const int64_t wslot = (int64_t)blockIdx.x * kLaneWarps + wid;
     uint64_t *my_block = p.lane_ws + (wslot * cpw + (lane_used ? j : 0)) * p.lane_elems;
     const uint64_t *in = s == 0 ? p.ptrace : my_block + p.lane_off[s];
-    unsigned long long batches = 0, alg_ops = 0;
+    // ring positions: index & mask (the trace and the slab are not rings)
+    const uint32_t K = 1u << p.lane_ring_log2;
+    const uint32_t in_mask = (RING && s != 0) ? K - 1u : 0xffffffffu;
+    const uint32_t mask_a = (RING && da >= 0) ? K - 1u : 0xffffffffu;
+    const uint32_t mask_b = (RING && db >= 0) ? K - 1u : 0xffffffffu;
+    const unsigned long long iter_limit = p.iter_limit;
+    const unsigned long long n_cand = (unsigned long long)p.n_cand;
+    const uint64_t slo_q = FEAS ? (uint64_t)p.slo_us << q : 0ull;   // the objective, aligned with a record's time field
+    unsigned long long batches = 0, alg_ops = 0, exits_seen = 0, exits_due = 0;
+    unsigned early = 0;          // candidates dropped before the end of the trace (feasibility only)
+
+    // The groups of a warp (one candidate each) are independent: a group whose lanes have all finished
+    // takes the next candidate from the work counter while the other groups carry on.  State of the
+    // lane's candidate:
+    int64_t c = 0;
+    bool has = false;            // the group holds a candidate
+    bool exhausted = !lane_used; // the group will get no further candidate
+    bool live = false, done = true, cand_bad = false;
+    uint32_t R = 1;
+    int mb = 1;
+    uint64_t *out_a = nullptr, *out_b = nullptr;
+    uint32_t epos = 0, lpos = 0, tpos = 0;   // ring positions, see WarpMem
+    uint64_t kfront = kInf;      // key at lpos (kInf when no slot is in use)
+    uint64_t ktail = 0;          // largest key in [lpos, tpos)
+    uint32_t head = 0;           // index of the open batch's first record
+    int b = 0;                   // size of the open batch (0: none)
+    uint64_t tk = 0;             // open batch's dispatch time as (t << q) | qmask
+    uint64_t e_base = 0;         // finish << q of the batch being handed on
+    uint32_t e_idx = 0;          // its next record in the arrival stream
+    uint32_t e_left = 0;         // records of it not yet fetched
+    uint32_t vmask = 0;          // bit k: the record fetched k + 1 iterations ago is on its way out
+    // fetch cursor of the arrival stream: records below fx have been requested; fx1..fx3 are its
+    // values at the end of the previous three iterations, so records below fx3 have arrived
+    uint32_t fx = 0, fx1 = 0, fx2 = 0, fx3 = 0;
+    uint32_t tail_a = 0, tail_b = 0;
+    unsigned nb = 0;
+    uint32_t guard = 0, guard_hi = 0;        // iteration bound, counted down in 32-bit pieces
+    // ring streams: how far the lane's children let it write, what it has told its own parent,
+    // and a new value for that, found at iteration k and published at k + 4 (see below)
+    uint32_t lim_a = 0xffffffffu, lim_b = 0xffffffffu;
+    uint32_t low_pub = 0, low_new = 0, pub_at = 0, e_first = 0;
+    bool low_pending = false, aborted = false;
+    uint32_t av = 0;             // mailbox word this iteration works with: the one read an iteration ago
+    int par = 0;                 // mailbox buffer this iteration publishes into; it reads the other one
+    uint32_t it = 0;
 
     for (;;) {
-        unsigned long long g = 0;
-        if (lane == 0) g = atomicAdd(&p.counters[0], (unsigned long long)cpw);
-        g = __shfl_sync(full, g, 0);
-        if (g >= (unsigned long long)p.n_cand) break;
-        const int64_t c = (int64_t)g + j;
-        const bool has = lane_used && c < p.n_cand;
-        il_stage_config cfg = {0, 1, 1, 0};
-        if (has) cfg = p.configs[c * S + s];
-        const bool bad = has && (cfg.hw >= p.H || cfg.max_batch < 1 || cfg.max_batch > p.Bmax ||
-                                 cfg.replicas < 1 || cfg.replicas > IL_MAX_REPLICAS);
-        const bool cand_bad = (__ballot_sync(full, bad) & group_mask) != 0u;
-        uint64_t *slab = reinterpret_cast<uint64_t *>(p.slab + (has ? c : 0) * p.slab_stride);
-        if (has && cand_bad) {
-            if (s == 0) atomicCAS(p.status, 0, IL_ERR_BAD_CONFIG);
-            for (int i = s; i < p.n; i += S) slab[i] = 0;
-        }
-        const bool live = has && !cand_bad && n_in > 0;
-
-        const uint32_t R = cfg.replicas;
-        const int mb = cfg.max_batch;
-        if (live) {
-            const int32_t *row = s_lat + (s * p.H + cfg.hw) * p.Bmax;
-            for (int k = 0; k < p.Bmax; k++) wm.lat[k][lane] = (uint32_t)row[k];
-        }
-        uint64_t *out_a = da < 0 ? slab + exit_off : my_block + p.lane_off[da];
-        uint64_t *out_b = db < 0 ? slab + exit_off : my_block + p.lane_off[db];
-
-        // the root's stream is complete from the start; a stage nobody visits is finished at once
-        const uint32_t avail0 = (s == 0 || !live) ? (n_in | kDone) : 0u;
-        wm.avail[0][lane] = avail0; wm.avail[1][lane] = avail0;
-        __syncwarp();
-
-        uint32_t epos = 0, lpos = 0, tpos = 0;   // ring positions, see WarpMem
-        uint64_t kfront = kInf;      // key at lpos (kInf when no slot is in use)
-        uint64_t ktail = 0;          // largest key in [lpos, tpos)
-        uint32_t head = 0;           // index of the open batch's first record
-        int b = 0;                   // size of the open batch (0: none)
-        uint64_t tk = 0;             // open batch's dispatch time as (t << q) | qmask
-        uint64_t e_base = 0;         // finish << q of the batch being handed on
-        uint32_t e_idx = 0;          // its next record in the arrival stream
-        uint32_t e_left = 0;         // records of it not yet fetched
-        uint32_t vmask = 0;          // bit k: the record fetched k + 1 iterations ago is on its way out
-        // fetch cursor of the arrival stream: records below fx have been requested; fx1..fx3 are its
-        // values at the end of the previous three iterations, so records below fx3 have arrived
-        uint32_t fx = 0, fx1 = 0, fx2 = 0, fx3 = 0;
-        uint32_t tail_a = 0, tail_b = 0;
-        unsigned nb = 0;
-        bool done = !live;
-        const unsigned long long limit = 8ull * (unsigned)p.n * (unsigned)(S + 1) + 4096ull;
-        uint32_t guard = limit > 0xffffffffull ? 0xffffffffu : (uint32_t)limit;
-        int par = 0;                 // mailbox buffer this iteration publishes into; it reads the other one
-        uint32_t av = avail0;        // mailbox word this iteration works with: the one read an iteration ago
-        uint32_t it = 0;
-
-        for (;;) {
-            const uint32_t av_next = wm.avail[par ^ 1][lane];
-            if (!done) {
-                // the record to hand on in this iteration (requested three iterations ago); its branch bits
-                // are fetched here, so that the load runs under the examine step
-                const bool h_valid = (vmask & 4u) != 0u;
-                const uint32_t h_sl = (it + 1u) & (kStage - 1);
-                const uint32_t h_qid = (uint32_t)wm.stage_e[h_sl][lane] & (uint32_t)qmask;   // unused unless h_valid
-                const uint64_t h_base = wm.stage_b[h_sl][lane];
-                uint32_t h_bits = 0;
-                if (BRANCHY && h_valid && bit >= 0) h_bits = p.bits[h_qid];
-                // likewise the next batch to hand on, if the one in hand is used up (a batch handed over in
-                // this iteration is picked up in the next), and the table entry a close would need
-                const bool f_valid = e_left == 0 && epos != lpos;
-                const uint64_t f_key = wm.key[epos & (kRing - 1)][lane];                      // unused unless f_valid
-                const uint32_t f_cnt = wm.cnt[epos & (kRing - 1)][lane];
-                // (latency << q) - qmask: finish key base = dispatch key + that
-                const uint64_t latq = ((uint64_t)wm.lat[b > 0 ? b - 1 : 0][lane] << q) - qmask;
-                // key of the second slot in use, the front after a hand-over (unused unless there are two)
-                uint64_t k2 = wm.key[(lpos + 1u) & (kRing - 1)][lane];
-                const uint32_t written = av & ~kDone;
-                const bool pdone = (av & kDone) != 0u;
-
-                // ---- examine one record of the arrival stream
-                const uint32_t i = head + (uint32_t)b;
-                const bool known = i < fx3;
-                const uint64_t ra = wm.stage_x[i & (kStage - 1)][lane];
-                const bool end = pdone && i >= written;
-                const bool join = known && b > 0 && b < mb && ra <= tk;
-                b += join ? 1 : 0;
-                const bool room = tpos - epos < (uint32_t)kRing;
-                const bool close = b > 0 && !join && (known || end || b == mb) && room;
-                // close and open as straight-line code under predicates (only the sorted insert branches),
-                // so that the hand-on and request steps below can overlap with it
-                const uint64_t key = (tk + latq) | head;
-                uint32_t pos = tpos;
-                const bool sorted_insert = close && tpos != lpos && key < ktail;
-                if (sorted_insert) {
-                    // a batch that finishes before one dispatched earlier
-#pragma unroll 1
-                    while (pos != lpos) {
-                        const uint64_t prev = wm.key[(pos - 1) & (kRing - 1)][lane];
-                        if (prev <= key) break;
-                        wm.key[pos & (kRing - 1)][lane] = prev;
-                        wm.cnt[pos & (kRing - 1)][lane] = wm.cnt[(pos - 1) & (kRing - 1)][lane];
-                        pos--;
+        // ---- every eighth iteration: drop decided candidates, hand finished groups their next candidate
+        if ((it & 7u) == 0u) {
+            if (FEAS && has && !done && wm.miss[j] > p.miss_allow) done = true;   // same word, same moment: the whole group
+            const unsigned dm = __ballot_sync(full, done);
+            const bool turn = !exhausted && (dm & group_mask) == group_mask;
+            if (__any_sync(full, turn)) {
+                // a candidate that was dropped (decided, given up, out of iterations) may still have
+                // copies under way into the lane's staging rings: let them land before the rings are reused
+                cp_async_wait<0>();
+                // wrap up the candidate the group has finished
+                const bool cand_aborted = RING && (__ballot_sync(full, aborted && turn) & group_mask) != 0u;
+                if (turn && has) {
+                    if (live && !cand_aborted) {
+                        batches += nb;
+                        alg_ops += 3ull * n_in + (unsigned long long)nb * (unsigned)(R + mb + 4);
+                    }
+                    const bool decided = FEAS && wm.miss[j] > p.miss_allow;
+                    // every query of a candidate that ran to its end must have left through exactly one
+                    // leaf (checked over all candidates of the warp when the kernel ends)
+                    if (live && !cand_aborted && !decided)
+                        exits_seen += (da < 0 ? tail_a : 0u) + ((db < 0 && bit >= 0) ? tail_b : 0u);
+                    if (s == 0 && !cand_bad && !cand_aborted && !decided) exits_due += (unsigned)p.n;
+                    if (FEAS && s == 0) {
+                        p.out_feasible[c] = cand_aborted ? 2 : (decided || cand_bad ? 0 : 1);
+                        early += (decided && head < n_in) ? 1u : 0u;     // the root had not reached the end of the trace
                     }
                 }
-                if (close) {
-                    wm.key[pos & (kRing - 1)][lane] = key;
-                    wm.cnt[pos & (kRing - 1)][lane] = (uint32_t)b;
+                // the group's next candidate
+                unsigned long long g = 0;
+                if (turn && s == 0) g = atomicAdd(&p.counters[0], 1ull);
+                g = __shfl_sync(full, g, root_lane);
+                il_stage_config cfg = {0, 1, 1, 0};
+                const bool got = turn && g < n_cand;
+                if (got) cfg = p.configs[g * S + s];
+                const bool bad = got && (cfg.hw >= p.H || cfg.max_batch < 1 || cfg.max_batch > p.Bmax ||
+                                         cfg.replicas < 1 || cfg.replicas > IL_MAX_REPLICAS);
+                const bool grp_bad = (__ballot_sync(full, bad) & group_mask) != 0u;
+                if (turn) {
+                    has = got;
+                    exhausted = !got;
+                    c = (int64_t)g;
+                    cand_bad = grp_bad;
+                    uint64_t *slab = FEAS ? nullptr : reinterpret_cast<uint64_t *>(p.slab + (got ? c : 0) * p.slab_stride);
+                    if (got && cand_bad) {
+                        if (s == 0) atomicCAS(p.status, 0, IL_ERR_BAD_CONFIG);
+                        if (!FEAS) for (int i = s; i < p.n; i += S) slab[i] = 0;
+                    }
+                    live = got && !cand_bad && n_in > 0;
+                    R = cfg.replicas;
+                    mb = cfg.max_batch;
+                    if (live) {
+                        const int32_t *row = s_lat + (s * p.H + cfg.hw) * p.Bmax;
+                        for (int k = 0; k < p.Bmax; k++) wm.lat[k][lane] = (uint32_t)row[k];
+                    }
+                    out_a = da < 0 ? slab + exit_off : my_block + p.lane_off[da];
+                    out_b = db < 0 ? slab + exit_off : my_block + p.lane_off[db];
+                    // the root's stream is complete from the start; a stage nobody visits is finished at once
+                    const uint32_t avail0 = (s == 0 || !live) ? (n_in | kDone) : 0u;
+                    wm.avail[0][lane] = avail0; wm.avail[1][lane] = avail0;
+                    if (RING) wm.freed[lane] = 0u;
+                    if (FEAS && s == 0) wm.miss[j] = 0u;
+                    epos = 0; lpos = 0; tpos = 0;
+                    kfront = kInf; ktail = 0;
+                    head = 0; b = 0; tk = 0;
+                    e_base = 0; e_idx = 0; e_left = 0; vmask = 0;
+                    fx = 0; fx1 = 0; fx2 = 0; fx3 = 0;
+                    tail_a = 0; tail_b = 0; nb = 0;
+                    done = !live;
+                    const unsigned long long limit =
+                        iter_limit ? iter_limit : 8ull * (unsigned)p.n * (unsigned)(S + 1) + 4096ull;
+                    guard = (uint32_t)(limit & 0xffffffffull) + 1u;
+                    guard_hi = (uint32_t)(limit >> 32);
+                    if (guard == 0u) guard = 0xffffffffu;
+                    lim_a = (RING && lane_a >= 0) ? K : 0xffffffffu;
+                    lim_b = (RING && lane_b >= 0) ? K : 0xffffffffu;
+                    low_pub = 0; low_new = 0; pub_at = 0; e_first = 0;
+                    low_pending = false; aborted = false;
+                    av = avail0;
                 }
-                ktail = (close && !sorted_insert) ? key : ktail;
-                const bool at_front = close && pos == lpos;
-                k2 = at_front ? kfront : ((close && pos == lpos + 1u) ? key : k2);
-                kfront = at_front ? key : kfront;
-                tpos += close ? 1u : 0u;
-                nb += close ? 1u : 0u;
-                head = close ? i : head;
-                b = close ? 0 : b;
-                // record i opens the next batch on the replica that is free first: one that was never used
-                // (free from time 0) while there is one, else the slot with the smallest key
-                const bool open = known && !join && b == 0;
-                const bool pop = open && tpos - lpos == R;
-                const uint64_t kf = pop ? kfront : 0ull;
-                lpos += pop ? 1u : 0u;
-                kfront = pop ? (lpos != tpos ? k2 : kInf) : kfront;
-                tk = open ? (max(kf, ra) | qmask) : tk;
-                b = open ? 1 : b;
-                if (end && b == 0) lpos = tpos;     // stream exhausted: everything still held leaves, in key order
-
-                // ---- hand on the record picked up at the top of the iteration
-                if (BRANCHY) {
-                    // under predicates: with lanes on both sides of a branch point in one warp this measured
-                    // 10 % faster than a branch around the block; without routing the branch is the faster form
-                    const uint64_t out = h_base | h_qid;
-                    const bool to_b = bit >= 0 && ((h_bits >> bit) & 1u);
-                    uint64_t *dst = to_b ? out_b + tail_b : out_a + tail_a;
-                    if (h_valid) *dst = out;
-                    tail_b += (h_valid && to_b) ? 1u : 0u;
-                    tail_a += (h_valid && !to_b) ? 1u : 0u;
-                } else if (h_valid) {
-                    out_a[tail_a] = h_base | h_qid;
-                    tail_a++;
-                }
-                // ---- request the next record to hand on
-                if (f_valid) {
-                    e_left = f_cnt;
-                    e_base = f_key & ~qmask;
-                    e_idx = (uint32_t)f_key & (uint32_t)qmask;
-                    epos++;
-                }
-                vmask = (vmask << 1) & 7u;
-                if (e_left > 0) {
-                    const uint32_t sl = it & (kStage - 1);
-                    cp_async8(&wm.stage_e[sl][lane], in + e_idx);
-                    wm.stage_b[sl][lane] = e_base;
-                    e_idx++; e_left--;
-                    vmask |= 1u;
-                }
-                // ---- request the next record to examine: up to kStage records from the one examined
-                // next, and (while the parent runs) kLag behind what it has written
-                const uint32_t i2 = head + (uint32_t)b;
-                if (fx < i2 + (uint32_t)kStage && (pdone ? fx < written : fx + (uint32_t)kLag < written)) {
-                    cp_async8(&wm.stage_x[fx & (kStage - 1)][lane], in + fx);
-                    fx++;
-                }
-                done = end && b == 0 && epos == tpos && vmask == 0u;
-                if (--guard == 0) { atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT); done = true; }
+                __syncwarp();     // the mailboxes are set before anybody reads them
+                if (__all_sync(full, exhausted)) break;
             }
-            fx3 = fx2; fx2 = fx1; fx1 = fx;
-            cp_async_commit();
-            cp_async_wait<kPending>();
-            // every lane publishes every iteration (a finished lane repeats its last words)
-            if (lane_a >= 0) wm.avail[par][lane_a] = tail_a | (done ? kDone : 0u);
-            if (lane_b >= 0) wm.avail[par][lane_b] = tail_b | (done ? kDone : 0u);
-            av = av_next;
-            par ^= 1;
-            it++;
-            __syncwarp();
-            if (__all_sync(full, done)) break;
         }
-        cp_async_wait<0>();
+        const uint32_t av_next = wm.avail[par ^ 1][lane];
+        if (!done) {
+            // the record to hand on in this iteration (requested three iterations ago); its branch bits
+            // are fetched here, so that the load runs under the examine step
+            const bool h_valid = (vmask & 4u) != 0u;
+            const uint32_t h_sl = (it + 1u) & (kStage - 1);
+            const uint32_t h_qid = (uint32_t)wm.stage_e[h_sl][lane] & (uint32_t)qmask;   // unused unless h_valid
+            const uint64_t h_base = wm.stage_b[h_sl][lane];
+            uint32_t h_bits = 0;
+            if (BRANCHY && h_valid && bit >= 0) h_bits = p.bits[h_qid];
+            // feasibility only: the arrival record of a query that may leave here, to test its latency
+            uint64_t h_arr = 0;
+            if (FEAS && h_valid && (da < 0 || (db < 0 && bit >= 0))) h_arr = p.ptrace[h_qid];
+            // likewise the next batch to hand on, if the one in hand is used up (a batch handed over in
+            // this iteration is picked up in the next), and the table entry a close would need
+            const bool f_valid = e_left == 0 && epos != lpos;
+            const uint64_t f_key = wm.key[epos & (kRing - 1)][lane];                      // unused unless f_valid
+            const uint32_t f_cnt = wm.cnt[epos & (kRing - 1)][lane];
+            // (latency << q) - qmask: finish key base = dispatch key + that
+            const uint64_t latq = ((uint64_t)wm.lat[b > 0 ? b - 1 : 0][lane] << q) - qmask;
+            // key of the second slot in use, the front after a hand-over (unused unless there are two)
+            uint64_t k2 = wm.key[(lpos + 1u) & (kRing - 1)][lane];
+            const uint32_t written = av & ~kDone;
+            const bool pdone = (av & kDone) != 0u;
+            // ring streams: may this lane start handing on another record?  Not while a child's
+            // ring could be overrun by the records under way (rare: the limits are re-read then)
+            bool can_emit = true;
+            if (RING) {
+                can_emit = tail_a + kRingSlack <= lim_a && tail_b + kRingSlack <= lim_b;
+                if (!can_emit) {
+                    const uint32_t fa = lane_a >= 0 ? wm.freed[lane_a] : 0u;
+                    const uint32_t fb = lane_b >= 0 ? wm.freed[lane_b] : 0u;
+                    if ((lane_a >= 0 && fa == kAbort) || (lane_b >= 0 && fb == kAbort)) aborted = true;
+                    lim_a = lane_a >= 0 ? fa + K : 0xffffffffu;
+                    lim_b = lane_b >= 0 ? fb + K : 0xffffffffu;
+                    can_emit = tail_a + kRingSlack <= lim_a && tail_b + kRingSlack <= lim_b;
+                }
+            }
 
-        if (live) {
-            batches += nb;
-            alg_ops += 3ull * n_in + (unsigned long long)nb * (unsigned)(R + mb + 4);
+            // ---- examine one record of the arrival stream
+            const uint32_t i = head + (uint32_t)b;
+            const bool known = i < fx3;
+            const uint64_t ra = wm.stage_x[i & (kStage - 1)][lane];
+            const bool end = pdone && i >= written;
+            const bool join = known && b > 0 && b < mb && ra <= tk;
+            b += join ? 1 : 0;
+            const bool room = tpos - epos < (uint32_t)kRing;
+            const bool close = b > 0 && !join && (known || end || b == mb) && room;
+            // close and open as straight-line code under predicates (only the sorted insert branches),
+            // so that the hand-on and request steps below can overlap with it
+            const uint64_t key = (tk + latq) | head;
+            uint32_t pos = tpos;
+            const bool sorted_insert = close && tpos != lpos && key < ktail;
+            if (sorted_insert) {
+                // a batch that finishes before one dispatched earlier
+#pragma unroll 1
+                while (pos != lpos) {
+                    const uint64_t prev = wm.key[(pos - 1) & (kRing - 1)][lane];
+                    if (prev <= key) break;
+                    wm.key[pos & (kRing - 1)][lane] = prev;
+                    wm.cnt[pos & (kRing - 1)][lane] = wm.cnt[(pos - 1) & (kRing - 1)][lane];
+                    pos--;
+                }
+            }
+            if (close) {
+                wm.key[pos & (kRing - 1)][lane] = key;
+                wm.cnt[pos & (kRing - 1)][lane] = (uint32_t)b;
+            }
+            ktail = (close && !sorted_insert) ? key : ktail;
+            const bool at_front = close && pos == lpos;
+            k2 = at_front ? kfront : ((close && pos == lpos + 1u) ? key : k2);
+            kfront = at_front ? key : kfront;
+            tpos += close ? 1u : 0u;
+            nb += close ? 1u : 0u;
+            head = close ? i : head;
+            b = close ? 0 : b;
+            // record i opens the next batch on the replica that is free first: one that was never used
+            // (free from time 0) while there is one, else the slot with the smallest key
+            const bool open = known && !join && b == 0;
+            const bool pop = open && tpos - lpos == R;
+            const uint64_t kf = pop ? kfront : 0ull;
+            lpos += pop ? 1u : 0u;
+            kfront = pop ? (lpos != tpos ? k2 : kInf) : kfront;
+            tk = open ? (max(kf, ra) | qmask) : tk;
+            b = open ? 1 : b;
+            if (end && b == 0) lpos = tpos;     // stream exhausted: everything still held leaves, in key order
+
+            // ---- hand on the record picked up at the top of the iteration
+            if (BRANCHY) {
+                // under predicates: with lanes on both sides of a branch point in one warp this measured
+                // 10 % faster than a branch around the block; without routing the branch is the faster form
+                const uint64_t out = h_base | h_qid;
+                const bool to_b = bit >= 0 && ((h_bits >> bit) & 1u);
+                if (FEAS) {
+                    const bool leaves = to_b ? db < 0 : da < 0;
+                    if (h_valid && leaves) {
+                        if (h_base > (h_arr & ~qmask) + slo_q) atomicAdd(&wm.miss[j], 1u);
+                    } else if (h_valid) {
+                        uint64_t *dst = to_b ? out_b + (tail_b & mask_b) : out_a + (tail_a & mask_a);
+                        *dst = out;
+                    }
+                } else {
+                    uint64_t *dst = to_b ? out_b + (tail_b & mask_b) : out_a + (tail_a & mask_a);
+                    if (h_valid) *dst = out;
+                }
+                tail_b += (h_valid && to_b) ? 1u : 0u;
+                tail_a += (h_valid && !to_b) ? 1u : 0u;
+            } else if (h_valid) {
+                if (FEAS && da < 0) {
+                    if (h_base > (h_arr & ~qmask) + slo_q) atomicAdd(&wm.miss[j], 1u);
+                } else {
+                    out_a[tail_a & mask_a] = h_base | h_qid;
+                }
+                tail_a++;
+            }
+            // ---- request the next record to hand on
+            if (f_valid) {
+                e_left = f_cnt;
+                e_base = f_key & ~qmask;
+                e_idx = (uint32_t)f_key & (uint32_t)qmask;
+                if (RING) e_first = e_idx;
+                epos++;
+            }
+            vmask = (vmask << 1) & 7u;
+            if (e_left > 0 && can_emit) {
+                const uint32_t sl = it & (kStage - 1);
+                cp_async8(&wm.stage_e[sl][lane], in + (e_idx & in_mask));
+                wm.stage_b[sl][lane] = e_base;
+                e_idx++; e_left--;
+                vmask |= 1u;
+            }
+            // ---- request the next record to examine: up to kStage records from the one examined
+            // next, and (while the parent runs) kLag behind what it has written
+            const uint32_t i2 = head + (uint32_t)b;
+            if (fx < i2 + (uint32_t)kStage && (pdone ? fx < written : fx + (uint32_t)kLag < written)) {
+                cp_async8(&wm.stage_x[fx & (kStage - 1)][lane], in + (fx & in_mask));
+                fx++;
+            }
+            done = end && b == 0 && epos == tpos && e_left == 0 && vmask == 0u;
+            if (RING && s != 0) {
+                // Tell the parent how far it may overwrite the ring.  The lane needs every record
+                // from the first one of any batch it still has to hand on, and from the open batch
+                // on.  The minimum is taken when half the ring is in use and published four
+                // iterations later: copies under way at the time it was taken (records of batches
+                // already picked up for handing on) have landed by then, and every later copy
+                // reads a batch that was counted.
+                if (!low_pending) {
+                    if (written - low_pub >= (K >> 1)) {
+                        uint32_t lo = head;
+                        if (e_left > 0) lo = min(lo, e_first);
+                        for (uint32_t pp = epos; pp != tpos; pp++)
+                            lo = min(lo, (uint32_t)wm.key[pp & (kRing - 1)][lane] & (uint32_t)qmask);
+                        low_new = lo;
+                        low_pending = true;
+                        pub_at = it + 4u;
+                    }
+                } else if (it == pub_at) {
+                    low_pending = false;
+                    if (low_new > low_pub) {
+                        low_pub = low_new;
+                        wm.freed[lane] = low_pub;
+                    } else if (!pdone && written - low_pub + kRingSlack >= K && fx + (uint32_t)kLag >= written &&
+                               i2 >= fx && epos == lpos && e_left == 0 && vmask == 0u) {
+                        // the ring is full, this lane has nothing left to examine or hand on, and
+                        // what pins the ring is a batch still in flight: parent and child would
+                        // wait for each other for ever.  Give the candidate up.
+                        aborted = true;
+                    }
+                }
+            }
+            if (RING && aborted) {
+                p.ovf[c] = 1;
+                wm.freed[lane] = kAbort;
+                done = true;
+            }
+            if (--guard == 0) {
+                if (guard_hi == 0) { atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT); atomicOr(&p.counters[5], 1ull); done = true; }
+                else { guard_hi--; }      // guard wraps to 2^32 - 1 on the next decrement
+            }
         }
-        // every query of the candidate must have left through exactly one leaf
-        int exits = 0;
-        if (live) exits = (da < 0 ? (int)tail_a : 0) + ((db < 0 && bit >= 0) ? (int)tail_b : 0);
-        for (int o = 16; o > 0; o >>= 1) exits += __shfl_xor_sync(full, exits, o);
-        int expect = 0;
-        if (has && !cand_bad && s == 0) expect = p.n;
-        for (int o = 16; o > 0; o >>= 1) expect += __shfl_xor_sync(full, expect, o);
-        if (lane == 0 && exits != expect) atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT);
+        fx3 = fx2; fx2 = fx1; fx1 = fx;
+        cp_async_commit();
+        cp_async_wait<kPending>();
+        // every lane publishes every iteration (a finished lane repeats its last words)
+        if (lane_a >= 0) wm.avail[par][lane_a] = tail_a | (done ? kDone : 0u);
+        if (lane_b >= 0) wm.avail[par][lane_b] = tail_b | (done ? kDone : 0u);
+        av = av_next;
+        par ^= 1;
+        it++;
         __syncwarp();
     }
+    cp_async_wait<0>();
+
     for (int o = 16; o > 0; o >>= 1) {
         batches += __shfl_xor_sync(full, batches, o);
         alg_ops += __shfl_xor_sync(full, alg_ops, o);
+        exits_seen += __shfl_xor_sync(full, exits_seen, o);
+        exits_due += __shfl_xor_sync(full, exits_due, o);
     }
+    if (lane == 0 && exits_seen != exits_due) { atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT); atomicOr(&p.counters[5], 2ull); }
     if (lane == 0 && batches) { atomicAdd(&p.counters[1], batches); atomicAdd(&p.counters[2], alg_ops); }
+    if (FEAS) {
+        for (int o = 16; o > 0; o >>= 1) early += __shfl_xor_sync(full, early, o);
+        if (lane == 0 && early) atomicAdd(&p.counters[6], (unsigned long long)early);
+    }
 }
 
 namespace {
@@ -355,16 +530,31 @@ bool any_branch(const DesParams &p)
 }
 }  // namespace
 
+namespace {
+template <bool BRANCHY, bool RING, bool FEAS>
+cudaError_t launch_one(const DesParams &p, int grid, size_t smem, cudaStream_t stream)
+{
+    cudaError_t e = cudaFuncSetAttribute(des_lane_kernel<BRANCHY, RING, FEAS>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    des_lane_kernel<BRANCHY, RING, FEAS><<<grid, kLaneWarps * 32, smem, stream>>>(p);
+    return cudaGetLastError();
+}
+
+template <bool BRANCHY, bool RING>
+cudaError_t launch_two(const DesParams &p, int grid, size_t smem, cudaStream_t stream)
+{
+    return p.out_feasible ? launch_one<BRANCHY, RING, true>(p, grid, smem, stream)
+                          : launch_one<BRANCHY, RING, false>(p, grid, smem, stream);
+}
+}  // namespace
+
+// Feasibility-only when p.out_feasible is set.
 cudaError_t launch_des_lane(const DesParams &p, int grid, size_t smem, cudaStream_t stream)
 {
     const bool br = any_branch(p);
-    cudaError_t e = br
-        ? cudaFuncSetAttribute(des_lane_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-        : cudaFuncSetAttribute(des_lane_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    if (br) des_lane_kernel<true><<<grid, kLaneWarps * 32, smem, stream>>>(p);
-    else des_lane_kernel<false><<<grid, kLaneWarps * 32, smem, stream>>>(p);
-    return cudaGetLastError();
+    if (p.lane_wrap) return br ? launch_two<true, true>(p, grid, smem, stream) : launch_two<false, true>(p, grid, smem, stream);
+    return br ? launch_two<true, false>(p, grid, smem, stream) : launch_two<false, false>(p, grid, smem, stream);
 }
 
 int des_lane_warps_per_cta() { return kLaneWarps; }
@@ -377,9 +567,9 @@ size_t des_lane_smem(int n_tab)
 int des_lane_max_ctas_per_sm(size_t smem)
 {
     int n = 0;
-    if (cudaFuncSetAttribute(des_lane_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(des_lane_kernel<true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return 0;
-    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, des_lane_kernel<true>, kLaneWarps * 32, smem);
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, des_lane_kernel<true, true, true>, kLaneWarps * 32, smem);
     return e == cudaSuccess ? n : 0;
 }
 

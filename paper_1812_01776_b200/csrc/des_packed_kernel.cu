@@ -886,7 +886,7 @@ __device__ __forceinline__ void simulate_candidate(const DesParams &p, const War
         alg_ops += 3ull * (unsigned)n_in + (unsigned long long)nb * (unsigned)(R + mb + 4);
         __syncwarp();   // this stage's stream writes are read by the next stage's other lanes
     }
-    if (lane == 0 && exits != p.n) atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT);
+    if (lane == 0 && exits != p.n) { atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT); atomicOr(&p.counters[5], 8ull); }
 }
 
 }  // namespace
@@ -926,12 +926,14 @@ des_packed_kernel(const __grid_constant__ DesParams p)
     unsigned long long batches = 0, alg_ops = 0;
 
     if (!STAGED) {
-        // every warp on its own: take the next candidate in the order array
+        // every warp on its own: take the next candidate in the order array (whose length may have
+        // been written by an earlier kernel of the stream)
+        const unsigned long long n_list = p.n_cand_dev ? *p.n_cand_dev : (unsigned long long)p.n_cand;
         for (;;) {
             unsigned long long c = 0;
             if (lane == 0) c = atomicAdd(&p.counters[0], 1ull);
             c = __shfl_sync(full, c, 0);
-            if (c >= (unsigned long long)p.n_cand) break;
+            if (c >= n_list) break;
             simulate_candidate<false>(p, w, s_lat, my_rec, nullptr, true, (int64_t)p.order[c], batches, alg_ops);
         }
     } else {

@@ -21,6 +21,8 @@ static thread_local int g_last_cuda_error = 0;
         }                                               \
     } while (0)
 
+static constexpr int kCounters = 8;
+
 struct il_estimator {
     int device = 0;
     int num_sms = 0;
@@ -43,14 +45,19 @@ struct il_estimator {
     bool lane_ok = false;              // the lane kernel applies (packed records, stream offsets fit 31 bits)
     int variant = IL_VARIANT_AUTO;
     int ctas_per_sm_wide = 0, ctas_per_sm_packed = 0, ctas_per_sm_staged = 0, ctas_per_sm_lane = 0;
-    int64_t lane_elems = 0;            // lane kernel: stream records per candidate
+    int64_t lane_elems = 0;            // lane kernel: stream records per candidate (all rings of a candidate)
+    int lane_ring_log2 = 0;            // lane kernel: a stream ring holds 2^this records
+    int lane_ring_cap_log2 = 13;       // ... at most 2^this (8,192 records = 64 KB per stage and resident candidate)
+    bool lane_wrap = false;            // the rings are shorter than the longest stream
+    unsigned long long iter_limit = 0; // test knob: iteration bound of the device loops (0 = their own)
     int cpw = 1;                       // lane kernel: candidates per warp
     size_t smem_lane = 0;
     uint8_t *d_bits = nullptr;
     int32_t *d_lat = nullptr;
-    unsigned long long *d_counters = nullptr;   // [4]
+    unsigned long long *d_counters = nullptr;   // [kCounters]: next candidate, batches, algorithmic ops,
+                                                // overflow list length of the chunk, overflows of the call
     int *d_status = nullptr;
-    unsigned long long *h_counters = nullptr;   // pinned: [4] counters, then the status word
+    unsigned long long *h_counters = nullptr;   // pinned: [kCounters] counters, then the status word
     int *h_status = nullptr;
 
     void *user_ws = nullptr; size_t user_ws_bytes = 0;
@@ -76,17 +83,13 @@ constexpr int kOneWaveCtasPerSm = 6;
 struct Plan {
     int64_t slots = 0;       // warp slots with stream buffers
     int64_t chunk = 0;       // candidates per (simulate, select) pair
-    size_t off_time = 0, off_qid = 0, off_slab = 0, off_or = 0, off_order = 0, total = 0;
+    int64_t fb_slots = 0;    // lane kernel with wrapping rings: warp slots of the kernel that takes over
+                             // the candidates given up on ring overflow
+    size_t off_time = 0, off_qid = 0, off_slab = 0, off_or = 0, off_order = 0, off_ovf = 0, off_fb = 0, total = 0;
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// The lane kernel keeps every stage's whole arrival stream per resident candidate.  Beyond this many
-// bytes per candidate too few candidates fit the device at once, and the warp-per-candidate kernel,
-// which needs two streams whatever the depth, takes over.  (At 72 MB per candidate, the 10-stage,
-// 10^6-query workload, a 150 GB workspace still holds 1,700 candidates and the lane kernel is 1.7x the
-// faster one.)
-constexpr int64_t kLaneAutoBytes = INT64_C(128) << 20;
 // Resident CTAs (of two warps) per SM for the lane kernel.  Two warps per scheduler keep the issue
 // slots about as busy as more would, and every further warp lengthens all chains through the
 // shared-memory pipe: on B200, workload 2 with 16,384 candidates took 101.7 / 79.2 / 68.4 / 71.1 / 85.5 ms
@@ -102,7 +105,7 @@ int sim_kernel(const il_estimator *e)
 {
     if (!use_packed(e)) return kSimWide;
     if (e->variant == IL_VARIANT_LANES && e->lane_ok) return kSimLane;
-    if (e->variant == IL_VARIANT_AUTO && e->lane_ok && e->lane_elems * 8 <= kLaneAutoBytes) return kSimLane;
+    if (e->variant == IL_VARIANT_AUTO && e->lane_ok) return kSimLane;
     return e->variant == IL_VARIANT_STAGED ? kSimPackedStaged : kSimPacked;
 }
 
@@ -127,7 +130,9 @@ size_t slot_time_bytes(const il_estimator *e)
 }
 size_t slot_qid_bytes(const il_estimator *e) { return is_lane(e) ? 0 : (size_t)e->slot_elems * 4; }
 size_t slot_bytes(const il_estimator *e) { return slot_time_bytes(e) + slot_qid_bytes(e); }
-size_t cand_bytes(const il_estimator *e) { return (size_t)e->n_pad * 8 + 12; }
+size_t cand_bytes(const il_estimator *e) { return (size_t)e->n_pad * 8 + 13; }
+bool lane_fallback(const il_estimator *e) { return is_lane(e) && e->lane_wrap; }
+size_t fb_slot_bytes(const il_estimator *e) { return (size_t)e->slot_elems * 8; }
 
 int64_t full_slots(const il_estimator *e)
 {
@@ -149,8 +154,19 @@ size_t layout(const il_estimator *e, Plan &pl)
     pl.off_slab = off; off = align_up(off + (size_t)pl.chunk * e->n_pad * 8, 256);
     pl.off_or = off;   off = align_up(off + (size_t)pl.chunk * 8, 256);
     pl.off_order = off; off = align_up(off + (size_t)pl.chunk * 4, 256);
+    pl.off_ovf = off;  off = align_up(off + (size_t)pl.chunk, 256);
+    pl.off_fb = off;   off = align_up(off + (size_t)pl.fb_slots * fb_slot_bytes(e), 256);
     pl.total = off;
     return off;
+}
+
+// Warp slots for the kernel that takes over after a ring overflow: about 6 % of the space, between one
+// CTA and one CTA per SM.
+int64_t fallback_slots(const il_estimator *e, size_t usable)
+{
+    if (!lane_fallback(e)) return 0;
+    const int64_t fit = (int64_t)(usable / 16 / fb_slot_bytes(e)) / kWarpsPerCta * kWarpsPerCta;
+    return std::max<int64_t>(kWarpsPerCta, std::min<int64_t>(fit, (int64_t)e->num_sms * kWarpsPerCta));
 }
 
 size_t recommended_bytes(const il_estimator *e, int64_t n_cand)
@@ -160,7 +176,8 @@ size_t recommended_bytes(const il_estimator *e, int64_t n_cand)
     pl.slots = wanted_slots(e, n_cand);
     pl.chunk = std::max<int64_t>(std::min<int64_t>(n_cand, 8 * full_slots(e) * cands_per_slot(e)),
                                  2 * pl.slots * cands_per_slot(e));
-    return layout(e, pl) + 1024;
+    pl.fb_slots = lane_fallback(e) ? (int64_t)e->num_sms * kWarpsPerCta : 0;
+    return layout(e, pl) + 2048;
 }
 
 size_t min_bytes(const il_estimator *e)
@@ -168,14 +185,17 @@ size_t min_bytes(const il_estimator *e)
     Plan pl;
     pl.slots = warps_per_cta(e);
     pl.chunk = 2 * warps_per_cta(e);
-    return layout(e, pl) + 1024;
+    pl.fb_slots = lane_fallback(e) ? kWarpsPerCta : 0;
+    return layout(e, pl) + 2048;
 }
 
 // Splits `bytes` of workspace between warp slots and the latency slab.
 bool make_plan(const il_estimator *e, size_t bytes, int64_t n_cand, Plan &pl)
 {
     if (bytes < min_bytes(e)) return false;
-    const size_t usable = bytes - 1024;
+    size_t usable = bytes - 1024;
+    pl.fb_slots = fallback_slots(e, usable);
+    if (pl.fb_slots > 0) usable -= (size_t)pl.fb_slots * fb_slot_bytes(e) + 256;
     const size_t sb = slot_bytes(e), cb = cand_bytes(e);
     const int64_t w = warps_per_cta(e);
     int64_t slots = std::min<int64_t>(wanted_slots(e, n_cand), (int64_t)(usable / (sb + 2 * cands_per_slot(e) * cb)));
@@ -183,6 +203,10 @@ bool make_plan(const il_estimator *e, size_t bytes, int64_t n_cand, Plan &pl)
     if (slots < w) return false;
     pl.slots = slots;
     pl.chunk = std::min<int64_t>(n_cand, (int64_t)((usable - (size_t)slots * sb) / cb));
+    // several chunks: whole waves of the resident warps per chunk, so that only the last chunk has a
+    // partly filled wave
+    const int64_t wave = slots * cands_per_slot(e);
+    if (pl.chunk < n_cand && pl.chunk > wave) pl.chunk = pl.chunk / wave * wave;
     // alignment padding may push the layout over: shrink the chunk until it fits
     while (pl.chunk > 0 && layout(e, pl) > bytes) pl.chunk -= std::max<int64_t>(1, pl.chunk / 64);
     return pl.chunk >= 1;
@@ -243,6 +267,25 @@ int64_t plan_stream_buffers(const il_profiles *pr, const int64_t *visits, int32_
         top = std::max(top, off + size);
     }
     return top;
+}
+
+// Ring length of the lane kernel's streams: long enough for the longest stream if the cap allows
+// (then nothing wraps), else the cap.  Sets the layout of a candidate's rings.
+void configure_lane_rings(il_estimator *e)
+{
+    int64_t longest = 8;
+    for (int s = 1; s < e->S; s++) longest = std::max(longest, e->visits[s]);
+    int need = 3;
+    while ((INT64_C(1) << need) < longest) need++;
+    e->lane_ring_log2 = std::min(need, e->lane_ring_cap_log2);
+    e->lane_wrap = (INT64_C(1) << e->lane_ring_log2) < longest;
+    DesParams &bp = e->base;
+    bp.lane_off[0] = 0;
+    for (int s = 1; s < e->S; s++) bp.lane_off[s] = (int32_t)((int64_t)(s - 1) << e->lane_ring_log2);
+    e->lane_elems = std::max<int64_t>((int64_t)(e->S - 1) << e->lane_ring_log2, 4);
+    bp.lane_elems = e->lane_elems;
+    bp.lane_ring_log2 = e->lane_ring_log2;
+    bp.lane_wrap = e->lane_wrap ? 1 : 0;
 }
 
 void free_device(il_estimator *e)
@@ -307,6 +350,85 @@ static int acquire_workspace(il_estimator *e, int64_t n_cand, char **ws_out, siz
     *ws_out = ws;
     *bytes_out = ws_bytes;
     return IL_OK;
+}
+
+// Device staging of the host entry points: configurations and the two output arrays.
+static int ensure_staging(il_estimator *e, int64_t n_cand)
+{
+    const int64_t total = n_cand * e->S;
+    if (e->d_cfg_cap < total) {
+        IL_CUDA(cudaStreamSynchronize(e->stream));
+        cudaFree(e->d_cfg); e->d_cfg = nullptr; e->d_cfg_cap = 0;
+        cudaError_t ce = cudaMalloc(&e->d_cfg, (size_t)total * sizeof(il_stage_config));
+        if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return IL_ERR_NOMEM; }
+        e->d_cfg_cap = total;
+    }
+    if (e->d_out_cap < n_cand) {
+        IL_CUDA(cudaStreamSynchronize(e->stream));
+        cudaFree(e->d_out); e->d_out = nullptr; e->d_out_cap = 0;
+        cudaError_t ce = cudaMalloc(&e->d_out, (size_t)n_cand * 24);   // P99, misses, feasibility flags
+        if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return IL_ERR_NOMEM; }
+        e->d_out_cap = n_cand;
+    }
+    return IL_OK;
+}
+
+// Kernel parameters of one chunk: the bound inputs plus this chunk's scratch.
+static DesParams chunk_params(const il_estimator *e, const Plan &pl, char *ws, const il_stage_config *d_configs,
+                              int64_t cnt)
+{
+    DesParams p = e->base;
+    p.configs = d_configs;
+    p.n_cand = cnt;
+    p.slot_elems = e->slot_elems;
+    p.ws_time = reinterpret_cast<int64_t *>(ws + pl.off_time);
+    p.ws_qid = reinterpret_cast<int32_t *>(ws + pl.off_qid);
+    p.lane_ws = reinterpret_cast<uint64_t *>(ws + pl.off_time);
+    p.slab = reinterpret_cast<int64_t *>(ws + pl.off_slab);
+    p.slab_stride = e->n_pad;
+    p.lat_or = reinterpret_cast<uint64_t *>(ws + pl.off_or);
+    p.order = reinterpret_cast<int32_t *>(ws + pl.off_order);
+    p.ovf = reinterpret_cast<uint8_t *>(ws + pl.off_ovf);
+    p.iter_limit = e->iter_limit;
+    return p;
+}
+
+// Enqueues the simulation of one chunk whose work counter is zero: the kernel the handle uses
+// and, behind the lane kernel with wrapping rings, the pass that evaluates the candidates it gave
+// up on with the warp-per-candidate kernel.  `launches` counts the kernels.
+static int enqueue_simulation(il_estimator *e, const DesParams &p, const Plan &pl, char *ws, int64_t ctas,
+                              cudaStream_t st, int64_t *launches)
+{
+    const int kernel = sim_kernel(e);
+    const bool fb = kernel == kSimLane && e->lane_wrap;
+    if (fb) IL_CUDA(cudaMemsetAsync(p.ovf, 0, (size_t)p.n_cand, st));
+    IL_CUDA(launch_simulation(p, kernel, (int)ctas, kernel == kSimLane ? e->smem_lane : e->smem, st));
+    (*launches)++;
+    if (fb) {
+        IL_CUDA(launch_overflow_list(p.ovf, p.n_cand, const_cast<int32_t *>(p.order), e->d_counters, st));
+        DesParams q = p;
+        q.ws_time = reinterpret_cast<int64_t *>(ws + pl.off_fb);
+        q.n_cand_dev = e->d_counters + 3;
+        IL_CUDA(launch_simulation(q, kSimPacked, (int)(pl.fb_slots / kWarpsPerCta), e->smem, st));
+        *launches += 2;
+    }
+    return IL_OK;
+}
+
+// Where each stage's leaving queries end in a slab row written by the lane kernel.
+static void slab_regions(const il_estimator *e, SelectParams &sp)
+{
+    sp.n_regions = 0;
+    int32_t off = 0;
+    for (int s = 0; s < e->S; s++) {
+        const int a = e->base.dest_a[s], b = e->base.dest_b[s];
+        int32_t kids = 0;
+        if (a >= 0) kids += e->base.n_s[a];
+        if (b >= 0 && b != a) kids += e->base.n_s[b];
+        const int32_t leaving = e->base.n_s[s] - kids;
+        off += leaving;
+        if (leaving > 0) sp.region_end[sp.n_regions++] = off;
+    }
 }
 
 extern "C" {
@@ -406,18 +528,10 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     for (int s = 0; s < S; s++) e->events_per_candidate += e->visits[s];
     e->slot_elems = std::max<int64_t>(32, plan_stream_buffers(pr, e->visits, bp.buf_off));
     for (int s = 0; s < S; s++) bp.n_s[s] = (int32_t)e->visits[s];
-    // lane kernel: every stage but the root keeps its whole arrival stream, one after the other
+    // lane kernel: every stage but the root reads its arrival stream from a ring
     e->cpw = 32 / S;
-    e->lane_elems = 0;
-    for (int s = 1; s < S; s++) {
-        bp.lane_off[s] = (int32_t)e->lane_elems;   // below 2^31: checked next
-        e->lane_elems += (e->visits[s] + 3) / 4 * 4;
-    }
-    bp.lane_off[0] = 0;
-    const bool lane_fits = e->lane_elems < (INT64_C(1) << 31);
-    e->lane_elems = std::max<int64_t>(e->lane_elems, 4);
-    bp.lane_elems = e->lane_elems;
     bp.cpw = e->cpw;
+    configure_lane_rings(e);
     bp.S = S; bp.H = H; bp.Bmax = B; bp.n = (int32_t)n;
     e->smem = (size_t)S * H * B * sizeof(int32_t);
 
@@ -430,7 +544,7 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     IL_CUDA_E(cudaMalloc(&e->d_arrival, (size_t)n * 8));
     IL_CUDA_E(cudaMalloc(&e->d_bits, (size_t)n));
     e->can_pack = can_pack;
-    e->lane_ok = can_pack && lane_fits;
+    e->lane_ok = can_pack;
     bp.qbits = qbits;
     if (can_pack) {
         // padded with "never" records to whole tiles, so that bulk copies always move full tiles
@@ -443,10 +557,10 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
         IL_CUDA_E(cudaMemcpy(e->d_ptrace, packed.data(), (size_t)n_padded * 8, cudaMemcpyHostToDevice));
     }
     IL_CUDA_E(cudaMalloc(&e->d_lat, e->smem));
-    IL_CUDA_E(cudaMalloc(&e->d_counters, 4 * sizeof(unsigned long long)));
+    IL_CUDA_E(cudaMalloc(&e->d_counters, kCounters * sizeof(unsigned long long)));
     IL_CUDA_E(cudaMalloc(&e->d_status, sizeof(int)));
-    IL_CUDA_E(cudaMallocHost(&e->h_counters, 6 * sizeof(unsigned long long)));
-    e->h_status = reinterpret_cast<int *>(e->h_counters + 4);
+    IL_CUDA_E(cudaMallocHost(&e->h_counters, (kCounters + 2) * sizeof(unsigned long long)));
+    e->h_status = reinterpret_cast<int *>(e->h_counters + kCounters);
     IL_CUDA_E(cudaMemcpy(e->d_arrival, tr->arrival_us, (size_t)n * 8, cudaMemcpyHostToDevice));
     if (tr->branch_bits) IL_CUDA_E(cudaMemcpy(e->d_bits, tr->branch_bits, (size_t)n, cudaMemcpyHostToDevice));
     else IL_CUDA_E(cudaMemset(e->d_bits, 0, (size_t)n));
@@ -494,6 +608,23 @@ int il_set_variant(il_estimator *e, int variant)
     e->variant = variant;
     e->ctas_per_sm = ctas_for(e);
     return IL_OK;
+}
+
+int il_set_test_knob(il_estimator *e, int knob, int64_t value)
+{
+    if (!e) return IL_ERR_INVALID_ARG;
+    if (knob == IL_KNOB_LANE_RING_LOG2) {
+        if (value < 6 || value > 24) return IL_ERR_INVALID_ARG;
+        e->lane_ring_cap_log2 = (int)value;
+        configure_lane_rings(e);
+        return IL_OK;
+    }
+    if (knob == IL_KNOB_ITER_LIMIT) {
+        if (value < 0) return IL_ERR_INVALID_ARG;
+        e->iter_limit = (unsigned long long)value;
+        return IL_OK;
+    }
+    return IL_ERR_INVALID_ARG;
 }
 
 const char *il_kernel_name(const il_estimator *e)
@@ -567,7 +698,7 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
     if (rc) return rc;
 
     cudaStream_t st = e->stream;
-    IL_CUDA(cudaMemsetAsync(e->d_counters, 0, 4 * sizeof(unsigned long long), st));
+    IL_CUDA(cudaMemsetAsync(e->d_counters, 0, kCounters * sizeof(unsigned long long), st));
     IL_CUDA(cudaMemsetAsync(e->d_status, 0, sizeof(int), st));
     IL_CUDA(cudaEventRecord(e->events[0], st));
 
@@ -575,62 +706,43 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
     for (int64_t ch = 0; ch < n_chunks; ch++) {
         const int64_t lo = ch * pl.chunk;
         const int64_t cnt = std::min(pl.chunk, n_cand - lo);
-        DesParams p = e->base;
-        p.configs = d_configs + lo * e->S;
-        p.n_cand = cnt;
-        p.slot_elems = e->slot_elems;
-        p.ws_time = reinterpret_cast<int64_t *>(ws + pl.off_time);
-        p.ws_qid = reinterpret_cast<int32_t *>(ws + pl.off_qid);
-        p.slab = reinterpret_cast<int64_t *>(ws + pl.off_slab);
-        p.slab_stride = e->n_pad;
-        p.lat_or = reinterpret_cast<uint64_t *>(ws + pl.off_or);
-        p.order = reinterpret_cast<int32_t *>(ws + pl.off_order);
-        OrderParams op;
-        op.configs = p.configs; op.n_cand = cnt; op.lat = e->d_lat;
-        op.S = e->S; op.H = e->H; op.Bmax = e->Bmax;
-        for (int s = 0; s < IL_MAX_STAGES; s++) op.n_s[s] = e->base.n_s[s];
-        op.span_us = e->span_us;
-        op.order = reinterpret_cast<int32_t *>(ws + pl.off_order);
+        DesParams p = chunk_params(e, pl, ws, d_configs + lo * e->S, cnt);
         if (ch > 0) IL_CUDA(cudaMemsetAsync(e->d_counters, 0, sizeof(unsigned long long), st));
         const bool lane = is_lane(e);
         const int64_t wpc = warps_per_cta(e);
         const int64_t groups = (cnt + cands_per_slot(e) - 1) / cands_per_slot(e);
         int64_t ctas = std::min<int64_t>(pl.slots / wpc, (groups + wpc - 1) / wpc);
-        if (lane) {
-            p.lane_ws = reinterpret_cast<uint64_t *>(ws + pl.off_time);   // warps take candidates in index order
-        } else {
+        if (!lane) {   // the lane kernel's warps take candidates in index order
+            OrderParams op;
+            op.configs = p.configs; op.n_cand = cnt; op.lat = e->d_lat;
+            op.S = e->S; op.H = e->H; op.Bmax = e->Bmax;
+            for (int s = 0; s < IL_MAX_STAGES; s++) op.n_s[s] = e->base.n_s[s];
+            op.span_us = e->span_us;
+            op.order = const_cast<int32_t *>(p.order);
             IL_CUDA(launch_order(op, st));
             launches++;
             if (2 * cnt <= 3 * full_slots(e))
                 ctas = std::min<int64_t>(ctas, (int64_t)e->num_sms * std::min(e->ctas_per_sm, kOneWaveCtasPerSm));
         }
         IL_CUDA(cudaEventRecord(e->events[2 + 3 * ch], st));
-        IL_CUDA(launch_simulation(p, sim_kernel(e), (int)ctas, lane ? e->smem_lane : e->smem, st));
+        rc = enqueue_simulation(e, p, pl, ws, ctas, st, &launches);
+        if (rc) return rc;
         IL_CUDA(cudaEventRecord(e->events[3 + 3 * ch], st));
-        SelectParams sp;
+        SelectParams sp = {};
         sp.slab = p.slab; sp.slab_stride = e->n_pad; sp.lat_or = p.lat_or;
         sp.arrival = e->d_arrival; sp.qbits = p.qbits; sp.packed = use_packed(e) ? 1 : 0;
-        sp.n_regions = 0;
-        if (lane) {   // where each stage's leaving queries end in a slab row (the lane kernel's layout)
-            int32_t off = 0;
-            for (int s = 0; s < e->S; s++) {
-                const int a = e->base.dest_a[s], b = e->base.dest_b[s];
-                int32_t kids = 0;
-                if (a >= 0) kids += e->base.n_s[a];
-                if (b >= 0 && b != a) kids += e->base.n_s[b];
-                const int32_t leaving = e->base.n_s[s] - kids;
-                off += leaving;
-                if (leaving > 0) sp.region_end[sp.n_regions++] = off;
-            }
+        if (lane) {
+            slab_regions(e, sp);
+            if (e->lane_wrap) sp.ovf = p.ovf;
         }
         sp.n = (int32_t)e->n; sp.n_cand = cnt; sp.slo_us = slo_us;
         sp.out_p99 = d_out_p99 + lo; sp.out_miss = d_out_miss + lo;
         IL_CUDA(launch_select(sp, st));
         IL_CUDA(cudaEventRecord(e->events[4 + 3 * ch], st));
-        launches += 2;
+        launches++;
     }
     IL_CUDA(cudaEventRecord(e->events[1], st));
-    IL_CUDA(cudaMemcpyAsync(e->h_counters, e->d_counters, 4 * sizeof(unsigned long long),
+    IL_CUDA(cudaMemcpyAsync(e->h_counters, e->d_counters, kCounters * sizeof(unsigned long long),
                             cudaMemcpyDeviceToHost, st));
     IL_CUDA(cudaMemcpyAsync(e->h_status, e->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
     IL_CUDA(cudaStreamSynchronize(st));
@@ -650,6 +762,10 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
     e->stats.algorithmic_ops = (int64_t)e->h_counters[2];
     e->stats.chunks = n_chunks;
     e->stats.kernel_launches = launches;
+    e->stats.fallback_candidates = (int64_t)e->h_counters[4];
+    e->stats.error_detail = (int64_t)e->h_counters[5];
+    e->stats.early_exits = 0;
+    e->stats.stage_runs = n_cand * e->S;
     return *e->h_status;
 }
 
@@ -664,22 +780,14 @@ int il_estimate_latencies(il_estimator *e, const il_stage_config *d_config, int6
     Plan pl;
     if (!make_plan(e, ws_bytes, 1, pl)) return IL_ERR_NOMEM;
     cudaStream_t st = e->stream;
-    IL_CUDA(cudaMemsetAsync(e->d_counters, 0, 4 * sizeof(unsigned long long), st));
+    IL_CUDA(cudaMemsetAsync(e->d_counters, 0, kCounters * sizeof(unsigned long long), st));
     IL_CUDA(cudaMemsetAsync(e->d_status, 0, sizeof(int), st));
-    DesParams p = e->base;
-    p.configs = d_config;
-    p.n_cand = 1;
-    p.slot_elems = e->slot_elems;
-    p.ws_time = reinterpret_cast<int64_t *>(ws + pl.off_time);
-    p.ws_qid = reinterpret_cast<int32_t *>(ws + pl.off_qid);
-    p.slab = reinterpret_cast<int64_t *>(ws + pl.off_slab);
-    p.slab_stride = e->n_pad;
-    p.lat_or = reinterpret_cast<uint64_t *>(ws + pl.off_or);
-    p.order = reinterpret_cast<int32_t *>(ws + pl.off_order);
+    DesParams p = chunk_params(e, pl, ws, d_config, 1);
     IL_CUDA(cudaMemsetAsync(ws + pl.off_order, 0, sizeof(int32_t), st));   // the one candidate is number 0
     const int kernel = sim_kernel(e);
-    p.lane_ws = reinterpret_cast<uint64_t *>(ws + pl.off_time);
-    IL_CUDA(launch_simulation(p, kernel, 1, kernel == kSimLane ? e->smem_lane : e->smem, st));
+    int64_t launches = 0;
+    rc = enqueue_simulation(e, p, pl, ws, 1, st, &launches);
+    if (rc) return rc;
     if (kernel == kSimWide)   // the wide kernel writes latencies in trace order
         IL_CUDA(cudaMemcpyAsync(d_out_latency, p.slab, (size_t)e->n * 8, cudaMemcpyDeviceToDevice, st));
     else
@@ -697,12 +805,12 @@ int il_traffic_envelope(il_estimator *e, const int64_t *window_us, int32_t n_win
     for (int w = 0; w < n_windows; w++) if (window_us[w] < 1) return IL_ERR_INVALID_ARG;
     IL_CUDA(cudaSetDevice(e->device));
     // the counts fit the 4-word counter block that every estimate call clears before use
-    static_assert(sizeof(unsigned long long) * 4 >= sizeof(int) * 8, "counter block too small");
+    static_assert(sizeof(unsigned long long) * kCounters >= sizeof(int) * 8, "counter block too small");
     int host_out[64];
     cudaStream_t st = e->stream;
     for (int w0 = 0; w0 < n_windows; w0 += 8) {
         const int cnt = std::min(8, n_windows - w0);
-        IL_CUDA(cudaMemsetAsync(e->d_counters, 0, 4 * sizeof(unsigned long long), st));
+        IL_CUDA(cudaMemsetAsync(e->d_counters, 0, kCounters * sizeof(unsigned long long), st));
         IL_CUDA(launch_envelope(e->d_arrival, (int)e->n, window_us + w0, cnt,
                                 reinterpret_cast<int *>(e->d_counters), e->num_sms, st));
         IL_CUDA(cudaMemcpyAsync(host_out + w0, e->d_counters, cnt * sizeof(int), cudaMemcpyDeviceToHost, st));
@@ -726,20 +834,8 @@ int il_estimate(il_estimator *e, const il_stage_config *configs, int64_t n_cand,
             return IL_ERR_BAD_CONFIG;
     }
     IL_CUDA(cudaSetDevice(e->device));
-    if (e->d_cfg_cap < total) {
-        IL_CUDA(cudaStreamSynchronize(e->stream));
-        cudaFree(e->d_cfg); e->d_cfg = nullptr; e->d_cfg_cap = 0;
-        cudaError_t ce = cudaMalloc(&e->d_cfg, (size_t)total * sizeof(il_stage_config));
-        if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return IL_ERR_NOMEM; }
-        e->d_cfg_cap = total;
-    }
-    if (e->d_out_cap < n_cand) {
-        IL_CUDA(cudaStreamSynchronize(e->stream));
-        cudaFree(e->d_out); e->d_out = nullptr; e->d_out_cap = 0;
-        cudaError_t ce = cudaMalloc(&e->d_out, (size_t)n_cand * 16);
-        if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return IL_ERR_NOMEM; }
-        e->d_out_cap = n_cand;
-    }
+    int rc0 = ensure_staging(e, n_cand);
+    if (rc0) return rc0;
     IL_CUDA(cudaMemcpyAsync(e->d_cfg, configs, (size_t)total * sizeof(il_stage_config),
                             cudaMemcpyHostToDevice, e->stream));
     int rc = il_estimate_device(e, e->d_cfg, n_cand, slo_us, e->d_out, e->d_out + e->d_out_cap);
@@ -747,6 +843,153 @@ int il_estimate(il_estimator *e, const il_stage_config *configs, int64_t n_cand,
     IL_CUDA(cudaMemcpyAsync(out_p99, e->d_out, (size_t)n_cand * 8, cudaMemcpyDeviceToHost, e->stream));
     IL_CUDA(cudaMemcpyAsync(out_miss, e->d_out + e->d_out_cap, (size_t)n_cand * 8,
                             cudaMemcpyDeviceToHost, e->stream));
+    IL_CUDA(cudaStreamSynchronize(e->stream));
+    return IL_OK;
+}
+
+int il_feasible_device(il_estimator *e, const il_stage_config *d_configs, int64_t n_cand, int64_t slo_us,
+                       uint8_t *d_out_feasible)
+{
+    if (!e || n_cand < 0) return IL_ERR_INVALID_ARG;
+    e->stats = il_stats{};
+    if (n_cand == 0) return IL_OK;
+    if (!d_configs || !d_out_feasible) return IL_ERR_INVALID_ARG;
+    IL_CUDA(cudaSetDevice(e->device));
+    cudaStream_t st = e->stream;
+
+    if (!is_lane(e)) {
+        // the other kernels have no early exit: P99 as usual, then the comparison
+        int rc = ensure_staging(e, n_cand);
+        if (rc) return rc;
+        rc = il_estimate_device(e, d_configs, n_cand, slo_us, e->d_out, e->d_out + e->d_out_cap);
+        if (rc) return rc;
+        IL_CUDA(launch_feasible_from_p99(e->d_out, nullptr, n_cand, slo_us, d_out_feasible, st));
+        IL_CUDA(cudaStreamSynchronize(st));
+        e->stats.kernel_launches++;
+        return IL_OK;
+    }
+
+    // lane kernel: no slab and no percentile pass, so the whole batch is one chunk
+    char *ws = nullptr;
+    size_t ws_bytes = 0;
+    int rc = acquire_workspace(e, std::min<int64_t>(n_cand, 4096), &ws, &ws_bytes);
+    if (rc) return rc;
+    const int64_t wpc = des_lane_warps_per_cta();
+    const size_t sb = slot_time_bytes(e);
+    const size_t tail_bytes = align_up((size_t)n_cand, 256) + align_up((size_t)n_cand * 4, 256) + 1024;
+    if (ws_bytes < tail_bytes + (size_t)wpc * sb) return IL_ERR_NOMEM;
+    int64_t slots = std::min<int64_t>(wanted_slots(e, n_cand), (int64_t)((ws_bytes - tail_bytes) / sb)) / wpc * wpc;
+    if (slots < wpc) return IL_ERR_NOMEM;
+    const size_t off_ovf = align_up((size_t)slots * sb, 256);
+    const size_t off_order = off_ovf + align_up((size_t)n_cand, 256);
+    rc = ensure_events(e, 4);
+    if (rc) return rc;
+
+    IL_CUDA(cudaMemsetAsync(e->d_counters, 0, kCounters * sizeof(unsigned long long), st));
+    IL_CUDA(cudaMemsetAsync(e->d_status, 0, sizeof(int), st));
+    DesParams p = e->base;
+    p.configs = d_configs;
+    p.n_cand = n_cand;
+    p.lane_ws = reinterpret_cast<uint64_t *>(ws);
+    p.ovf = reinterpret_cast<uint8_t *>(ws + off_ovf);
+    p.iter_limit = e->iter_limit;
+    p.out_feasible = d_out_feasible;
+    // latency > objective is tested on time fields shifted by qbits: keep the objective in that range
+    // (latencies are at least 1 and every reachable time is below 2^(63 - qbits))
+    p.slo_us = std::min<int64_t>(std::max<int64_t>(slo_us, 0), INT64_C(1) << (62 - p.qbits));
+    p.miss_allow = (uint32_t)(e->n - (99 * e->n + 99) / 100);
+    if (e->lane_wrap) IL_CUDA(cudaMemsetAsync(p.ovf, 0, (size_t)n_cand, st));
+    const int64_t groups = (n_cand + e->cpw - 1) / e->cpw;
+    const int64_t ctas = std::min<int64_t>(slots / wpc, (groups + wpc - 1) / wpc);
+    IL_CUDA(cudaEventRecord(e->events[0], st));
+    IL_CUDA(launch_des_lane(p, (int)ctas, e->smem_lane, st));
+    IL_CUDA(cudaEventRecord(e->events[1], st));
+    int64_t launches = 1;
+    if (e->lane_wrap) {
+        IL_CUDA(launch_overflow_list(p.ovf, n_cand, reinterpret_cast<int32_t *>(ws + off_order), e->d_counters, st));
+        launches++;
+    }
+    IL_CUDA(cudaMemcpyAsync(e->h_counters, e->d_counters, kCounters * sizeof(unsigned long long),
+                            cudaMemcpyDeviceToHost, st));
+    IL_CUDA(cudaMemcpyAsync(e->h_status, e->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+    IL_CUDA(cudaStreamSynchronize(st));
+    float ms = 0.f;
+    IL_CUDA(cudaEventElapsedTime(&ms, e->events[0], e->events[1]));
+    il_stats stats = {};
+    stats.candidates = n_cand;
+    stats.query_events = n_cand * e->events_per_candidate;
+    stats.batches = (int64_t)e->h_counters[1];
+    stats.algorithmic_ops = (int64_t)e->h_counters[2];
+    stats.chunks = 1;
+    stats.sim_ms = ms;
+    stats.total_ms = ms;
+    stats.fallback_candidates = (int64_t)e->h_counters[3];
+    stats.error_detail = (int64_t)e->h_counters[5];
+    stats.early_exits = (int64_t)e->h_counters[6];
+    stats.stage_runs = n_cand * e->S;
+    rc = *e->h_status;
+    const int64_t n_fb = (int64_t)e->h_counters[3];
+    if (rc == IL_OK && n_fb > 0) {
+        // Rare: candidates the lane kernel gave up on (stream ring overflow).  They are evaluated in
+        // full by the warp-per-candidate kernel; this path allocates its temporaries.
+        char *tmp = nullptr;
+        const size_t cfg_b = align_up((size_t)n_fb * e->S * sizeof(il_stage_config), 256);
+        const size_t lst_b = align_up((size_t)n_fb * 4, 256), out_b = align_up((size_t)n_fb * 8, 256);
+        cudaError_t ce = cudaMalloc(&tmp, cfg_b + lst_b + 2 * out_b);
+        if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return IL_ERR_NOMEM; }
+        il_stage_config *cfg2 = reinterpret_cast<il_stage_config *>(tmp);
+        int32_t *list = reinterpret_cast<int32_t *>(tmp + cfg_b);
+        int64_t *p99 = reinterpret_cast<int64_t *>(tmp + cfg_b + lst_b);
+        int64_t *miss = reinterpret_cast<int64_t *>(tmp + cfg_b + lst_b + out_b);
+        cudaError_t c1 = cudaMemcpyAsync(list, ws + off_order, (size_t)n_fb * 4, cudaMemcpyDeviceToDevice, st);
+        if (c1 == cudaSuccess) c1 = launch_gather_configs(d_configs, list, n_fb, e->S, cfg2, st);
+        const int variant = e->variant;
+        if (c1 == cudaSuccess) {
+            il_set_variant(e, IL_VARIANT_PACKED);
+            rc = il_estimate_device(e, cfg2, n_fb, slo_us, p99, miss);
+            il_set_variant(e, variant);
+            stats.batches += e->stats.batches;
+            stats.algorithmic_ops += e->stats.algorithmic_ops;
+            stats.sim_ms += e->stats.sim_ms;
+            stats.select_ms += e->stats.select_ms;
+            stats.total_ms += e->stats.total_ms;
+            launches += e->stats.kernel_launches + 2;
+            if (rc == IL_OK) c1 = launch_feasible_from_p99(p99, list, n_fb, slo_us, d_out_feasible, st);
+        }
+        if (c1 == cudaSuccess) c1 = cudaStreamSynchronize(st);
+        else cudaStreamSynchronize(st);
+        cudaFree(tmp);
+        if (c1 != cudaSuccess) { g_last_cuda_error = (int)c1; return IL_ERR_CUDA; }
+    }
+    stats.kernel_launches = launches;
+    e->stats = stats;
+    return rc;
+}
+
+int il_feasible(il_estimator *e, const il_stage_config *configs, int64_t n_cand, int64_t slo_us,
+                uint8_t *out_feasible)
+{
+    if (!e || n_cand < 0) return IL_ERR_INVALID_ARG;
+    if (n_cand == 0) { e->stats = il_stats{}; return IL_OK; }
+    if (!configs || !out_feasible) return IL_ERR_INVALID_ARG;
+    const int64_t total = n_cand * e->S;
+    for (int64_t i = 0; i < total; i++) {
+        const il_stage_config &c = configs[i];
+        if (c.hw >= e->H || c.max_batch < 1 || c.max_batch > e->Bmax || c.replicas < 1 ||
+            c.replicas > IL_MAX_REPLICAS)
+            return IL_ERR_BAD_CONFIG;
+    }
+    IL_CUDA(cudaSetDevice(e->device));
+    int rc = ensure_staging(e, n_cand);
+    if (rc) return rc;
+    IL_CUDA(cudaMemcpyAsync(e->d_cfg, configs, (size_t)total * sizeof(il_stage_config),
+                            cudaMemcpyHostToDevice, e->stream));
+    // the flags go behind the two output arrays of the staging (which the warp-per-candidate
+    // kernels fill with P99 and misses first)
+    uint8_t *d_flags = reinterpret_cast<uint8_t *>(e->d_out + 2 * e->d_out_cap);
+    rc = il_feasible_device(e, e->d_cfg, n_cand, slo_us, d_flags);
+    if (rc) return rc;
+    IL_CUDA(cudaMemcpyAsync(out_feasible, d_flags, (size_t)n_cand, cudaMemcpyDeviceToHost, e->stream));
     IL_CUDA(cudaStreamSynchronize(e->stream));
     return IL_OK;
 }

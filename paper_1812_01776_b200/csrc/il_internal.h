@@ -42,6 +42,17 @@ struct DesParams {
     int64_t lane_elems;           // stream records per candidate: every stage's arrival stream but the root's
     int32_t lane_off[IL_MAX_STAGES]; // record offset of stage s's arrival stream inside a candidate's block
     int32_t cpw;                  // candidates per warp, floor(32 / S)
+    int32_t lane_ring_log2;       // a stream ring holds 2^this records
+    int32_t lane_wrap;            // the rings are shorter than the longest stream: positions wrap
+    uint8_t *ovf;                 // [n_cand] set to 1 for a candidate given up on ring overflow (lane_wrap only)
+    // lane kernel, feasibility only: set out_feasible to select that instantiation
+    uint8_t *out_feasible;        // [n_cand] 1: P99 <= slo_us, 0: not, 2: given up on ring overflow (see ovf)
+    int64_t slo_us;               // the objective, clamped by the host to 0 .. 2^(62 - qbits)
+    uint32_t miss_allow;          // n - ceil(0.99 n): a candidate with more misses than this is infeasible
+    // all simulation kernels
+    unsigned long long iter_limit;   // iteration bound of a device loop; 0 = the bound the loop derives itself
+    const unsigned long long *n_cand_dev;   // if set, the number of candidates is read from here (device
+                                            // memory) instead of n_cand: the list in `order` was built on the device
 };
 
 struct SelectParams {
@@ -55,6 +66,8 @@ struct SelectParams {
     int32_t n_regions;            // 0: not known
     int32_t region_end[IL_MAX_STAGES];   // one past the last record of each non-empty region
     const uint64_t *lat_or;       // [n_cand]: OR of the latencies (wide kernel)
+    const uint8_t *ovf;           // if set: candidates whose row does not have the region layout (they were
+                                  // evaluated by the warp-per-candidate kernel after a ring overflow)
     int32_t n;
     int64_t n_cand;
     int64_t slo_us;
@@ -112,6 +125,12 @@ struct OrderParams {
     int32_t *order;                  // [n_cand] out
 };
 cudaError_t launch_order(const OrderParams &p, cudaStream_t stream);
+cudaError_t launch_gather_configs(const il_stage_config *configs, const int32_t *list, int64_t count, int S,
+                                  il_stage_config *out, cudaStream_t stream);
+cudaError_t launch_feasible_from_p99(const int64_t *p99, const int32_t *list, int64_t count, int64_t slo_us,
+                                     uint8_t *out, cudaStream_t stream);
+cudaError_t launch_overflow_list(const uint8_t *ovf, int64_t n_cand, int32_t *order, unsigned long long *counters,
+                                 cudaStream_t stream);
 int des_max_ctas_per_sm(size_t smem);
 cudaError_t launch_envelope(const int64_t *d_arrival, int n, const int64_t *h_windows, int n_windows,
                             int *d_out, int num_sms, cudaStream_t stream);

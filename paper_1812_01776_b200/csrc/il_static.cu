@@ -76,7 +76,7 @@ static int enqueue_static(const BoundView &v, unsigned char *base, const il_stag
     IL_ST(launch_order(op, st));
     IL_ST(launch_simulation(p, v.kernel, (int)(slots / kWarpsPerCta), v.smem, st));
 
-    SelectParams sp;
+    SelectParams sp = {};
     sp.slab = p.slab; sp.slab_stride = v.n_pad; sp.lat_or = p.lat_or;
     sp.arrival = p.arrival; sp.qbits = p.qbits; sp.packed = v.kernel != kSimWide ? 1 : 0;
     sp.n_regions = 0;

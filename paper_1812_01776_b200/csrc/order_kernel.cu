@@ -10,6 +10,8 @@
 // mean arrival rate; it only affects the order, never a result.
 #include "il_internal.h"
 
+#include <algorithm>
+
 namespace il {
 
 namespace {
@@ -63,7 +65,65 @@ __global__ void __launch_bounds__(kOrderThreads) order_kernel(const __grid_const
     }
 }
 
+// Candidates the lane kernel gave up on (ring overflow), as a list for the warp-per-candidate
+// kernel: order[0 .. count) in any order, count to counters[3] (and added to counters[4]); the
+// work counter counters[0] is cleared for the kernel that follows.
+__global__ void __launch_bounds__(1024) overflow_list_kernel(const uint8_t *ovf, int64_t n_cand, int32_t *order,
+                                                            unsigned long long *counters)
+{
+    __shared__ unsigned count;
+    if (threadIdx.x == 0) count = 0;
+    __syncthreads();
+    for (int64_t c = threadIdx.x; c < n_cand; c += blockDim.x)
+        if (ovf[c]) order[atomicAdd(&count, 1u)] = (int32_t)c;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        counters[3] = count;
+        counters[4] += count;
+        counters[0] = 0;
+    }
+}
+
+// configs of the listed candidates, packed one after the other
+__global__ void gather_configs_kernel(const il_stage_config *configs, const int32_t *list, int64_t count, int S,
+                                      il_stage_config *out)
+{
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < count * S; i += (int64_t)gridDim.x * blockDim.x)
+        out[i] = configs[(int64_t)list[i / S] * S + i % S];
+}
+
+// Feasible (Section 4.3): P99 <= objective.  With a list, entry i belongs to candidate list[i].
+__global__ void feasible_from_p99_kernel(const int64_t *p99, const int32_t *list, int64_t count, int64_t slo_us,
+                                         uint8_t *out)
+{
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
+        out[list ? list[i] : i] = p99[i] <= slo_us ? 1 : 0;
+}
+
 }  // namespace
+
+cudaError_t launch_gather_configs(const il_stage_config *configs, const int32_t *list, int64_t count, int S,
+                                  il_stage_config *out, cudaStream_t stream)
+{
+    const int grid = (int)std::min<int64_t>((count * S + 255) / 256, 1184);
+    gather_configs_kernel<<<grid, 256, 0, stream>>>(configs, list, count, S, out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_feasible_from_p99(const int64_t *p99, const int32_t *list, int64_t count, int64_t slo_us,
+                                     uint8_t *out, cudaStream_t stream)
+{
+    const int grid = (int)std::min<int64_t>((count + 255) / 256, 1184);
+    feasible_from_p99_kernel<<<grid, 256, 0, stream>>>(p99, list, count, slo_us, out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_overflow_list(const uint8_t *ovf, int64_t n_cand, int32_t *order, unsigned long long *counters,
+                                 cudaStream_t stream)
+{
+    overflow_list_kernel<<<1, 1024, 0, stream>>>(ovf, n_cand, order, counters);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_order(const OrderParams &p, cudaStream_t stream)
 {

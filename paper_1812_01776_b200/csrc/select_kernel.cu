@@ -37,7 +37,7 @@ select_kernel(const __grid_constant__ SelectParams p)
         unsigned miss = 0;
         bool counted_miss = false;
         uint64_t bits_used;
-        if (p.packed && p.n_regions > 0) {
+        if (p.packed && p.n_regions > 0 && !(p.ovf && p.ovf[c])) {
             uint64_t last = 0;
 #pragma unroll
             for (int r = 0; r < IL_MAX_STAGES; r++)      // unrolled: constant indices into the parameter block

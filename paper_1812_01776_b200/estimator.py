@@ -24,11 +24,13 @@ IL_ERR_BAD_CONFIG, IL_ERR_NOMEM, IL_ERR_CUDA, IL_ERR_ITER_LIMIT = -5, -6, -7, -8
 IL_ERR_TOO_LARGE = -9
 IL_VARIANT_AUTO, IL_VARIANT_WIDE, IL_VARIANT_STAGED, IL_VARIANT_LANES, IL_VARIANT_PACKED = 0, 1, 2, 3, 4
 IL_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
+IL_KNOB_LANE_RING_LOG2, IL_KNOB_ITER_LIMIT = 1, 2
 
 EXPORTS = ["il_estimator_create", "il_estimator_destroy", "il_estimate", "il_estimate_device",
            "il_set_stream", "il_workspace_bytes", "il_workspace_min_bytes", "il_set_workspace",
            "il_get_stats", "il_stage_visits", "il_strerror", "il_last_cuda_error",
-           "il_measure_int_issue", "il_estimate_device_static", "il_set_variant", "il_estimate_latencies", "il_traffic_envelope", "il_kernel_name"]
+           "il_measure_int_issue", "il_estimate_device_static", "il_set_variant", "il_estimate_latencies", "il_traffic_envelope", "il_kernel_name",
+           "il_set_test_knob", "il_feasible", "il_feasible_device"]
 
 
 class ILError(RuntimeError):
@@ -63,7 +65,9 @@ class Stats(ctypes.Structure):
                 ("batches", ctypes.c_int64), ("algorithmic_ops", ctypes.c_int64),
                 ("chunks", ctypes.c_int64),
                 ("kernel_launches", ctypes.c_int64), ("sim_ms", ctypes.c_double),
-                ("select_ms", ctypes.c_double), ("total_ms", ctypes.c_double)]
+                ("select_ms", ctypes.c_double), ("total_ms", ctypes.c_double),
+                ("fallback_candidates", ctypes.c_int64), ("stage_runs", ctypes.c_int64),
+                ("error_detail", ctypes.c_int64), ("early_exits", ctypes.c_int64)]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}
@@ -92,6 +96,10 @@ def load_library():
     lib.il_estimate.argtypes = [vp, vp, i64, i64, vp, vp]
     lib.il_estimate_device.restype = ctypes.c_int
     lib.il_estimate_device.argtypes = [vp, vp, i64, i64, vp, vp]
+    lib.il_feasible.restype = ctypes.c_int
+    lib.il_feasible.argtypes = [vp, vp, i64, i64, vp]
+    lib.il_feasible_device.restype = ctypes.c_int
+    lib.il_feasible_device.argtypes = [vp, vp, i64, i64, vp]
     lib.il_estimate_device_static.restype = ctypes.c_int
     lib.il_estimate_device_static.argtypes = [vp, vp, i64, i64, vp, vp]
     lib.il_estimate_latencies.restype = ctypes.c_int
@@ -104,6 +112,8 @@ def load_library():
     lib.il_set_variant.argtypes = [vp, ctypes.c_int]
     lib.il_set_stream.restype = ctypes.c_int
     lib.il_set_stream.argtypes = [vp, vp]
+    lib.il_set_test_knob.restype = ctypes.c_int
+    lib.il_set_test_knob.argtypes = [vp, ctypes.c_int, i64]
     lib.il_workspace_bytes.restype = ctypes.c_int
     lib.il_workspace_bytes.argtypes = [vp, i64, ctypes.POINTER(ctypes.c_size_t)]
     lib.il_workspace_min_bytes.restype = ctypes.c_int
@@ -189,6 +199,23 @@ def il_estimate_device(handle, d_configs: int, n: int, slo_us: int, d_out_p99: i
                                              d_out_miss), "il_estimate_device")
 
 
+def il_feasible(handle, configs: np.ndarray, slo_us: int) -> np.ndarray:
+    """il_feasible: host configs [n][S][4] uint8 in, host bool array out (P99 <= slo_us)."""
+    configs = np.ascontiguousarray(configs, dtype=np.uint8)
+    if configs.ndim != 3 or configs.shape[2] != 4:
+        raise ValueError("configs must be [n][S][4] uint8")
+    out = np.empty(configs.shape[0], dtype=np.uint8)
+    _check(load_library().il_feasible(handle, configs.ctypes.data, configs.shape[0], int(slo_us),
+                                      out.ctypes.data), "il_feasible")
+    return out.astype(bool)
+
+
+def il_feasible_device(handle, d_configs: int, n: int, slo_us: int, d_out_feasible: int) -> None:
+    """il_feasible_device: raw device pointers (ints) in, one byte per candidate written in place."""
+    _check(load_library().il_feasible_device(handle, d_configs, int(n), int(slo_us), d_out_feasible),
+           "il_feasible_device")
+
+
 def il_estimate_device_static(handle, d_configs: int, n: int, slo_us: int, d_out_p99: int,
                               d_out_miss: int) -> None:
     """il_estimate_device_static: like il_estimate_device, but the library
@@ -214,6 +241,11 @@ def il_traffic_envelope(handle, window_us) -> np.ndarray:
 
 def il_set_variant(handle, variant: int) -> None:
     _check(load_library().il_set_variant(handle, int(variant)), "il_set_variant")
+
+
+def il_set_test_knob(handle, knob: int, value: int) -> None:
+    """il_set_test_knob: hooks for the tests (ring length of the lane kernel, iteration bound)."""
+    _check(load_library().il_set_test_knob(handle, int(knob), int(value)), "il_set_test_knob")
 
 
 def il_kernel_name(handle) -> str:
@@ -327,6 +359,12 @@ class Estimator:
     def kernel_name(self) -> str:
         return il_kernel_name(self._h)
 
+    def set_test_knob(self, knob: int, value: int) -> None:
+        """Test hook (IL_KNOB_*); invalidates a workspace reserved earlier."""
+        il_set_workspace(self._h, 0, 0)
+        self._ws = None
+        il_set_test_knob(self._h, knob, value)
+
     def use_current_stream(self) -> None:
         il_set_stream(self._h, self._torch.cuda.current_stream(self.device).cuda_stream)
 
@@ -347,6 +385,21 @@ class Estimator:
         il_estimate_device(self._h, d_configs.data_ptr(), n, slo_us, out_p99.data_ptr(),
                            out_miss.data_ptr())
         return out_p99, out_miss
+
+    def feasible(self, configs: np.ndarray, slo_us: int) -> np.ndarray:
+        """Host arrays in and out: True where the candidate meets the objective at P99."""
+        return il_feasible(self._h, configs, slo_us)
+
+    def feasible_device(self, d_configs, slo_us: int, out=None):
+        """torch uint8 tensor [n][S][4] on the device in, uint8 tensor [n] out (1 = feasible)."""
+        torch = self._torch
+        assert d_configs.is_cuda and d_configs.dtype == torch.uint8 and d_configs.is_contiguous()
+        assert d_configs.dim() == 3 and d_configs.shape[1] == self.n_stages and d_configs.shape[2] == 4
+        n = d_configs.shape[0]
+        if out is None:
+            out = torch.empty(n, dtype=torch.uint8, device=d_configs.device)
+        il_feasible_device(self._h, d_configs.data_ptr(), n, slo_us, out.data_ptr())
+        return out
 
     def latencies(self, config: np.ndarray):
         """Per-query latencies (int64 numpy array, trace order) of one candidate [S][4]."""

@@ -59,6 +59,7 @@ class PlanResult:
     estimator_calls: int                  # batched calls made
     candidates_evaluated: int             # configurations simulated in total
     steps: List[str]                      # what was done, in order
+    trajectory: List[np.ndarray] = None   # configuration after Initialize and after every accepted action
 
 
 class Planner:
@@ -189,7 +190,8 @@ class Planner:
         steps: List[str] = []
         cfg = self.initialize(steps)
         if cfg is None:
-            return PlanResult(False, None, float("inf"), -1, self.calls, self.evaluated, steps)
+            return PlanResult(False, None, float("inf"), -1, self.calls, self.evaluated, steps, [])
+        trajectory = [cfg.copy()]
         while True:
             cands, labels = [], []
             for s in range(self.S):
@@ -213,10 +215,11 @@ class Planner:
             if best is None:
                 break
             cfg = cands[best]
+            trajectory.append(cfg.copy())
             steps.append(f"{labels[best]} -> cost {self.cost(cfg):.4f}")
         ok, p99 = self.feasible_many(cfg[None])
         assert ok[0]
-        return PlanResult(True, cfg, self.cost(cfg), int(p99[0]), self.calls, self.evaluated, steps)
+        return PlanResult(True, cfg, self.cost(cfg), int(p99[0]), self.calls, self.evaluated, steps, trajectory)
 
     def single_actions(self, cfg: np.ndarray) -> List[np.ndarray]:
         """All configurations one action away (used to check the termination guarantee)."""

@@ -26,3 +26,21 @@ def oracle_pool(oracle):
     pool = oracle.make_pool()
     yield pool
     pool.terminate()
+
+
+_ORACLE_RESULTS = {}
+
+
+@pytest.fixture(scope="session")
+def oracle_on(oracle, oracle_pool):
+    """oracle_on(key, w, configs) -> (p99, miss) of the oracle for `configs` on workload w, computed
+    once per session and key (the full-size samples take minutes of CPU time)."""
+    import numpy as np
+
+    def run(key, w, configs):
+        if key not in _ORACLE_RESULTS:
+            _ORACLE_RESULTS[key] = oracle.estimate_many_parallel(
+                w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us, w.branch_bits,
+                np.ascontiguousarray(configs), w.slo_us, pool=oracle_pool)
+        return _ORACLE_RESULTS[key]
+    return run

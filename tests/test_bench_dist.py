@@ -72,3 +72,37 @@ def test_reduce_helpers_without_process_group():
     import bench
     assert bench.reduce_max([1.0, 2.0]) == [1.0, 2.0]
     assert bench.reduce_sum([3.0]) == [3.0]
+
+
+def test_shard_range_partitions_exactly():
+    from paper_1812_01776_b200 import shard_range
+    for total in (0, 1, 7, 64, 4096, 1_048_577):
+        for world in (1, 2, 3, 8):
+            cuts = [shard_range(total, r, world) for r in range(world)]
+            assert cuts[0][0] == 0 and cuts[-1][1] == total
+            assert all(cuts[r][1] == cuts[r + 1][0] for r in range(world - 1))
+            sizes = [hi - lo for lo, hi in cuts]
+            assert max(sizes) - min(sizes) <= 1 and sizes == sorted(sizes, reverse=True)
+    with pytest.raises(ValueError):
+        shard_range(10, 2, 2)
+
+
+@pytest.mark.gpu
+def test_sharded_estimator_on_the_visible_devices(oracle):
+    """The package's sharded call on however many devices this process sees (one is fine):
+    results in candidate order, equal to the oracle's."""
+    import torch
+    import workloads
+    import paper_1812_01776_b200 as il
+    w = workloads.make(3, n_queries=2500, n_candidates=101)
+    exp = oracle.estimate_workload(w)
+    with il.ShardedEstimator.from_workload(w) as sh:
+        assert len(sh.shards) == torch.cuda.device_count()
+        p99, miss = sh.estimate(w.configs, w.slo_us)
+        assert np.array_equal(p99, exp[0]) and np.array_equal(miss, exp[1])
+        assert sum(s["candidates"] for s in sh.stats()) == 101
+    # the same through two handles on one device: the split and the reassembly are what is tested
+    with il.ShardedEstimator.from_workload(w, devices=[0, 0]) as sh:
+        p99, miss = sh.estimate(w.configs, w.slo_us)
+        assert np.array_equal(p99, exp[0]) and np.array_equal(miss, exp[1])
+        assert [s["candidates"] for s in sh.stats()] == [51, 50]

@@ -30,6 +30,23 @@ def test_oracle_against_brute_force(oracle, seed):
     assert got[0] == np.bincount(a).max() and got[-1] == len(a)
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_oracle_against_every_integer_window_start(oracle, seed):
+    """The definition itself on a tiny trace: every half-open window [t, t + w) for EVERY integer
+    start t (not only starts at an arrival, which is the reduction the oracle relies on), counted
+    one arrival at a time."""
+    rng = np.random.default_rng(100 + seed)
+    a = np.sort(rng.integers(5, 160, size=int(rng.integers(20, 50)))).astype(np.int64)
+    wins = np.array([1, 2, 3, 5, 8, 13, 40, 155, 156, 400], np.int64)
+    exp = []
+    for w in wins:
+        best = 0
+        for t in range(int(a[0]) - int(w) - 1, int(a[-1]) + 2):
+            best = max(best, sum(1 for x in a if t <= x < t + w))
+        exp.append(best)
+    assert oracle.traffic_envelope(a, wins).tolist() == exp
+
+
 def test_oracle_rejects_bad_input(oracle):
     with pytest.raises(oracle.OracleError):
         oracle.traffic_envelope(np.array([5, 4], np.int64), [10])

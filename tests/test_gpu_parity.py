@@ -22,12 +22,14 @@ def il():
     return il_
 
 
-def gpu_run(il, w, configs=None, slo=None, host=True, ws_bytes=None, variant=0):
+def gpu_run(il, w, configs=None, slo=None, host=True, ws_bytes=None, variant=0, knobs=None):
     import torch
     configs = w.configs if configs is None else configs
     slo = w.slo_us if slo is None else slo
     with il.Estimator.from_workload(w) as est:
         est.set_variant(variant)
+        for knob, value in (knobs or {}).items():
+            est.set_test_knob(knob, value)
         if ws_bytes is not None:
             est.reserve_workspace(len(configs), max_bytes=ws_bytes)
         if host:
@@ -131,6 +133,35 @@ def test_sparse_traces_move_the_epoch(il, oracle, seed, variant):
     check(il, oracle, w, variant=variant)
 
 
+@pytest.mark.parametrize("ring_log2", [6, 8, 10])
+@pytest.mark.parametrize("seed", range(12))
+def test_lane_kernel_short_stream_rings(il, oracle, seed, ring_log2):
+    """Stream rings of 64 / 256 / 1,024 records on traces of 700 to 1,100 queries: ring positions wrap,
+    parents wait for room, and candidates whose oldest batch in flight pins more than a ring are
+    handed to the warp-per-candidate kernel.  Results must not change."""
+    w = workloads.random_small(seed, S=1 + seed % 6, H=3, Bmax=[4, 33, 64][seed % 3], n=700 + 37 * seed,
+                               C=40, max_replicas=[3, 8, 32][seed % 3], tree=(seed % 2 == 1),
+                               qps=400.0, cv=3.0, lat_lo=1, lat_hi=20000,
+                               equal_stamp_every=(3 if seed % 4 == 0 else 0))
+    check(il, oracle, w, host=(seed % 2 == 0), variant=3, knobs={1: ring_log2})
+
+
+@pytest.mark.parametrize("cid,n,C", [(2, 5000, 300), (3, 6001, 200), (4, 3000, 150), (5, 4097, 260)])
+def test_configs_reduced_short_stream_rings(il, oracle, cid, n, C):
+    """The five workload shapes with 256-record rings: with the workloads' affine tables most
+    candidates finish on the lane kernel, the others take the overflow path."""
+    st = check(il, oracle, workloads.make(cid, n_queries=n, n_candidates=C), host=False, variant=3, knobs={1: 8})
+    assert 0 <= st["fallback_candidates"] <= C
+
+
+def test_default_rings_rarely_overflow(il, oracle):
+    """With the default ring length (8,192 records) and the workloads' tables, a trace far longer
+    than a ring runs on the lane kernel alone."""
+    w = workloads.make(2, n_queries=40000, n_candidates=192)
+    st = check(il, oracle, w, host=False)
+    assert st["fallback_candidates"] <= 2
+
+
 def test_config1_full(il, oracle):
     st = check(il, oracle, workloads.make(1))
     # the lane kernel needs no ordering pass: (simulate, select) or (order, simulate, select) per chunk
@@ -228,16 +259,25 @@ def test_repeatable_and_stream(il, oracle):
                 assert np.array_equal(b.cpu().numpy(), exp[1])
 
 
-_ORACLE_CACHE = {}
-
-
-def _oracle_on(oracle, pool, key, w, configs):
-    """Oracle results for `configs`, computed once per test session and key."""
-    if key not in _ORACLE_CACHE:
-        _ORACLE_CACHE[key] = oracle.estimate_many_parallel(
-            w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us, w.branch_bits,
-            np.ascontiguousarray(configs), w.slo_us, pool=pool)
-    return _ORACLE_CACHE[key]
+def full_size_sample(cid):
+    """The candidates of workloads 2-5 that the full-size tests check against the oracle: the workload
+    the GPU runs, the indices (into its candidates) that are checked, and the extremes checked beside
+    them.  Workload 2: all 4,096.  Workload 3: a seeded 4,096 of 65,536.  Workload 5: a seeded 1,024 of
+    1,048,576.  Workload 4: every 16th (1,024) of the seeded 16,384-candidate sample the bench times,
+    itself drawn from the whole set of 262,144."""
+    if cid == 2:
+        w = workloads.make(2)
+        return w, np.arange(w.n_candidates), _extremes(4, 3, (1, 32), (1, 8))
+    if cid == 3:
+        w = workloads.make(3)
+        return w, np.sort(np.random.default_rng(3).choice(w.n_candidates, size=4096, replace=False)), \
+            _extremes(6, 3, (1, 64), (1, 8))
+    if cid == 5:
+        w = workloads.make(5)
+        return w, np.sort(np.random.default_rng(5).choice(w.n_candidates, size=1024, replace=False)), \
+            _extremes(8, 4, (1, 64), (1, 32))
+    w, _ = workloads.sub_batch(4, 16384)
+    return w, np.arange(0, w.n_candidates, 16), _extremes(10, 4, (1, 64), (1, 16))
 
 
 def _extremes(S, H, mbs, Rs):
@@ -273,26 +313,15 @@ def _properties(w, p99, miss):
     assert (p99 > 0).all() and (miss >= 0).all() and (miss <= w.n_queries).all()
 
 
-@pytest.mark.parametrize("variant", [0, 4], ids=["auto", "packed"])
-def test_config2_full_size_all_4096(il, oracle, oracle_pool, variant):
-    """Workload 2 in full: ALL 4,096 candidates x 50,000 queries against the oracle,
-    plus 12 structured extremes (every hardware type, 1 / 8 replicas, max batch 1 / 32)."""
-    w = workloads.make(2)
-    ext = _extremes(4, 3, (1, 32), (1, 8))
-    exp = _oracle_on(oracle, oracle_pool, "w2", w, np.concatenate([w.configs, ext]))
-    p99, miss = _run_all(il, w, variant)
-    e = gpu_run(il, w, configs=ext, host=True, variant=variant)
-    got = (np.concatenate([p99, e[0]]), np.concatenate([miss, e[1]]))
-    _assert_equal(w, got, exp, np.concatenate([w.configs, ext]))
-    _properties(w, p99, miss)
-
-
-def _sampled_check(il, oracle, pool, key, w, idx, extremes, variant=0):
-    """All candidates of w on the GPU; the candidates idx of w plus the extremes
-    against the oracle one by one; the size-free properties on all."""
-    ext = np.ascontiguousarray(extremes, dtype=np.uint8)
+def _sampled_check(il, oracle_on, cid, variant=0, gpu_subset_only=False):
+    """All candidates of the workload on the GPU; the sampled candidates plus the extremes against
+    the oracle one by one; the size-free properties on all."""
+    w, idx, ext = full_size_sample(cid)
     both = np.concatenate([w.configs[idx], ext])
-    exp = _oracle_on(oracle, pool, key, w, both)
+    exp = oracle_on(f"w{cid}", w, both)
+    if gpu_subset_only:
+        w.configs = np.ascontiguousarray(w.configs[idx])
+        idx = np.arange(w.n_candidates)
     p99, miss = _run_all(il, w, variant)
     e = gpu_run(il, w, configs=ext, host=True, variant=variant)
     got = (np.concatenate([p99[idx], e[0]]), np.concatenate([miss[idx], e[1]]))
@@ -300,35 +329,33 @@ def _sampled_check(il, oracle, pool, key, w, idx, extremes, variant=0):
     _properties(w, p99, miss)
 
 
-def test_config3_full_size_sample_4096(il, oracle, oracle_pool):
+@pytest.mark.parametrize("variant", [0, 4], ids=["auto", "packed"])
+def test_config2_full_size_all_4096(il, oracle_on, variant):
+    """Workload 2 in full: ALL 4,096 candidates x 50,000 queries against the oracle,
+    plus 12 structured extremes (every hardware type, 1 / 8 replicas, max batch 1 / 32)."""
+    _sampled_check(il, oracle_on, 2, variant)
+
+
+def test_config3_full_size_sample_4096(il, oracle_on):
     """All 65,536 candidates x 200,000 queries of the 6-stage tree on the GPU; a seeded
     sample of 4,096 candidates and 12 extremes against the oracle."""
-    w = workloads.make(3)
-    idx = np.sort(np.random.default_rng(3).choice(w.n_candidates, size=4096, replace=False))
-    _sampled_check(il, oracle, oracle_pool, "w3", w, idx, _extremes(6, 3, (1, 64), (1, 8)))
+    _sampled_check(il, oracle_on, 3)
 
 
-def test_config5_full_size_sample_1024(il, oracle, oracle_pool):
+def test_config5_full_size_sample_1024(il, oracle_on):
     """All 1,048,576 candidates x 100,000 queries of the 8-stage tree (R up to 32, max batch up
     to 64) on the GPU; a seeded sample of 1,024 candidates and 16 extremes against the oracle."""
-    w = workloads.make(5)
-    idx = np.sort(np.random.default_rng(5).choice(w.n_candidates, size=1024, replace=False))
-    _sampled_check(il, oracle, oracle_pool, "w5", w, idx, _extremes(8, 4, (1, 64), (1, 32)))
+    _sampled_check(il, oracle_on, 5)
 
 
 @pytest.mark.parametrize("variant", [0, 4], ids=["auto", "packed"])
-def test_config4_full_trace_sample_1024(il, oracle, oracle_pool, variant):
+def test_config4_full_trace_sample_1024(il, oracle_on, variant):
     """The 10-stage pipeline on its full 1,000,000-query trace.  The whole sweep is 262,144
     candidates (2.6e12 query-events, minutes of GPU time), so the GPU runs the seeded
     16,384-candidate sub-batch the bench times, drawn from the WHOLE candidate set; 1,024 of
     those (every 16th) and 16 extremes are checked against the oracle.  The warp-per-candidate
     kernel runs the 1,024 checked candidates only."""
-    w, _ = workloads.sub_batch(4, 16384)
-    idx = np.arange(0, w.n_candidates, 16)
-    if variant != 0:
-        w.configs = np.ascontiguousarray(w.configs[idx])
-        idx = np.arange(w.n_candidates)
-    _sampled_check(il, oracle, oracle_pool, "w4", w, idx, _extremes(10, 4, (1, 64), (1, 16)), variant=variant)
+    _sampled_check(il, oracle_on, 4, variant, gpu_subset_only=(variant != 0))
 
 
 @pytest.mark.parametrize("variant", [3, 4, 1], ids=["lanes", "packed", "wide"])
@@ -351,8 +378,7 @@ def test_percentile_kernel_on_chosen_latency_multisets(il, oracle, case, variant
 
 
 def test_kernel_choice(il):
-    """The default picks the lane kernel while a candidate's inter-stage streams are small, the
-    warp-per-candidate packed kernel beyond, and the wide kernel when times do not fit a record."""
+    """The default picks the lane kernel, and the wide kernel when times do not fit a record."""
     from paper_1812_01776_b200 import estimator as E
     w = workloads.make(2, n_queries=5000, n_candidates=4)
     with il.Estimator.from_workload(w) as est:
@@ -366,10 +392,8 @@ def test_kernel_choice(il):
         assert est.kernel_name() == "des_kernel"
         est.set_variant(E.IL_VARIANT_LANES)
         assert est.kernel_name() == "des_kernel"
-    w = workloads.make(4, n_queries=2_000_000, n_candidates=2)   # 18 x 10^6 stream records per candidate
-    with il.Estimator.from_workload(w) as est:
-        assert est.kernel_name() == "des_packed_kernel"
-        est.set_variant(E.IL_VARIANT_LANES)
+    w = workloads.make(4, n_queries=2_000_000, n_candidates=2)   # 18 x 10^6 stream records per candidate:
+    with il.Estimator.from_workload(w) as est:                   # the lane kernel's rings do not grow with that
         assert est.kernel_name() == "des_lane_kernel"
 
 

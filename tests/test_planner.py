@@ -95,6 +95,87 @@ def test_tuner_handoff_with_the_oracle(oracle):
     assert np.array_equal(envelope_windows(1000)[:3], [1000, 2000, 4000])
 
 
+def tree_workload():
+    # 5-stage tree: 0 -> {1 (bit 0 = 0), 2 (bit 0 = 1)}; 1 -> 3; 2 -> 4 guarded by bit 1 (a cascade)
+    w = workloads.random_small(21, S=5, H=3, Bmax=16, n=1200, C=1, qps=180.0, cv=2.0, tree=True)
+    w.parent = np.array([-1, 0, 0, 1, 2], np.int32)
+    w.cond_bit = np.array([-1, 0, 0, -1, 1], np.int8)
+    w.cond_val = np.array([0, 0, 1, 0, 1], np.uint8)
+    b = np.arange(1, 17)
+    lat = np.zeros((5, 3, 16), np.int32)
+    rng = np.random.default_rng(5)
+    for s in range(5):
+        a0, c0 = rng.integers(3000, 9000), rng.integers(150, 500)
+        lat[s, 0] = a0 + c0 * b                       # accelerator-like
+        lat[s, 1] = a0 * 1.3 + c0 * 3 * b             # mid
+        lat[s, 2] = a0 * 0.6 + c0 * 12 * b            # CPU-like
+    w.latency_us = lat
+    return w, np.array([0.90, 0.40, 0.06])
+
+
+def two_stage_workload():
+    w = workloads.random_small(11, S=2, H=2, Bmax=4, n=600, C=1, qps=120.0, cv=1.0)
+    b = np.arange(1, 5)
+    w.latency_us = np.stack([np.stack([5000 + 400 * b, 3000 + 3500 * b]),
+                             np.stack([8000 + 600 * b, 6000 + 7000 * b])]).astype(np.int32)
+    return w, np.array([1.0, 0.1])
+
+
+@pytest.mark.parametrize("make,slo", [(small_workload, 60_000), (small_workload, 35_000), (tree_workload, 80_000),
+                                      (tree_workload, 40_000), (two_stage_workload, 20_000),
+                                      (two_stage_workload, 45_000), (small_workload, 9_000)])
+def test_batched_planner_equals_the_sequential_algorithms(oracle, make, slo):
+    """The Planner batches its questions; Algorithms 1 and 2 written out in the paper's listing
+    order, asking one Feasible question at a time (oracle/planner_sequential.py), must reach the
+    same plan through the same sequence of accepted actions."""
+    from oracle.planner_sequential import SequentialPlanner
+    w, prices = make()
+    visits = w.visits_per_stage()
+
+    def feasible_one(cfg):
+        p99, _, = oracle.estimate_one(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us,
+                                      w.branch_bits, cfg, slo)
+        return p99 <= slo
+
+    seq = SequentialPlanner(w.parent, w.latency_us, visits, prices, slo, feasible_one)
+    want = seq.minimize_cost()
+    got = Planner(w.parent, w.latency_us, visits, prices, slo, oracle_fn(oracle, w, slo)).minimize_cost()
+    assert got.feasible == (want is not None)
+    if want is not None:
+        assert np.array_equal(got.config, want)
+        assert len(got.trajectory) == len(seq.trajectory)
+        for a, b_ in zip(got.trajectory, seq.trajectory):
+            assert np.array_equal(a, b_)
+        assert got.cost == pytest.approx(seq.cost(want))
+        # one question at a time costs many more estimator calls than the batched Planner makes
+        assert seq.questions >= got.estimator_calls
+
+
+def test_tuner_handoff_on_a_hand_computed_case():
+    """Section 5, initialisation: rho_m = lambda * s_m / (k_m * mu_m), mu_m the throughput of one
+    replica at the planned batch size.  Two models: the trace has 1,001 arrivals over 10 s
+    (lambda = 100.1 per second); model 0 sees every query, model 1 a quarter of them.
+    Model 0: batch 4 takes 20 ms -> mu = 200 per second, 2 replicas -> rho = 100.1 / 400 = 0.25025.
+    Model 1: batch 1 takes 8 ms  -> mu = 125 per second, 1 replica -> rho = 25.025 / 125 = 0.2002."""
+    from paper_1812_01776_b200.planner import tuner_handoff
+    lat = np.zeros((2, 1, 4), np.int32)
+    lat[0, 0] = [9_000, 12_000, 16_000, 20_000]
+    lat[1, 0] = [8_000, 9_000, 10_000, 11_000]
+    pl = Planner(np.array([-1, 0]), lat, np.array([1001, 250]), [1.0], 100_000, lambda c: None)
+    cfg = np.array([[0, 4, 2, 0], [0, 1, 1, 0]], np.uint8)
+    seen = {}
+
+    def env(windows):
+        seen["w"] = windows
+        return np.arange(1, len(windows) + 1)
+    h = tuner_handoff(pl, cfg, 1001, 10_000_000, env)
+    assert seen["w"][0] == 9_000 + 8_000                      # service time: batch-1 latencies along the path
+    assert h["mu_per_us"] == pytest.approx([200e-6, 125e-6])
+    assert h["scale_factor"] == pytest.approx([1.0, 250 / 1001])
+    assert h["rho"] == pytest.approx([0.25025, 100.1 * (250 / 1001) / 125])
+    assert h["rho"][1] == pytest.approx(0.2)                  # 25 queries per second over 125
+
+
 @pytest.mark.gpu
 def test_planner_same_plan_on_gpu_and_oracle(oracle):
     import torch
@@ -125,7 +206,6 @@ def test_planner_on_the_image_pipeline(oracle):
                      lambda cfgs: est.estimate(cfgs, w.slo_us))
         res = pl.minimize_cost()
     assert res.feasible
-    acts = pl.single_actions(res.config) if False else []   # single_actions re-queries the GPU; use the oracle below
     p99, _ = oracle.estimate_many(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us,
                                   w.branch_bits, res.config[None], w.slo_us)
     assert p99[0] == res.p99_us <= w.slo_us
