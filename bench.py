@@ -57,6 +57,7 @@ NCU_CAPTURES = {
         "dram_bytes_per_query_event": 12.24, "warp_inst_per_query_event": 32.9,
         "summary": "profiles/des_packed_kernel_config2.md"},
 }
+RING_LOG2 = None         # --ring-log2: ring length of the lane kernel's streams, for side measurements
 METRIC = "candidate_configs_per_s"
 UNIT = "candidates/s"
 
@@ -272,6 +273,8 @@ def measure(il, torch, w, dev, stream, flush, steps, warmup, e2e_steps, variant,
     events_per_cand = w.query_events()
     est = il.Estimator.from_workload(w, device=dev.index)
     est.set_variant(variant)
+    if RING_LOG2 is not None:
+        est.set_test_knob(1, RING_LOG2)
     kernel = est.kernel_name()
     ws_bytes = est.reserve_workspace(n_cand)
     cfg_pinned = torch.from_numpy(cfg_host).pin_memory()
@@ -508,7 +511,11 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5, help="host-buffer steps timed (at most --steps)")
     ap.add_argument("--no-per-workload", action="store_true",
                     help="skip the short measurements of the other workloads")
+    ap.add_argument("--ring-log2", type=int, default=None,
+                    help="largest stream ring of the lane kernel, log2 records (side measurements; default 13)")
     args = ap.parse_args()
+    global RING_LOG2
+    RING_LOG2 = args.ring_log2
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -314,12 +314,15 @@ IL_API int il_set_workspace(il_estimator *est, void *d_workspace, size_t bytes);
  * IL_VARIANT_AUTO (default): the lane kernel.
  * IL_VARIANT_LANES: one lane per (candidate, stage); the stages of a candidate
  *   run side by side as a pipeline inside one warp, floor(32 / S) candidates per
- *   warp.  A stage's arrival stream lives in a ring of at most 8,192 records, so
- *   the scratch per resident candidate does not grow with the trace; a parent
- *   stage waits when it would overrun its child's ring.  A candidate in which one
- *   batch stays in flight while more than a ring of later records passes through
- *   the other replicas of its stage cannot be finished that way: it is
- *   evaluated by the IL_VARIANT_PACKED kernel in the same call
+ *   warp; a group of lanes takes its next candidate as soon as it has finished
+ *   one.  While the inter-stage streams of all resident candidates fit 48 GiB
+ *   every stage keeps its whole arrival stream in the workspace.  Beyond that
+ *   (long traces through deep pipelines) a stage's stream lives in a ring of
+ *   8,192 records, so the scratch per resident candidate does not grow with the
+ *   trace, and a parent stage waits when it would overrun its child's ring.  A
+ *   candidate in which one batch stays in flight while more than a ring of later
+ *   records passes through the other replicas of its stage cannot be finished
+ *   that way: it is evaluated by the IL_VARIANT_PACKED kernel in the same call
  *   (il_stats.fallback_candidates counts them).
  * IL_VARIANT_PACKED: one candidate per warp, stages one after the other, replica
  *   slots across the lanes, warp-level primitives for the queue count and the
@@ -342,8 +345,9 @@ IL_API int il_set_variant(il_estimator *est, int variant);
 
 /*
  * Hooks for the library's own tests; not for production use.
- *   IL_KNOB_LANE_RING_LOG2  value 6..24: largest ring length (log2 records) of the lane kernel's
- *                           streams (default 13).  Small rings force the overflow path.
+ *   IL_KNOB_LANE_RING_LOG2  value 6..24: the lane kernel keeps its streams in rings of at most 2^value
+ *                           records whatever the sizes (by default the library chooses between whole
+ *                           streams and rings of 2^13).  Small rings force the overflow path.
  *   IL_KNOB_ITER_LIMIT      value >= 0: iteration bound of the simulation kernels' loops; 0 restores
  *                           the bound each loop derives from its input.  A small bound makes a call
  *                           return IL_ERR_ITER_LIMIT; the handle stays usable.

@@ -89,6 +89,8 @@ des_kernel(const __grid_constant__ DesParams p)
         int64_t *slab = p.slab + c * p.slab_stride;
         int32_t exits = 0;
         uint64_t lat_or = 0;
+        unsigned long long cand_batches = 0;
+        bool over = false;      // more batches than the iteration bound allows: the candidate is given up
 
         for (int s = 0; s < p.S; s++) {
             const int n_in = p.n_s[s];
@@ -213,6 +215,13 @@ des_kernel(const __grid_constant__ DesParams p)
                 if (lane == sel) { fin = kNever; sl_b = 0; }
             }
             __syncwarp();   // order this stage's stream writes before the next stage's reads
+            // the bound is checked between stages, where nothing is half-written
+            cand_batches += (unsigned)guard;
+            if (p.iter_limit && cand_batches > p.iter_limit) {
+                if (lane == 0) atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT);
+                over = true;
+                break;
+            }
         }
 
         // OR-reduce the latencies' bit pattern (tells the select kernel which digits matter)
@@ -220,7 +229,7 @@ des_kernel(const __grid_constant__ DesParams p)
         const uint32_t hi = __reduce_or_sync(full, (uint32_t)(lat_or >> 32));
         if (lane == 0) {
             p.lat_or[c] = ((uint64_t)hi << 32) | lo;
-            if (exits != p.n) atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT);
+            if (!over && exits != p.n) atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT);
         }
     }
     if (lane == 0 && batches) { atomicAdd(&p.counters[1], batches); atomicAdd(&p.counters[2], alg_ops); }

@@ -223,9 +223,9 @@ des_lane_kernel(const __grid_constant__ DesParams p)
     unsigned nb = 0;
     uint32_t guard = 0, guard_hi = 0;        // iteration bound, counted down in 32-bit pieces
     // ring streams: how far the lane's children let it write, what it has told its own parent,
-    // and a new value for that, found at iteration k and published at k + 4 (see below)
+    // and a new value for that, found at one eighth iteration and published at the next
     uint32_t lim_a = 0xffffffffu, lim_b = 0xffffffffu;
-    uint32_t low_pub = 0, low_new = 0, pub_at = 0, e_first = 0;
+    uint32_t low_pub = 0, low_new = 0, e_first = 0;
     bool low_pending = false, aborted = false;
     uint32_t av = 0;             // mailbox word this iteration works with: the one read an iteration ago
     int par = 0;                 // mailbox buffer this iteration publishes into; it reads the other one
@@ -234,6 +234,47 @@ des_lane_kernel(const __grid_constant__ DesParams p)
     for (;;) {
         // ---- every eighth iteration: drop decided candidates, hand finished groups their next candidate
         if ((it & 7u) == 0u) {
+            if (RING && !done) {
+                // parent side: how far the children have moved on, and whether one has given up
+                if (lane_a >= 0) { const uint32_t f = wm.freed[lane_a]; aborted |= f == kAbort; lim_a = f + K; }
+                if (lane_b >= 0) { const uint32_t f = wm.freed[lane_b]; aborted |= f == kAbort; lim_b = f + K; }
+                if (s != 0) {
+                    // Child side: tell the parent how far it may overwrite the ring.  The lane needs every
+                    // record from the first one of any batch it still has to hand on, and from the open
+                    // batch on.  The minimum is taken when half the ring is in use and published eight
+                    // iterations later: copies under way at the time it was taken (records of batches
+                    // already picked up for handing on) have landed by then, and every later copy reads a
+                    // batch that was counted.
+                    const uint32_t written = av & ~kDone;
+                    if (low_pending) {
+                        low_pending = false;
+                        if (low_new > low_pub) {
+                            low_pub = low_new;
+                            wm.freed[lane] = low_pub;
+                        } else if ((av & kDone) == 0u && written - low_pub + kRingSlack >= K &&
+                                   fx + (uint32_t)kLag >= written && head + (uint32_t)b >= fx && epos == lpos &&
+                                   e_left == 0 && vmask == 0u) {
+                            // the ring is full, this lane has nothing left to examine or hand on, and what
+                            // pins the ring is a batch still in flight: parent and child would wait for
+                            // each other for ever.  Give the candidate up.
+                            aborted = true;
+                        }
+                    }
+                    if (written - low_pub >= (K >> 1)) {
+                        uint32_t lo = head;
+                        if (e_left > 0) lo = min(lo, e_first);
+                        for (uint32_t pp = epos; pp != tpos; pp++)
+                            lo = min(lo, (uint32_t)wm.key[pp & (kRing - 1)][lane] & (uint32_t)qmask);
+                        low_new = lo;
+                        low_pending = true;
+                    }
+                }
+                if (aborted) {
+                    p.ovf[c] = 1;
+                    wm.freed[lane] = kAbort;
+                    done = true;
+                }
+            }
             if (FEAS && has && !done && wm.miss[j] > p.miss_allow) done = true;   // same word, same moment: the whole group
             const unsigned dm = __ballot_sync(full, done);
             const bool turn = !exhausted && (dm & group_mask) == group_mask;
@@ -307,7 +348,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                     if (guard == 0u) guard = 0xffffffffu;
                     lim_a = (RING && lane_a >= 0) ? K : 0xffffffffu;
                     lim_b = (RING && lane_b >= 0) ? K : 0xffffffffu;
-                    low_pub = 0; low_new = 0; pub_at = 0; e_first = 0;
+                    low_pub = 0; low_new = 0; e_first = 0;
                     low_pending = false; aborted = false;
                     av = avail0;
                 }
@@ -339,20 +380,9 @@ des_lane_kernel(const __grid_constant__ DesParams p)
             uint64_t k2 = wm.key[(lpos + 1u) & (kRing - 1)][lane];
             const uint32_t written = av & ~kDone;
             const bool pdone = (av & kDone) != 0u;
-            // ring streams: may this lane start handing on another record?  Not while a child's
-            // ring could be overrun by the records under way (rare: the limits are re-read then)
-            bool can_emit = true;
-            if (RING) {
-                can_emit = tail_a + kRingSlack <= lim_a && tail_b + kRingSlack <= lim_b;
-                if (!can_emit) {
-                    const uint32_t fa = lane_a >= 0 ? wm.freed[lane_a] : 0u;
-                    const uint32_t fb = lane_b >= 0 ? wm.freed[lane_b] : 0u;
-                    if ((lane_a >= 0 && fa == kAbort) || (lane_b >= 0 && fb == kAbort)) aborted = true;
-                    lim_a = lane_a >= 0 ? fa + K : 0xffffffffu;
-                    lim_b = lane_b >= 0 ? fb + K : 0xffffffffu;
-                    can_emit = tail_a + kRingSlack <= lim_a && tail_b + kRingSlack <= lim_b;
-                }
-            }
+            // ring streams: may this lane start handing on another record?  Not while a child's ring
+            // could be overrun by the records under way (the limits are refreshed every eighth iteration)
+            const bool can_emit = !RING || (tail_a + kRingSlack <= lim_a && tail_b + kRingSlack <= lim_b);
 
             // ---- examine one record of the arrival stream
             const uint32_t i = head + (uint32_t)b;
@@ -454,42 +484,6 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                 fx++;
             }
             done = end && b == 0 && epos == tpos && e_left == 0 && vmask == 0u;
-            if (RING && s != 0) {
-                // Tell the parent how far it may overwrite the ring.  The lane needs every record
-                // from the first one of any batch it still has to hand on, and from the open batch
-                // on.  The minimum is taken when half the ring is in use and published four
-                // iterations later: copies under way at the time it was taken (records of batches
-                // already picked up for handing on) have landed by then, and every later copy
-                // reads a batch that was counted.
-                if (!low_pending) {
-                    if (written - low_pub >= (K >> 1)) {
-                        uint32_t lo = head;
-                        if (e_left > 0) lo = min(lo, e_first);
-                        for (uint32_t pp = epos; pp != tpos; pp++)
-                            lo = min(lo, (uint32_t)wm.key[pp & (kRing - 1)][lane] & (uint32_t)qmask);
-                        low_new = lo;
-                        low_pending = true;
-                        pub_at = it + 4u;
-                    }
-                } else if (it == pub_at) {
-                    low_pending = false;
-                    if (low_new > low_pub) {
-                        low_pub = low_new;
-                        wm.freed[lane] = low_pub;
-                    } else if (!pdone && written - low_pub + kRingSlack >= K && fx + (uint32_t)kLag >= written &&
-                               i2 >= fx && epos == lpos && e_left == 0 && vmask == 0u) {
-                        // the ring is full, this lane has nothing left to examine or hand on, and
-                        // what pins the ring is a batch still in flight: parent and child would
-                        // wait for each other for ever.  Give the candidate up.
-                        aborted = true;
-                    }
-                }
-            }
-            if (RING && aborted) {
-                p.ovf[c] = 1;
-                wm.freed[lane] = kAbort;
-                done = true;
-            }
             if (--guard == 0) {
                 if (guard_hi == 0) { atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT); atomicOr(&p.counters[5], 1ull); done = true; }
                 else { guard_hi--; }      // guard wraps to 2^32 - 1 on the next decrement

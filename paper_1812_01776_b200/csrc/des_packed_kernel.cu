@@ -858,6 +858,8 @@ __device__ __forceinline__ void simulate_candidate(const DesParams &p, const War
     }
 
     int exits = 0;
+    unsigned long long cand_batches = 0;
+    bool over = false;       // the candidate has dispatched more batches than the iteration bound allows
     for (int s = 0; s < p.S; s++) {
         const int n_in = p.n_s[s];
         if (n_in == 0) continue;
@@ -885,8 +887,17 @@ __device__ __forceinline__ void simulate_candidate(const DesParams &p, const War
         batches += (unsigned)nb;
         alg_ops += 3ull * (unsigned)n_in + (unsigned long long)nb * (unsigned)(R + mb + 4);
         __syncwarp();   // this stage's stream writes are read by the next stage's other lanes
+        // Every stage loop ends by itself (a batch takes at least one query); the bound is checked
+        // between stages, where giving the candidate up leaves nothing half-written behind.
+        cand_batches += (unsigned)nb;
+        if (p.iter_limit && cand_batches > p.iter_limit) {
+            if (lane == 0) atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT);
+            over = true;
+            break;
+        }
     }
-    if (lane == 0 && exits != p.n) { atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT); atomicOr(&p.counters[5], 8ull); }
+    // (the root stage, the only one that reads the staged trace, has been run to its end either way)
+    if (lane == 0 && !over && exits != p.n) { atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT); atomicOr(&p.counters[5], 8ull); }
 }
 
 }  // namespace
@@ -965,6 +976,64 @@ des_packed_kernel(const __grid_constant__ DesParams p)
         __syncthreads();
     }
     if (lane == 0 && batches) { atomicAdd(&p.counters[1], batches); atomicAdd(&p.counters[2], alg_ops); }
+}
+
+// One stage of the shared-prefix evaluation (prefix_kernel.cu): every warp takes nodes of stage
+// p.s from the work counter and runs the stage's queue simulation once per node, from the
+// completion stream of the node's parent (or the trace) to the node's own output streams.
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+des_node_stage_kernel(const __grid_constant__ NodeStageParams p)
+{
+    extern __shared__ int32_t s_row[];     // the stage's profile, [H][Bmax]
+    __shared__ uint64_t s_slot_key[kWarpsPerCta][32];
+    __shared__ uint32_t s_slot_q[kWarpsPerCta][32];
+    __shared__ int s_slot_b[kWarpsPerCta][32];
+    for (int i = threadIdx.x; i < p.H * p.Bmax; i += blockDim.x) s_row[i] = p.lat_stage[i];
+    __syncthreads();
+
+    const unsigned full = 0xffffffffu;
+    const int wid = threadIdx.x >> 5;
+    WarpCtx w;
+    w.lane = threadIdx.x & 31;
+    w.lt_mask = (1u << w.lane) - 1u;
+    w.qbits = p.qbits;
+    w.qmask = (1u << p.qbits) - 1u;
+    w.bits = p.bits;
+    w.slot_key = s_slot_key[wid];
+    w.slot_q = s_slot_q[wid];
+    w.slot_b = s_slot_b[wid];
+    unsigned long long batches = 0, alg_ops = 0;
+    for (;;) {
+        unsigned long long k = 0;
+        if (w.lane == 0) k = atomicAdd(p.work, 1ull);
+        k = __shfl_sync(full, k, 0);
+        if (k >= (unsigned long long)p.n_nodes) break;
+        const uint32_t cfg = p.node_cfg[k];
+        const int hw = (int)(cfg & 0xffu), mb = (int)((cfg >> 8) & 0xffu), R = (int)((cfg >> 16) & 0xffu);
+        Sink sk;
+        sk.bit = p.bit;
+        sk.out_a = p.out_a + (int64_t)k * p.stride_a;
+        sk.out_b = p.out_b + (int64_t)k * p.stride_b;
+        sk.tail_a = 0; sk.tail_b = 0;
+        GlobalSrc src = {p.in ? p.in + (int64_t)p.node_parent[k] * p.stride_in : p.ptrace, p.in == nullptr};
+        const int nb = dispatch_stage(w, s_row + hw * p.Bmax, mb, R, p.n_in, src, sk, p.status);
+        batches += (unsigned)nb;
+        alg_ops += 3ull * (unsigned)p.n_in + (unsigned long long)nb * (unsigned)(R + mb + 4);
+        // every record of the stage must have gone to one of the two sides
+        if (w.lane == 0 && sk.tail_a + sk.tail_b != p.n_in) {
+            atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT);
+            atomicOr(&p.counters[5], 8ull);
+        }
+        __syncwarp();
+    }
+    if (w.lane == 0 && batches) { atomicAdd(&p.counters[1], batches); atomicAdd(&p.counters[2], alg_ops); }
+}
+
+cudaError_t launch_node_stage(const NodeStageParams &p, int grid, cudaStream_t stream)
+{
+    const size_t smem = (size_t)p.H * p.Bmax * sizeof(int32_t);
+    des_node_stage_kernel<<<grid, kWarpsPerCta * 32, smem, stream>>>(p);
+    return cudaGetLastError();
 }
 
 namespace {

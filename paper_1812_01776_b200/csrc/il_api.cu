@@ -47,7 +47,7 @@ struct il_estimator {
     int ctas_per_sm_wide = 0, ctas_per_sm_packed = 0, ctas_per_sm_staged = 0, ctas_per_sm_lane = 0;
     int64_t lane_elems = 0;            // lane kernel: stream records per candidate (all rings of a candidate)
     int lane_ring_log2 = 0;            // lane kernel: a stream ring holds 2^this records
-    int lane_ring_cap_log2 = 13;       // ... at most 2^this (8,192 records = 64 KB per stage and resident candidate)
+    int lane_ring_cap_log2 = 0;        // test knob: force rings of at most 2^this records (0: the library's choice)
     bool lane_wrap = false;            // the rings are shorter than the longest stream
     unsigned long long iter_limit = 0; // test knob: iteration bound of the device loops (0 = their own)
     int cpw = 1;                       // lane kernel: candidates per warp
@@ -269,20 +269,41 @@ int64_t plan_stream_buffers(const il_profiles *pr, const int64_t *visits, int32_
     return top;
 }
 
-// Ring length of the lane kernel's streams: long enough for the longest stream if the cap allows
-// (then nothing wraps), else the cap.  Sets the layout of a candidate's rings.
+// Layout of a candidate's inter-stage streams in the lane kernel.  While the streams of all resident
+// candidates fit kLaneExactBytes, every stage keeps its whole arrival stream (nothing wraps, and the
+// kernel instantiation without the ring protocol runs, which is the faster one per iteration).  Beyond
+// that -- long traces through deep pipelines -- a stage's stream lives in a ring of 2^13 records and the
+// scratch per resident candidate no longer grows with the trace.  lane_ring_cap_log2 > 0 (test knob)
+// forces rings of at most that length.
+constexpr int64_t kLaneExactBytes = INT64_C(48) << 30;
+constexpr int kLaneRingLog2 = 13;
+
 void configure_lane_rings(il_estimator *e)
 {
-    int64_t longest = 8;
-    for (int s = 1; s < e->S; s++) longest = std::max(longest, e->visits[s]);
-    int need = 3;
-    while ((INT64_C(1) << need) < longest) need++;
-    e->lane_ring_log2 = std::min(need, e->lane_ring_cap_log2);
-    e->lane_wrap = (INT64_C(1) << e->lane_ring_log2) < longest;
     DesParams &bp = e->base;
+    int64_t longest = 8, exact = 0;
+    for (int s = 1; s < e->S; s++) {
+        longest = std::max(longest, e->visits[s]);
+        exact += (e->visits[s] + 3) / 4 * 4;
+    }
+    const int64_t resident = (int64_t)e->num_sms * kLaneCtasPerSm * des_lane_warps_per_cta() * e->cpw;
+    const bool rings = e->lane_ring_cap_log2 > 0 || exact * 8 * resident > kLaneExactBytes ||
+                       exact >= (INT64_C(1) << 31);
     bp.lane_off[0] = 0;
-    for (int s = 1; s < e->S; s++) bp.lane_off[s] = (int32_t)((int64_t)(s - 1) << e->lane_ring_log2);
-    e->lane_elems = std::max<int64_t>((int64_t)(e->S - 1) << e->lane_ring_log2, 4);
+    if (!rings) {
+        int64_t off = 0;
+        for (int s = 1; s < e->S; s++) { bp.lane_off[s] = (int32_t)off; off += (e->visits[s] + 3) / 4 * 4; }
+        e->lane_elems = std::max<int64_t>(exact, 4);
+        e->lane_ring_log2 = 31;
+        e->lane_wrap = false;
+    } else {
+        int need = 3;
+        while ((INT64_C(1) << need) < longest) need++;
+        e->lane_ring_log2 = std::min(need, e->lane_ring_cap_log2 > 0 ? e->lane_ring_cap_log2 : kLaneRingLog2);
+        e->lane_wrap = (INT64_C(1) << e->lane_ring_log2) < longest;
+        for (int s = 1; s < e->S; s++) bp.lane_off[s] = (int32_t)((int64_t)(s - 1) << e->lane_ring_log2);
+        e->lane_elems = std::max<int64_t>((int64_t)(e->S - 1) << e->lane_ring_log2, 4);
+    }
     bp.lane_elems = e->lane_elems;
     bp.lane_ring_log2 = e->lane_ring_log2;
     bp.lane_wrap = e->lane_wrap ? 1 : 0;

@@ -113,6 +113,60 @@ cudaError_t launch_select(const SelectParams &p, cudaStream_t stream);
 cudaError_t launch_scatter_latency(const int64_t *slab_row, const int64_t *arrival, int n, int qbits,
                                    int64_t *out, cudaStream_t stream);
 
+// ---- shared-prefix evaluation (prefix_kernel.cu) ----------------------------------------------
+// One stage of the node simulation: node k of the stage reads the stream of node node_parent[k] of
+// the parent stage (or the trace) and writes its own streams at k * stride.
+struct NodeStageParams {
+    const int32_t *lat_stage;     // [H][Bmax] profile of this stage
+    const uint8_t *bits;          // [n] branch bits
+    const uint64_t *ptrace;       // packed trace (root stage)
+    int32_t qbits, H, Bmax;
+    int32_t n_in;                 // queries visiting the stage
+    int32_t bit;                  // branch bit tested after the stage, -1 = none
+    int64_t n_nodes;
+    const uint32_t *node_cfg;     // [n_nodes] hw | max batch << 8 | replicas << 16
+    const int32_t *node_parent;   // [n_nodes] node of the parent stage
+    const uint64_t *in;           // parent stage's streams for this stage, nullptr at the root
+    int64_t stride_in;
+    uint64_t *out_a, *out_b;      // this stage's streams per side: to a child stage, or the leaving records
+    int64_t stride_a, stride_b;
+    unsigned long long *work;     // work counter (zero at launch)
+    unsigned long long *counters; // the handle's counter block
+    int *status;
+};
+cudaError_t launch_node_stage(const NodeStageParams &p, int grid, cudaStream_t stream);
+cudaError_t launch_prefix_stage(const il_stage_config *configs, int64_t n_cand, int S, int s, int H, int Bmax,
+                                const int32_t *parent_node, uint64_t *keys, uint32_t cap, int32_t *vals,
+                                int32_t *slot_of, int *count, uint32_t *node_cfg, int32_t *node_parent,
+                                int32_t *node_of, int *status, cudaStream_t stream);
+// Largest latencies of every node of a stage that queries leave after (select_kernel.cu).
+struct NodeTopParams {
+    uint64_t *records;            // [n_nodes][stride] leaving records (finish << qbits | query); overwritten
+    int64_t stride;
+    int32_t len;                  // records per node
+    const int64_t *arrival;
+    int32_t qbits;
+    int64_t slo_us;
+    int32_t top_len;              // T + 1 entries kept per node, T = queries allowed above the P99
+    int64_t *top;                 // [n_nodes][top_len] descending, zero-filled beyond the node's count
+    int64_t *miss;                // [n_nodes]
+    int64_t n_nodes;
+};
+cudaError_t launch_node_top(const NodeTopParams &p, cudaStream_t stream);
+size_t node_top_smem(int top_len);
+struct CombineParams {
+    int64_t n_cand;
+    const int32_t *node_of;       // [S][n_cand]
+    int32_t n_exit;               // stages that queries leave after
+    int32_t exit_stage[IL_MAX_STAGES];
+    const int64_t *top[IL_MAX_STAGES];
+    const int64_t *miss[IL_MAX_STAGES];
+    int32_t top_len;
+    int64_t allowed;              // T = n - k
+    int64_t *out_p99, *out_miss;
+};
+cudaError_t launch_prefix_combine(const CombineParams &p, cudaStream_t stream);
+
 // Fills order[0..n_cand) with the chunk's candidate indices, costliest first
 // (longest-processing-time-first scheduling over the warps).
 struct OrderParams {

@@ -180,6 +180,121 @@ select_kernel(const __grid_constant__ SelectParams p)
     }
 }
 
+// Shared-prefix evaluation: the largest latencies of one node of a stage that queries leave after.
+// A candidate's P99 is the (T + 1)-th largest latency of the union of its leaving nodes, T = n - k
+// being the number of queries allowed above it, so no node ever contributes more than its own T + 1
+// largest: they are kept, in descending order, for the combine step (prefix_kernel.cu), together with
+// the node's miss count.  One CTA per node: records -> latencies (in place), radix select of the
+// (T + 1)-th largest, collection of everything above it into shared memory, bitonic sort.
+__global__ void __launch_bounds__(kSelectThreads)
+node_top_kernel(const __grid_constant__ NodeTopParams p)
+{
+    extern __shared__ __align__(16) unsigned char top_raw[];
+    int64_t *s_top = reinterpret_cast<int64_t *>(top_raw);
+    __shared__ unsigned hist[256];
+    __shared__ unsigned long long s_prefix, s_or;
+    __shared__ unsigned s_rank, s_miss, s_fill;
+
+    int pow2 = 1;
+    while (pow2 < p.top_len) pow2 <<= 1;
+    const uint64_t qmask = (1ull << p.qbits) - 1ull;
+    for (int64_t node = blockIdx.x; node < p.n_nodes; node += gridDim.x) {
+        int64_t *lat = reinterpret_cast<int64_t *>(p.records + node * p.stride);
+        if (threadIdx.x == 0) { s_or = 0; s_miss = 0; s_fill = 0; s_prefix = 0; }
+        __syncthreads();
+        unsigned miss = 0;
+        unsigned long long my_or = 0;
+        for (int i = threadIdx.x; i < p.len; i += kSelectThreads) {
+            const uint64_t rec = (uint64_t)lat[i];
+            const int64_t l = (int64_t)(rec >> p.qbits) - p.arrival[rec & qmask];
+            lat[i] = l;
+            my_or |= (unsigned long long)l;
+            miss += (l > p.slo_us);
+        }
+        for (int o = 16; o > 0; o >>= 1) my_or |= __shfl_xor_sync(0xffffffffu, my_or, o);
+        if ((threadIdx.x & 31) == 0 && my_or) atomicOr(&s_or, my_or);
+        if (miss) atomicAdd(&s_miss, miss);
+        __syncthreads();
+        long long threshold = -1;       // keep every latency above this value
+        if (p.len > p.top_len) {
+            // the top_len-th largest = the (len - top_len + 1)-th smallest
+            int top = 0;
+            while (top < 8 && (s_or >> (8 * top)) != 0) top++;
+            if (threadIdx.x == 0) s_rank = (unsigned)(p.len - p.top_len + 1);
+            __syncthreads();
+            for (int d = top - 1; d >= 0; d--) {
+                hist[threadIdx.x] = 0;
+                __syncthreads();
+                const unsigned long long prefix = s_prefix;
+                const int shift = 8 * d;
+                const unsigned long long himask = (d == 7) ? 0ull : (~0ull << (shift + 8));
+                for (int i = threadIdx.x; i < p.len; i += kSelectThreads) {
+                    const unsigned long long v = (unsigned long long)lat[i];
+                    if ((v & himask) == prefix) atomicAdd(&hist[(v >> shift) & 0xff], 1u);
+                }
+                __syncthreads();
+                if (threadIdx.x == 0) {
+                    unsigned r = s_rank, acc = 0;
+                    int b = 0;
+                    for (; b < 255; b++) {
+                        if (acc + hist[b] >= r) break;
+                        acc += hist[b];
+                    }
+                    s_rank = r - acc;
+                    s_prefix = prefix | ((unsigned long long)b << shift);
+                }
+                __syncthreads();
+            }
+            threshold = (long long)s_prefix;
+        }
+        // everything above the threshold, then copies of the threshold up to top_len entries, then zeros
+        for (int i = threadIdx.x; i < p.len; i += kSelectThreads) {
+            const int64_t l = lat[i];
+            if (l > threshold) s_top[atomicAdd(&s_fill, 1u)] = l;
+        }
+        __syncthreads();
+        const int got = (int)s_fill;
+        const int keep = p.len > p.top_len ? p.top_len : got;
+        for (int i = got + (int)threadIdx.x; i < pow2; i += kSelectThreads) s_top[i] = i < keep ? threshold : 0;
+        __syncthreads();
+        // bitonic sort, descending
+        for (int k = 2; k <= pow2; k <<= 1) {
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                for (int i = threadIdx.x; i < pow2; i += kSelectThreads) {
+                    const int partner = i ^ j;
+                    if (partner > i) {
+                        const int64_t a = s_top[i], b = s_top[partner];
+                        const bool desc = (i & k) == 0;
+                        if (desc ? a < b : a > b) { s_top[i] = b; s_top[partner] = a; }
+                    }
+                }
+                __syncthreads();
+            }
+        }
+        int64_t *out = p.top + node * p.top_len;
+        for (int i = threadIdx.x; i < p.top_len; i += kSelectThreads) out[i] = s_top[i];
+        if (threadIdx.x == 0) p.miss[node] = (int64_t)s_miss;
+        __syncthreads();
+    }
+}
+
+size_t node_top_smem(int top_len)
+{
+    size_t pow2 = 1;
+    while (pow2 < (size_t)top_len) pow2 <<= 1;
+    return pow2 * sizeof(int64_t);
+}
+
+cudaError_t launch_node_top(const NodeTopParams &p, cudaStream_t stream)
+{
+    const size_t smem = node_top_smem(p.top_len);
+    cudaError_t e = cudaFuncSetAttribute(node_top_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const int grid = (int)(p.n_nodes < 148 * 8 ? p.n_nodes : 148 * 8);
+    node_top_kernel<<<grid, kSelectThreads, smem, stream>>>(p);
+    return cudaGetLastError();
+}
+
 // Per-query answer of one candidate: the slab row holds one (finish, query)
 // record per query, in the order the queries left the pipeline; the latency of
 // query q goes to out[q].

@@ -64,13 +64,16 @@ class PlanResult:
 
 class Planner:
     def __init__(self, parent, latency_us, visits, prices: Sequence[float], slo_us: int,
-                 estimate: EstimateFn):
+                 estimate: EstimateFn, feasible: Optional[Callable[[np.ndarray], np.ndarray]] = None):
         """
         parent       [S] parent stage of every stage (-1 for the root)
         latency_us   [S][H][Bmax] model profiles
         visits       [S] queries visiting each stage (il_stage_visits); visits / visits[0] is the scale factor
         prices       [H] cost per replica-hour of each hardware type
         estimate     configs [n][S][4] uint8 -> (p99_us[n], miss[n]) for the bound trace and this objective
+        feasible     optional: configs -> bool[n], the same answer as p99_us <= slo_us but cheaper to get
+                     (Estimator.feasible drops a candidate as soon as it is decided); the search then asks
+                     only this, and `estimate` is called once, for the P99 of the final plan
         """
         self.parent = np.asarray(parent, dtype=np.int64)
         self.lat = np.asarray(latency_us, dtype=np.int64)
@@ -80,6 +83,7 @@ class Planner:
         assert self.prices.shape == (self.H,)
         self.slo_us = int(slo_us)
         self._estimate = estimate
+        self._feasible = feasible
         self.calls = 0
         self.evaluated = 0
         self.batches = [b for b in (1 << np.arange(7)) if b <= self.Bmax]
@@ -90,9 +94,11 @@ class Planner:
         configs = np.ascontiguousarray(configs, dtype=np.uint8)
         if configs.shape[0] == 0:
             return np.zeros(0, bool), np.zeros(0, np.int64)
-        p99, _ = self._estimate(configs)
         self.calls += 1
         self.evaluated += configs.shape[0]
+        if self._feasible is not None:
+            return np.asarray(self._feasible(configs), dtype=bool), np.full(configs.shape[0], -1, np.int64)
+        p99, _ = self._estimate(configs)
         p99 = np.asarray(p99, dtype=np.int64)
         return p99 <= self.slo_us, p99
 
@@ -217,8 +223,10 @@ class Planner:
             cfg = cands[best]
             trajectory.append(cfg.copy())
             steps.append(f"{labels[best]} -> cost {self.cost(cfg):.4f}")
-        ok, p99 = self.feasible_many(cfg[None])
-        assert ok[0]
+        p99, _ = self._estimate(np.ascontiguousarray(cfg[None], dtype=np.uint8))
+        self.calls += 1
+        self.evaluated += 1
+        assert int(p99[0]) <= self.slo_us
         return PlanResult(True, cfg, self.cost(cfg), int(p99[0]), self.calls, self.evaluated, steps, trajectory)
 
     def single_actions(self, cfg: np.ndarray) -> List[np.ndarray]:

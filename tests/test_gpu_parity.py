@@ -154,11 +154,11 @@ def test_configs_reduced_short_stream_rings(il, oracle, cid, n, C):
     assert 0 <= st["fallback_candidates"] <= C
 
 
-def test_default_rings_rarely_overflow(il, oracle):
-    """With the default ring length (8,192 records) and the workloads' tables, a trace far longer
-    than a ring runs on the lane kernel alone."""
+def test_production_ring_length_rarely_overflows(il, oracle):
+    """With the ring length the library uses for long traces (8,192 records) and the workloads'
+    tables, a trace five times longer than a ring runs on the lane kernel alone."""
     w = workloads.make(2, n_queries=40000, n_candidates=192)
-    st = check(il, oracle, w, host=False)
+    st = check(il, oracle, w, host=False, knobs={1: 13})
     assert st["fallback_candidates"] <= 2
 
 
@@ -414,3 +414,27 @@ def test_largest_table_shape(il, oracle, variant):
     w = workloads.random_small(500, S=16, H=8, Bmax=64, n=1200, C=19, max_replicas=32, tree=True,
                                qps=300.0, cv=2.0, lat_lo=50, lat_hi=9000)
     check(il, oracle, w, host=False, variant=variant)
+
+
+@pytest.mark.parametrize("variant", [3, 4, 1, 2], ids=["lanes", "packed", "wide", "staged"])
+def test_iteration_bound_is_reported_and_the_handle_survives(il, oracle, variant):
+    """Every simulation kernel bounds its loops and reports IL_ERR_ITER_LIMIT instead of spinning.
+    The bound cannot be reached on valid input, so the test shortens it through the test knob: the
+    call must come back with that code, and the same handle must give oracle-exact results again
+    once the bound is restored."""
+    from paper_1812_01776_b200 import estimator as E
+    w = workloads.make(3, n_queries=3000, n_candidates=40)
+    exp = oracle.estimate_workload(w)
+    with il.Estimator.from_workload(w) as est:
+        est.set_variant(variant)
+        est.set_test_knob(E.IL_KNOB_ITER_LIMIT, 50)
+        with pytest.raises(E.ILError) as ei:
+            est.estimate(w.configs, w.slo_us)
+        assert ei.value.code == E.IL_ERR_ITER_LIMIT
+        with pytest.raises(E.ILError) as ei:
+            est.feasible(w.configs, w.slo_us)
+        assert ei.value.code == E.IL_ERR_ITER_LIMIT
+        est.set_test_knob(E.IL_KNOB_ITER_LIMIT, 0)
+        p99, miss = est.estimate(w.configs, w.slo_us)
+        assert np.array_equal(p99, exp[0]) and np.array_equal(miss, exp[1])
+        assert np.array_equal(est.feasible(w.configs, w.slo_us), exp[0] <= w.slo_us)

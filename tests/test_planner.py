@@ -189,9 +189,13 @@ def test_planner_same_plan_on_gpu_and_oracle(oracle):
         assert np.array_equal(est.visits, visits)
         got = Planner(w.parent, w.latency_us, est.visits, prices, slo,
                       lambda cfgs: est.estimate(cfgs, slo)).minimize_cost()
-    assert got.feasible == ref.feasible
-    assert np.array_equal(got.config, ref.config)
-    assert got.cost == ref.cost and got.p99_us == ref.p99_us and got.steps == ref.steps
+        # and with the feasibility-only entry point answering the search's questions
+        fea = Planner(w.parent, w.latency_us, est.visits, prices, slo,
+                      lambda cfgs: est.estimate(cfgs, slo), feasible=lambda cfgs: est.feasible(cfgs, slo)).minimize_cost()
+    for res in (got, fea):
+        assert res.feasible == ref.feasible
+        assert np.array_equal(res.config, ref.config)
+        assert res.cost == ref.cost and res.p99_us == ref.p99_us and res.steps == ref.steps
 
 
 @pytest.mark.gpu
