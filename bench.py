@@ -384,6 +384,46 @@ def measure(il, torch, w, dev, stream, flush, steps, warmup, e2e_steps, variant,
     return rec
 
 
+def measure_feasibility(il, torch, dev, stream, flush):
+    """Feasibility-only mode against the full estimate: workload 2's 4,096 candidates (device-resident,
+    best of 3 each), and a Planner run on workload 2's trace whose questions are answered either way."""
+    from paper_1812_01776_b200.planner import Planner
+    w = workloads.make(2)
+    out = {"workload": WORKLOADS[2]}
+    with il.Estimator.from_workload(w, device=dev.index) as est, torch.cuda.stream(stream):
+        est.reserve_workspace(w.n_candidates)
+        est.use_current_stream()
+        d_cfg = torch.from_numpy(w.configs).to(dev)
+        d_flag = torch.empty(w.n_candidates, dtype=torch.uint8, device=dev)
+
+        def timed(fn):
+            best = None
+            for _ in range(3):
+                flush.fill_(1)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream); fn(); b.record(stream); b.synchronize()
+                best = a.elapsed_time(b) if best is None else min(best, a.elapsed_time(b))
+            return best
+        full_ms = timed(lambda: est.estimate_device(d_cfg, w.slo_us))
+        feas_ms = timed(lambda: est.feasible_device(d_cfg, w.slo_us, d_flag))
+        st = est.stats()
+        out.update(estimate_ms=full_ms, feasible_ms=feas_ms, speedup=full_ms / feas_ms,
+                   infeasible_fraction=1.0 - float(d_flag.float().mean().item()),
+                   dropped_early=st["early_exits"], candidates=w.n_candidates)
+        prices = np.array([0.90, 0.35, 0.10])
+        plans = {}
+        for name, feas in (("estimate", None), ("feasible", lambda c: est.feasible(c, w.slo_us))):
+            pl = Planner(w.parent, w.latency_us, est.visits, prices, w.slo_us,
+                         lambda c: est.estimate(c, w.slo_us), feasible=feas)
+            t0 = time.perf_counter()
+            res = pl.minimize_cost()
+            plans[name] = {"seconds": time.perf_counter() - t0, "estimator_calls": res.estimator_calls,
+                           "candidates_evaluated": res.candidates_evaluated, "cost": res.cost}
+        out["planner"] = plans
+        out["planner"]["same_plan"] = plans["estimate"]["cost"] == plans["feasible"]["cost"]
+    return out
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -433,6 +473,9 @@ def run_cuda(args):
             for k in ("step_ms_sum", "e2e_ms_sum"):
                 r.pop(k)
             per_workload.append(r)
+    feas = None
+    if world == 1 and not args.no_per_workload:
+        feas = measure_feasibility(il, torch, dev, stream, flush)
     if world > 1:
         dist.destroy_process_group()
     if rank != 0:
@@ -469,6 +512,7 @@ def run_cuda(args):
         "gpu_launches": main["gpu_launches"],
         "clocks": main.get("clocks", {}),
         "per_workload": per_workload,
+        "feasible_only": feas,
     }
     if world == 1 and not args.no_cpu_baseline:
         cores = os.cpu_count() or 1

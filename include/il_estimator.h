@@ -72,6 +72,8 @@ extern "C" {
 #define IL_ERR_CUDA          -7  /* a CUDA runtime call failed; see il_last_cuda_error     */
 #define IL_ERR_ITER_LIMIT    -8  /* a device loop hit its iteration bound (internal error) */
 #define IL_ERR_TOO_LARGE     -9  /* il_estimate_device_static: needs more than IL_STATIC_SCRATCH_BYTES */
+#define IL_ERR_BOUNDS       -10  /* checked build only (-DIL_CHECKED): a device index left its array; the access
+                                    was skipped and recorded instead (internal error)                        */
 
 typedef struct il_estimator il_estimator;   /* opaque; owns its device copies */
 
@@ -180,6 +182,18 @@ IL_API int il_estimate(il_estimator *est, const il_stage_config *configs, int64_
  * Work is enqueued on the handle's stream and the call waits for it.
  * Candidates are validated on the device; an invalid one makes the call return
  * BAD_CONFIG after the stream has drained, and outputs are then undefined.
+ *
+ * Shared prefixes.  The completion stream of a stage depends only on the
+ * configurations of the stages on its path from the root, so candidates that
+ * agree there need that part simulated once.  With the default kernel choice
+ * (IL_VARIANT_AUTO), a batch of at least 2,048 candidates, n - ceil(0.99 n) <
+ * 16,384 and enough workspace, the call first builds the set of distinct (stage,
+ * configuration, parent) nodes on the device; if there are at most a quarter as
+ * many nodes as candidates x stages (an exhaustive sweep over per-stage choices,
+ * not a uniform random draw) it simulates every node once and assembles each
+ * candidate's P99 and miss count from the nodes where its queries leave.  Results
+ * are the same integers; il_stats.stage_runs tells how many stage simulations
+ * were carried out.
  */
 IL_API int il_estimate_device(il_estimator *est, const il_stage_config *d_configs, int64_t n,
                               int64_t slo_us, int64_t *d_out_p99_us, int64_t *d_out_miss);
@@ -351,10 +365,14 @@ IL_API int il_set_variant(il_estimator *est, int variant);
  *   IL_KNOB_ITER_LIMIT      value >= 0: iteration bound of the simulation kernels' loops; 0 restores
  *                           the bound each loop derives from its input.  A small bound makes a call
  *                           return IL_ERR_ITER_LIMIT; the handle stays usable.
+ *   IL_KNOB_SHARE_PREFIXES  0: the library decides per call whether to evaluate a batch through shared
+ *                           configuration prefixes (see il_estimate_device); 1: always, when the
+ *                           preconditions hold; 2: never.
  * Set a knob before il_workspace_bytes / il_set_workspace: sizes depend on the ring length.
  */
 #define IL_KNOB_LANE_RING_LOG2 1
 #define IL_KNOB_ITER_LIMIT 2
+#define IL_KNOB_SHARE_PREFIXES 3
 IL_API int il_set_test_knob(il_estimator *est, int knob, int64_t value);
 
 /* Name of the simulation kernel the handle's next estimate call will launch

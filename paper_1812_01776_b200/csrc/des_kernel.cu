@@ -121,21 +121,23 @@ des_kernel(const __grid_constant__ DesParams p)
                     int32_t q = 0;
                     if (act) q = (s == 0) ? start + j : in_q[start + j];
                     bool bitv = false;
-                    if (act && rt.bit >= 0) bitv = (p.bits[q] >> rt.bit) & 1;
+                    if (act && rt.bit >= 0 && IL_IN_RANGE(q, p.n, p.status)) bitv = (p.bits[q] >> rt.bit) & 1;
                     const unsigned ma = __ballot_sync(full, act && !bitv);
                     const unsigned mb_ = __ballot_sync(full, act && bitv);
                     if (ma) {
                         const bool mine = act && !bitv;
                         const int rank = __popc(ma & lt_mask);
                         if (rt.a_exit) {
-                            if (mine) {
+                            if (mine && IL_IN_RANGE(q, p.n, p.status)) {
                                 const int64_t l = tfin - p.arrival[q];
                                 slab[q] = l;   // trace order: the slab doubles as the per-query answer
                                 lat_or |= (uint64_t)l;
                             }
                             exits += __popc(ma);
                         } else {
-                            if (mine) { rt.a_time[rt.a_tail + rank] = tfin; rt.a_qid[rt.a_tail + rank] = q; }
+                            if (mine && IL_IN_RANGE(p.buf_off[da] + rt.a_tail + rank, p.slot_elems, p.status)) {
+                                rt.a_time[rt.a_tail + rank] = tfin; rt.a_qid[rt.a_tail + rank] = q;
+                            }
                             rt.a_tail += __popc(ma);
                         }
                     }
@@ -143,14 +145,16 @@ des_kernel(const __grid_constant__ DesParams p)
                         const bool mine = act && bitv;
                         const int rank = __popc(mb_ & lt_mask);
                         if (rt.b_exit) {
-                            if (mine) {
+                            if (mine && IL_IN_RANGE(q, p.n, p.status)) {
                                 const int64_t l = tfin - p.arrival[q];
                                 slab[q] = l;   // trace order: the slab doubles as the per-query answer
                                 lat_or |= (uint64_t)l;
                             }
                             exits += __popc(mb_);
                         } else {
-                            if (mine) { rt.b_time[rt.b_tail + rank] = tfin; rt.b_qid[rt.b_tail + rank] = q; }
+                            if (mine && IL_IN_RANGE(p.buf_off[db] + rt.b_tail + rank, p.slot_elems, p.status)) {
+                                rt.b_time[rt.b_tail + rank] = tfin; rt.b_qid[rt.b_tail + rank] = q;
+                            }
                             rt.b_tail += __popc(mb_);
                         }
                     }

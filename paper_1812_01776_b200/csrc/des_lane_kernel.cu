@@ -192,6 +192,14 @@ des_lane_kernel(const __grid_constant__ DesParams p)
     const uint32_t mask_b = (RING && db >= 0) ? K - 1u : 0xffffffffu;
     const unsigned long long iter_limit = p.iter_limit;
     const unsigned long long n_cand = (unsigned long long)p.n_cand;
+    // sizes of what this lane reads and writes, for the checked build: its arrival stream (or the trace),
+    // and per side the child's stream or the rest of the slab row
+    const unsigned long long in_size = s == 0 ? (unsigned long long)p.n : (unsigned long long)(p.lane_elems - p.lane_off[s]);
+    const unsigned long long size_a = da < 0 ? (unsigned long long)(p.slab_stride - exit_off)
+                                             : (unsigned long long)(p.lane_elems - p.lane_off[da]);
+    const unsigned long long size_b = db < 0 ? (unsigned long long)(p.slab_stride - exit_off)
+                                             : (unsigned long long)(p.lane_elems - p.lane_off[db]);
+    (void)in_size; (void)size_a; (void)size_b;
     const uint64_t slo_q = FEAS ? (uint64_t)p.slo_us << q : 0ull;   // the objective, aligned with a record's time field
     unsigned long long batches = 0, alg_ops = 0, exits_seen = 0, exits_due = 0;
     unsigned early = 0;          // candidates dropped before the end of the trace (feasibility only)
@@ -313,8 +321,8 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                 if (turn) {
                     has = got;
                     exhausted = !got;
-                    c = (int64_t)g;
-                    cand_bad = grp_bad;
+                    c = (int64_t)g;      // g < n_cand whenever the group got a candidate: rows of the slab, the
+                    cand_bad = grp_bad;  // overflow array and the output exist for it
                     uint64_t *slab = FEAS ? nullptr : reinterpret_cast<uint64_t *>(p.slab + (got ? c : 0) * p.slab_stride);
                     if (got && cand_bad) {
                         if (s == 0) atomicCAS(p.status, 0, IL_ERR_BAD_CONFIG);
@@ -365,10 +373,11 @@ des_lane_kernel(const __grid_constant__ DesParams p)
             const uint32_t h_qid = (uint32_t)wm.stage_e[h_sl][lane] & (uint32_t)qmask;   // unused unless h_valid
             const uint64_t h_base = wm.stage_b[h_sl][lane];
             uint32_t h_bits = 0;
-            if (BRANCHY && h_valid && bit >= 0) h_bits = p.bits[h_qid];
+            if (BRANCHY && h_valid && bit >= 0 && IL_IN_RANGE(h_qid, p.n, p.status)) h_bits = p.bits[h_qid];
             // feasibility only: the arrival record of a query that may leave here, to test its latency
             uint64_t h_arr = 0;
-            if (FEAS && h_valid && (da < 0 || (db < 0 && bit >= 0))) h_arr = p.ptrace[h_qid];
+            if (FEAS && h_valid && (da < 0 || (db < 0 && bit >= 0)) && IL_IN_RANGE(h_qid, p.n, p.status))
+                h_arr = p.ptrace[h_qid];
             // likewise the next batch to hand on, if the one in hand is used up (a batch handed over in
             // this iteration is picked up in the next), and the table entry a close would need
             const bool f_valid = e_left == 0 && epos != lpos;
@@ -444,18 +453,20 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                         if (h_base > (h_arr & ~qmask) + slo_q) atomicAdd(&wm.miss[j], 1u);
                     } else if (h_valid) {
                         uint64_t *dst = to_b ? out_b + (tail_b & mask_b) : out_a + (tail_a & mask_a);
-                        *dst = out;
+                        if (IL_IN_RANGE(to_b ? (tail_b & mask_b) : (tail_a & mask_a), to_b ? size_b : size_a, p.status))
+                            *dst = out;
                     }
                 } else {
                     uint64_t *dst = to_b ? out_b + (tail_b & mask_b) : out_a + (tail_a & mask_a);
-                    if (h_valid) *dst = out;
+                    if (h_valid && IL_IN_RANGE(to_b ? (tail_b & mask_b) : (tail_a & mask_a), to_b ? size_b : size_a, p.status))
+                        *dst = out;
                 }
                 tail_b += (h_valid && to_b) ? 1u : 0u;
                 tail_a += (h_valid && !to_b) ? 1u : 0u;
             } else if (h_valid) {
                 if (FEAS && da < 0) {
                     if (h_base > (h_arr & ~qmask) + slo_q) atomicAdd(&wm.miss[j], 1u);
-                } else {
+                } else if (IL_IN_RANGE(tail_a & mask_a, size_a, p.status)) {
                     out_a[tail_a & mask_a] = h_base | h_qid;
                 }
                 tail_a++;
@@ -471,7 +482,8 @@ des_lane_kernel(const __grid_constant__ DesParams p)
             vmask = (vmask << 1) & 7u;
             if (e_left > 0 && can_emit) {
                 const uint32_t sl = it & (kStage - 1);
-                cp_async8(&wm.stage_e[sl][lane], in + (e_idx & in_mask));
+                if (IL_IN_RANGE(e_idx & in_mask, in_size, p.status))
+                    cp_async8(&wm.stage_e[sl][lane], in + (e_idx & in_mask));
                 wm.stage_b[sl][lane] = e_base;
                 e_idx++; e_left--;
                 vmask |= 1u;
@@ -480,7 +492,8 @@ des_lane_kernel(const __grid_constant__ DesParams p)
             // next, and (while the parent runs) kLag behind what it has written
             const uint32_t i2 = head + (uint32_t)b;
             if (fx < i2 + (uint32_t)kStage && (pdone ? fx < written : fx + (uint32_t)kLag < written)) {
-                cp_async8(&wm.stage_x[fx & (kStage - 1)][lane], in + (fx & in_mask));
+                if (IL_IN_RANGE(fx & in_mask, in_size, p.status))
+                    cp_async8(&wm.stage_x[fx & (kStage - 1)][lane], in + (fx & in_mask));
                 fx++;
             }
             done = end && b == 0 && epos == tpos && e_left == 0 && vmask == 0u;

@@ -51,6 +51,7 @@ struct WarpCtx {
     uint32_t qmask;
     int qbits;
     const uint8_t *bits;
+    int n_queries;           // length of bits
     uint64_t *slot_key;      // shared memory, 32 slot keys: staging for re-ordering the slots
     uint32_t *slot_q;        // shared memory, 32 slot query ids
     int *slot_b;             // shared memory, 32 slot batch sizes
@@ -213,6 +214,8 @@ struct Sink {
     uint64_t *out_a, *out_b;
     int tail_a, tail_b;
     int bit;
+    int size_a, size_b;      // records each side can take (compared with in the checked build)
+    int *status;
 };
 
 // Appends the records held by lanes [0, n_act) in lane order.
@@ -221,16 +224,20 @@ __device__ __forceinline__ void append(const WarpCtx &w, Sink &sk, const uint64_
 {
     const bool act = w.lane < n_act;
     if (KIND == kForward) {
-        if (act) sk.out_a[sk.tail_a + w.lane] = rec;
+        if (act && IL_IN_RANGE(sk.tail_a + w.lane, sk.size_a, sk.status)) sk.out_a[sk.tail_a + w.lane] = rec;
         sk.tail_a += n_act;
     } else {
         bool bitv = false;
-        if (act) bitv = (w.bits[(uint32_t)rec & w.qmask] >> sk.bit) & 1;
+        if (act && IL_IN_RANGE((uint32_t)rec & w.qmask, w.n_queries, sk.status))
+            bitv = (w.bits[(uint32_t)rec & w.qmask] >> sk.bit) & 1;
         const unsigned ma = __ballot_sync(0xffffffffu, act && !bitv);
         const unsigned mb = __ballot_sync(0xffffffffu, act && bitv);
         if (act) {
-            if (bitv) sk.out_b[sk.tail_b + __popc(mb & w.lt_mask)] = rec;
-            else sk.out_a[sk.tail_a + __popc(ma & w.lt_mask)] = rec;
+            const int at = bitv ? sk.tail_b + __popc(mb & w.lt_mask) : sk.tail_a + __popc(ma & w.lt_mask);
+            if (IL_IN_RANGE(at, bitv ? sk.size_b : sk.size_a, sk.status)) {
+                if (bitv) sk.out_b[at] = rec;
+                else sk.out_a[at] = rec;
+            }
         }
         sk.tail_a += __popc(ma);
         sk.tail_b += __popc(mb);
@@ -873,6 +880,9 @@ __device__ __forceinline__ void simulate_candidate(const DesParams &p, const War
         sk.out_a = da < 0 ? slab + exits : my_rec + p.buf_off[da];
         sk.out_b = db < 0 ? slab + exits : my_rec + p.buf_off[db];
         sk.tail_a = 0; sk.tail_b = 0;
+        sk.size_a = da < 0 ? (int)p.slab_stride - exits : (int)(p.slot_elems - p.buf_off[da]);
+        sk.size_b = db < 0 ? (int)p.slab_stride - exits : (int)(p.slot_elems - p.buf_off[db]);
+        sk.status = p.status;
         int nb;
         if (STAGED && s == 0) {
             TileSrc src = {ring, p.ptrace, n_tiles, 0, -1, false, p.status};
@@ -928,6 +938,7 @@ des_packed_kernel(const __grid_constant__ DesParams p)
     w.qbits = p.qbits;
     w.qmask = (1u << p.qbits) - 1u;
     w.bits = p.bits;
+    w.n_queries = p.n;
     w.slot_key = s_slot_key[wid];
     w.slot_q = s_slot_q[wid];
     w.slot_b = s_slot_b[wid];
@@ -999,6 +1010,7 @@ des_node_stage_kernel(const __grid_constant__ NodeStageParams p)
     w.qbits = p.qbits;
     w.qmask = (1u << p.qbits) - 1u;
     w.bits = p.bits;
+    w.n_queries = p.n_queries;
     w.slot_key = s_slot_key[wid];
     w.slot_q = s_slot_q[wid];
     w.slot_b = s_slot_b[wid];
@@ -1015,6 +1027,8 @@ des_node_stage_kernel(const __grid_constant__ NodeStageParams p)
         sk.out_a = p.out_a + (int64_t)k * p.stride_a;
         sk.out_b = p.out_b + (int64_t)k * p.stride_b;
         sk.tail_a = 0; sk.tail_b = 0;
+        sk.size_a = (int)p.stride_a; sk.size_b = (int)p.stride_b;
+        sk.status = p.status;
         GlobalSrc src = {p.in ? p.in + (int64_t)p.node_parent[k] * p.stride_in : p.ptrace, p.in == nullptr};
         const int nb = dispatch_stage(w, s_row + hw * p.Bmax, mb, R, p.n_in, src, sk, p.status);
         batches += (unsigned)nb;

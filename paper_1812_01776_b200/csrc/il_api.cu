@@ -50,6 +50,8 @@ struct il_estimator {
     int lane_ring_cap_log2 = 0;        // test knob: force rings of at most 2^this records (0: the library's choice)
     bool lane_wrap = false;            // the rings are shorter than the longest stream
     unsigned long long iter_limit = 0; // test knob: iteration bound of the device loops (0 = their own)
+    int share_mode = 0;                // shared-prefix evaluation: 0 when it pays, 1 always (tests), 2 never
+    int32_t parent[IL_MAX_STAGES] = {};
     int cpw = 1;                       // lane kernel: candidates per warp
     size_t smem_lane = 0;
     uint8_t *d_bits = nullptr;
@@ -452,6 +454,164 @@ static void slab_regions(const il_estimator *e, SelectParams &sp)
     }
 }
 
+
+// ---- shared-prefix evaluation -------------------------------------------------------------------
+// Candidates that agree on the configurations of all stages on a path from the root have the same
+// completion stream at the end of that path; the batch is turned into the set of distinct (stage,
+// configuration, parent node) nodes, every node is simulated once, and each candidate's P99 and miss
+// count are put together from the nodes where its queries leave (prefix_kernel.cu).  Used when the
+// node count is at most a quarter of candidates x stages (exhaustive sweeps over per-stage choices);
+// *used tells whether the batch was evaluated here.
+constexpr int64_t kShareMinCandidates = 2048;
+constexpr int kShareMaxTop = 16384;
+
+static int estimate_shared(il_estimator *e, const il_stage_config *d_configs, int64_t n_cand, int64_t slo_us,
+                           int64_t *d_out_p99, int64_t *d_out_miss, char *ws, size_t ws_bytes, bool *used)
+{
+    *used = false;
+    const int S = e->S;
+    const int64_t n = e->n;
+    const int64_t allowed = n - (99 * n + 99) / 100;           // T: queries allowed above the P99
+    const int64_t top_len = allowed + 1;
+    if (e->share_mode == 2 || !e->can_pack || e->variant != IL_VARIANT_AUTO || top_len > kShareMaxTop ||
+        n_cand >= (INT64_C(1) << 30) || (e->share_mode == 0 && n_cand < kShareMinCandidates))
+        return IL_OK;
+    uint32_t cap = 1024;
+    while ((int64_t)cap < 2 * n_cand) cap <<= 1;
+
+    size_t off = 0;
+    auto take = [&](size_t bytes) { const size_t at = off; off = align_up(off + bytes, 256); return at; };
+    const size_t o_node_of = take((size_t)S * n_cand * 4), o_slot = take((size_t)n_cand * 4);
+    const size_t o_keys = take((size_t)cap * 8), o_vals = take((size_t)cap * 4);
+    const size_t o_cfg = take((size_t)S * n_cand * 4), o_par = take((size_t)S * n_cand * 4);
+    const size_t o_count = take((size_t)IL_MAX_STAGES * 4), o_work = take((size_t)IL_MAX_STAGES * 8);
+    if (off > ws_bytes) return IL_OK;
+    int32_t *node_of = reinterpret_cast<int32_t *>(ws + o_node_of);
+    uint32_t *node_cfg = reinterpret_cast<uint32_t *>(ws + o_cfg);
+    int32_t *node_par = reinterpret_cast<int32_t *>(ws + o_par);
+    int *d_count = reinterpret_cast<int *>(ws + o_count);
+    unsigned long long *d_work = reinterpret_cast<unsigned long long *>(ws + o_work);
+
+    int rc = ensure_events(e, 5);
+    if (rc) return rc;
+    cudaStream_t st = e->stream;
+    IL_CUDA(cudaMemsetAsync(e->d_counters, 0, kCounters * sizeof(unsigned long long), st));
+    IL_CUDA(cudaMemsetAsync(e->d_status, 0, sizeof(int), st));
+    IL_CUDA(cudaMemsetAsync(d_count, 0, (size_t)IL_MAX_STAGES * 4, st));
+    IL_CUDA(cudaMemsetAsync(d_work, 0, (size_t)IL_MAX_STAGES * 8, st));
+    IL_CUDA(cudaEventRecord(e->events[0], st));
+    for (int s = 0; s < S; s++)
+        IL_CUDA(launch_prefix_stage(d_configs, n_cand, S, s, e->H, e->Bmax,
+                                    s == 0 ? nullptr : node_of + (size_t)e->parent[s] * n_cand,
+                                    reinterpret_cast<uint64_t *>(ws + o_keys), cap,
+                                    reinterpret_cast<int32_t *>(ws + o_vals), reinterpret_cast<int32_t *>(ws + o_slot),
+                                    d_count + s, node_cfg + (size_t)s * n_cand, node_par + (size_t)s * n_cand,
+                                    node_of + (size_t)s * n_cand, e->d_status, st));
+    int h_count[IL_MAX_STAGES];
+    IL_CUDA(cudaMemcpyAsync(h_count, d_count, (size_t)IL_MAX_STAGES * 4, cudaMemcpyDeviceToHost, st));
+    IL_CUDA(cudaMemcpyAsync(e->h_status, e->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+    IL_CUDA(cudaStreamSynchronize(st));
+    if (*e->h_status) { *used = true; return *e->h_status; }       // an invalid candidate: the call fails here
+    int64_t total_nodes = 0;
+    for (int s = 0; s < S; s++) total_nodes += h_count[s];
+    if (e->share_mode == 0 && total_nodes * 4 > n_cand * S) return IL_OK;
+
+    // streams between the nodes, leaving records, top lists and miss counts
+    int64_t leaving[IL_MAX_STAGES], stride_in[IL_MAX_STAGES], stride_ex[IL_MAX_STAGES];
+    size_t o_in[IL_MAX_STAGES] = {}, o_ex[IL_MAX_STAGES] = {}, o_top[IL_MAX_STAGES] = {}, o_miss[IL_MAX_STAGES] = {};
+    for (int s = 0; s < S; s++) {
+        const int a = e->base.dest_a[s], b = e->base.dest_b[s];
+        int64_t kids = 0;
+        if (a >= 0) kids += e->visits[a];
+        if (b >= 0 && b != a) kids += e->visits[b];
+        leaving[s] = e->visits[s] - kids;
+        stride_in[s] = (e->visits[s] + 3) / 4 * 4;
+        stride_ex[s] = (leaving[s] + 3) / 4 * 4;
+        if (s > 0 && e->visits[s] > 0)
+            o_in[s] = take((size_t)h_count[e->parent[s]] * stride_in[s] * 8);
+        if (leaving[s] > 0) {
+            o_ex[s] = take((size_t)h_count[s] * stride_ex[s] * 8);
+            o_top[s] = take((size_t)h_count[s] * top_len * 8);
+            o_miss[s] = take((size_t)h_count[s] * 8);
+        }
+    }
+    if (off > ws_bytes) return IL_OK;
+    *used = true;
+
+    int64_t launches = 3 * S;
+    for (int s = 0; s < S; s++) {
+        if (e->visits[s] == 0) continue;
+        const int a = e->base.dest_a[s], b = e->base.dest_b[s];
+        NodeStageParams np = {};
+        np.lat_stage = e->d_lat + (size_t)s * e->H * e->Bmax;
+        np.bits = e->d_bits; np.ptrace = e->d_ptrace;
+        np.qbits = e->base.qbits; np.H = e->H; np.Bmax = e->Bmax;
+        np.n_queries = (int32_t)e->n;
+        np.n_in = (int32_t)e->visits[s];
+        np.bit = e->base.bit[s];
+        np.n_nodes = h_count[s];
+        np.node_cfg = node_cfg + (size_t)s * n_cand;
+        np.node_parent = node_par + (size_t)s * n_cand;
+        np.in = s == 0 ? nullptr : reinterpret_cast<const uint64_t *>(ws + o_in[s]);
+        np.stride_in = stride_in[s];
+        uint64_t *ex = reinterpret_cast<uint64_t *>(ws + o_ex[s]);
+        np.out_a = a >= 0 ? reinterpret_cast<uint64_t *>(ws + o_in[a]) : ex;
+        np.stride_a = a >= 0 ? stride_in[a] : stride_ex[s];
+        np.out_b = b >= 0 ? reinterpret_cast<uint64_t *>(ws + o_in[b]) : ex;
+        np.stride_b = b >= 0 ? stride_in[b] : stride_ex[s];
+        np.work = d_work + s;
+        np.counters = e->d_counters;
+        np.status = e->d_status;
+        const int grid = (int)std::min<int64_t>((h_count[s] + kWarpsPerCta - 1) / kWarpsPerCta,
+                                                (int64_t)e->num_sms * kOneWaveCtasPerSm);
+        IL_CUDA(launch_node_stage(np, grid, st));
+        launches++;
+    }
+    IL_CUDA(cudaEventRecord(e->events[1], st));
+    CombineParams cp = {};
+    cp.n_cand = n_cand; cp.node_of = node_of; cp.top_len = (int32_t)top_len; cp.allowed = allowed;
+    cp.out_p99 = d_out_p99; cp.out_miss = d_out_miss;
+    for (int s = 0; s < S; s++) {
+        if (leaving[s] <= 0) continue;
+        NodeTopParams tp = {};
+        tp.records = reinterpret_cast<uint64_t *>(ws + o_ex[s]);
+        tp.stride = stride_ex[s]; tp.len = (int32_t)leaving[s];
+        tp.arrival = e->d_arrival; tp.qbits = e->base.qbits; tp.slo_us = slo_us;
+        tp.top_len = (int32_t)top_len;
+        tp.top = reinterpret_cast<int64_t *>(ws + o_top[s]);
+        tp.miss = reinterpret_cast<int64_t *>(ws + o_miss[s]);
+        tp.n_nodes = h_count[s];
+        IL_CUDA(launch_node_top(tp, st));
+        launches++;
+        cp.exit_stage[cp.n_exit] = s;
+        cp.top[cp.n_exit] = tp.top;
+        cp.miss[cp.n_exit] = tp.miss;
+        cp.n_exit++;
+    }
+    IL_CUDA(launch_prefix_combine(cp, st));
+    launches++;
+    IL_CUDA(cudaEventRecord(e->events[2], st));
+    IL_CUDA(cudaMemcpyAsync(e->h_counters, e->d_counters, kCounters * sizeof(unsigned long long),
+                            cudaMemcpyDeviceToHost, st));
+    IL_CUDA(cudaMemcpyAsync(e->h_status, e->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+    IL_CUDA(cudaStreamSynchronize(st));
+    float ms = 0.f;
+    IL_CUDA(cudaEventElapsedTime(&ms, e->events[0], e->events[1]));
+    e->stats.sim_ms = ms;
+    IL_CUDA(cudaEventElapsedTime(&ms, e->events[1], e->events[2]));
+    e->stats.select_ms = ms;
+    e->stats.total_ms = e->stats.sim_ms + e->stats.select_ms;
+    e->stats.candidates = n_cand;
+    e->stats.query_events = n_cand * e->events_per_candidate;
+    e->stats.batches = (int64_t)e->h_counters[1];
+    e->stats.algorithmic_ops = (int64_t)e->h_counters[2];
+    e->stats.chunks = 1;
+    e->stats.kernel_launches = launches;
+    e->stats.error_detail = (int64_t)e->h_counters[5];
+    e->stats.stage_runs = total_nodes;
+    return *e->h_status;
+}
+
 extern "C" {
 
 const char *il_strerror(int code)
@@ -467,6 +627,7 @@ const char *il_strerror(int code)
     case IL_ERR_CUDA: return "CUDA call failed";
     case IL_ERR_ITER_LIMIT: return "device loop exceeded its iteration bound";
     case IL_ERR_TOO_LARGE: return "request needs more than the built-in static scratch (IL_STATIC_SCRATCH_BYTES)";
+    case IL_ERR_BOUNDS: return "a device index left its array (checked build)";
     default: return "unknown error";
     }
 }
@@ -533,6 +694,7 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
             if (pr->cond_val[c] == 0) bp.dest_a[par] = (int8_t)c; else bp.dest_b[par] = (int8_t)c;
         }
     }
+    for (int s = 0; s < S; s++) e->parent[s] = pr->parent[s];
     e->visits[0] = n;
     for (int64_t q = 0; q < n; q++) {   // walk every query down its path
         int s = 0;
@@ -640,6 +802,11 @@ int il_set_test_knob(il_estimator *e, int knob, int64_t value)
         configure_lane_rings(e);
         return IL_OK;
     }
+    if (knob == IL_KNOB_SHARE_PREFIXES) {
+        if (value < 0 || value > 2) return IL_ERR_INVALID_ARG;
+        e->share_mode = (int)value;
+        return IL_OK;
+    }
     if (knob == IL_KNOB_ITER_LIMIT) {
         if (value < 0) return IL_ERR_INVALID_ARG;
         e->iter_limit = (unsigned long long)value;
@@ -711,6 +878,9 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
     size_t ws_bytes = 0;
     int wrc = acquire_workspace(e, n_cand, &ws, &ws_bytes);
     if (wrc) return wrc;
+    bool shared = false;
+    int src = estimate_shared(e, d_configs, n_cand, slo_us, d_out_p99, d_out_miss, ws, ws_bytes, &shared);
+    if (shared || src) return src;
     Plan pl;
     if (!make_plan(e, ws_bytes, n_cand, pl)) return IL_ERR_NOMEM;
 
@@ -752,6 +922,7 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
         SelectParams sp = {};
         sp.slab = p.slab; sp.slab_stride = e->n_pad; sp.lat_or = p.lat_or;
         sp.arrival = e->d_arrival; sp.qbits = p.qbits; sp.packed = use_packed(e) ? 1 : 0;
+        sp.status = e->d_status;
         if (lane) {
             slab_regions(e, sp);
             if (e->lane_wrap) sp.ovf = p.ovf;
@@ -895,6 +1066,20 @@ int il_feasible_device(il_estimator *e, const il_stage_config *d_configs, int64_
     size_t ws_bytes = 0;
     int rc = acquire_workspace(e, std::min<int64_t>(n_cand, 4096), &ws, &ws_bytes);
     if (rc) return rc;
+    if (e->share_mode == 1 || (e->share_mode == 0 && n_cand >= kShareMinCandidates)) {
+        // a batch full of common configuration prefixes is cheaper to evaluate node by node
+        rc = ensure_staging(e, n_cand);
+        if (rc) return rc;
+        bool shared = false;
+        rc = estimate_shared(e, d_configs, n_cand, slo_us, e->d_out, e->d_out + e->d_out_cap, ws, ws_bytes, &shared);
+        if (rc) return rc;
+        if (shared) {
+            IL_CUDA(launch_feasible_from_p99(e->d_out, nullptr, n_cand, slo_us, d_out_feasible, st));
+            IL_CUDA(cudaStreamSynchronize(st));
+            e->stats.kernel_launches++;
+            return IL_OK;
+        }
+    }
     const int64_t wpc = des_lane_warps_per_cta();
     const size_t sb = slot_time_bytes(e);
     const size_t tail_bytes = align_up((size_t)n_cand, 256) + align_up((size_t)n_cand * 4, 256) + 1024;

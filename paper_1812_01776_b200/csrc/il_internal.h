@@ -5,6 +5,17 @@
 #include <stdint.h>
 #include "il_estimator.h"
 
+// Checked build (-DIL_CHECKED): every index into a stream, ring, slab or bound input that a kernel
+// computes is compared with the size of its array first; an index outside is recorded as
+// IL_ERR_BOUNDS in the status word and the access is skipped, so that a wrong index shows up as an
+// error code and never as a fault.  In the normal build the macro is the constant true.
+#ifdef IL_CHECKED
+#define IL_IN_RANGE(idx, size, status) \
+    ((unsigned long long)(idx) < (unsigned long long)(size) ? true : (atomicCAS((status), 0, IL_ERR_BOUNDS), false))
+#else
+#define IL_IN_RANGE(idx, size, status) true
+#endif
+
 namespace il {
 
 constexpr int kWarpsPerCta = 4;
@@ -68,6 +79,7 @@ struct SelectParams {
     const uint64_t *lat_or;       // [n_cand]: OR of the latencies (wide kernel)
     const uint8_t *ovf;           // if set: candidates whose row does not have the region layout (they were
                                   // evaluated by the warp-per-candidate kernel after a ring overflow)
+    int *status;                  // checked build: where an index out of range is recorded
     int32_t n;
     int64_t n_cand;
     int64_t slo_us;
@@ -121,6 +133,7 @@ struct NodeStageParams {
     const uint8_t *bits;          // [n] branch bits
     const uint64_t *ptrace;       // packed trace (root stage)
     int32_t qbits, H, Bmax;
+    int32_t n_queries;            // length of the trace (and of bits)
     int32_t n_in;                 // queries visiting the stage
     int32_t bit;                  // branch bit tested after the stage, -1 = none
     int64_t n_nodes;

@@ -62,7 +62,8 @@ select_kernel(const __grid_constant__ SelectParams p)
                     uint32_t l = 0;
                     if (i < p.n) {
                         const uint64_t rec = (uint64_t)lat[i];
-                        l = (uint32_t)((int64_t)(rec >> p.qbits) - p.arrival[rec & qmask]);
+                        if (IL_IN_RANGE(rec & qmask, p.n, p.status))
+                            l = (uint32_t)((int64_t)(rec >> p.qbits) - p.arrival[rec & qmask]);
                         miss += ((int64_t)l > p.slo_us);
                     }
                     __syncthreads();        // all records of this block are read before their row space is reused
@@ -114,7 +115,8 @@ select_kernel(const __grid_constant__ SelectParams p)
             unsigned long long my_or = 0;
             for (int i = threadIdx.x; i < p.n; i += kSelectThreads) {
                 const uint64_t rec = (uint64_t)lat[i];
-                const int64_t l = (int64_t)(rec >> p.qbits) - p.arrival[rec & qmask];
+                int64_t l = 0;
+                if (IL_IN_RANGE(rec & qmask, p.n, p.status)) l = (int64_t)(rec >> p.qbits) - p.arrival[rec & qmask];
                 lat[i] = l;
                 my_or |= (unsigned long long)l;
                 miss += (l > p.slo_us);

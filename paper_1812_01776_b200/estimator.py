@@ -15,16 +15,19 @@ from typing import Optional, Tuple
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libil_estimator.so")
+# IL_ESTIMATOR_CHECKED=1 in the environment selects the bounds-checked build of the same sources
+_LIB_PATH = os.path.join(_HERE, "libil_estimator_checked.so" if os.environ.get("IL_ESTIMATOR_CHECKED") == "1"
+                         else "libil_estimator.so")
 _lib = None
 
 IL_OK = 0
 IL_ERR_INVALID_ARG, IL_ERR_BAD_TOPOLOGY, IL_ERR_BAD_PROFILE, IL_ERR_BAD_TRACE = -1, -2, -3, -4
 IL_ERR_BAD_CONFIG, IL_ERR_NOMEM, IL_ERR_CUDA, IL_ERR_ITER_LIMIT = -5, -6, -7, -8
 IL_ERR_TOO_LARGE = -9
+IL_ERR_BOUNDS = -10
 IL_VARIANT_AUTO, IL_VARIANT_WIDE, IL_VARIANT_STAGED, IL_VARIANT_LANES, IL_VARIANT_PACKED = 0, 1, 2, 3, 4
 IL_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
-IL_KNOB_LANE_RING_LOG2, IL_KNOB_ITER_LIMIT = 1, 2
+IL_KNOB_LANE_RING_LOG2, IL_KNOB_ITER_LIMIT, IL_KNOB_SHARE_PREFIXES = 1, 2, 3
 
 EXPORTS = ["il_estimator_create", "il_estimator_destroy", "il_estimate", "il_estimate_device",
            "il_set_stream", "il_workspace_bytes", "il_workspace_min_bytes", "il_set_workspace",

@@ -40,11 +40,11 @@ def test_binding_lists_every_declared_symbol():
 
 def test_strerror_covers_codes(lib):
     seen = set()
-    for code in range(0, -9, -1):
+    for code in range(0, -11, -1):
         msg = lib.il_strerror(code).decode()
         assert msg and msg != "unknown error"
         seen.add(msg)
-    assert len(seen) == 9
+    assert len(seen) == 11
     assert lib.il_strerror(-99).decode() == "unknown error"
 
 

@@ -344,8 +344,15 @@ def test_config3_full_size_sample_4096(il, oracle_on):
 
 def test_config5_full_size_sample_1024(il, oracle_on):
     """All 1,048,576 candidates x 100,000 queries of the 8-stage tree (R up to 32, max batch up
-    to 64) on the GPU; a seeded sample of 1,024 candidates and 16 extremes against the oracle."""
+    to 64) on the GPU; a seeded sample of 1,024 candidates and 16 extremes against the oracle.  The
+    candidate set is a product of per-stage choices, so the full sweep goes through the shared-prefix
+    path; the sampled candidates are also run on the lane kernel alone."""
     _sampled_check(il, oracle_on, 5)
+    w, idx, ext = full_size_sample(5)
+    exp = oracle_on("w5", w, np.concatenate([w.configs[idx], ext]))
+    got = gpu_run(il, w, configs=w.configs[idx], host=False, knobs={3: 2})
+    assert got[2]["stage_runs"] == idx.shape[0] * w.n_stages
+    assert np.array_equal(got[0], exp[0][:idx.shape[0]]) and np.array_equal(got[1], exp[1][:idx.shape[0]])
 
 
 @pytest.mark.parametrize("variant", [0, 4], ids=["auto", "packed"])
