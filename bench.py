@@ -57,6 +57,7 @@ NCU_CAPTURES = {
         "dram_bytes_per_query_event": 12.24, "warp_inst_per_query_event": 32.9,
         "summary": "profiles/des_packed_kernel_config2.md"},
 }
+LANE_CTAS = None         # --lane-ctas: resident CTAs per SM of the lane kernel, for side measurements
 RING_LOG2 = None         # --ring-log2: ring length of the lane kernel's streams, for side measurements
 METRIC = "candidate_configs_per_s"
 UNIT = "candidates/s"
@@ -275,6 +276,8 @@ def measure(il, torch, w, dev, stream, flush, steps, warmup, e2e_steps, variant,
     est.set_variant(variant)
     if RING_LOG2 is not None:
         est.set_test_knob(1, RING_LOG2)
+    if LANE_CTAS is not None:
+        est.set_test_knob(4, LANE_CTAS)
     kernel = est.kernel_name()
     ws_bytes = est.reserve_workspace(n_cand)
     cfg_pinned = torch.from_numpy(cfg_host).pin_memory()
@@ -331,14 +334,27 @@ def measure(il, torch, w, dev, stream, flush, steps, warmup, e2e_steps, variant,
     est.close()
 
     n, S = w.n_queries, w.n_stages
+    shared = bool(st.get("stage_runs")) and st["stage_runs"] < n_cand * S
+    if shared:
+        kernel = "des_node_stage_kernel (shared configuration prefixes: every distinct stage run simulated once)"
     sim_s = statistics.mean(sim_ms) * 1e-3
     sel_s = statistics.mean(sel_ms) * 1e-3
     total_events = events_per_cand * n_cand
     rec_bytes = 12 if kernel == "des_kernel" else 8  # separate time/query streams, else one 64-bit record
     slab_bytes = 8 * n * n_cand                       # written once by the simulation, read once by the select
     stream_bytes = (events_per_cand - n) * 2 * rec_bytes * n_cand   # written once, read once
-    cap = ncu_capture(kernel)
+    cap = None if shared else ncu_capture(kernel)
     alu_peak = issue_rate * 32.0
+    hbm_note = ("latency slab written once + every inter-stage stream record written once "
+                "and read once (the streams are this design's, not the method's)")
+    if shared:
+        # only the distinct stage runs move data: per run its arrival stream read and its output written
+        # (about 16 B per simulated query-event); the method's own count does not apply
+        simulated_events = total_events * st["stage_runs"] / float(n_cand * S)
+        stream_bytes = 16.0 * simulated_events
+        slab_bytes = 0
+        hbm_note = ("shared prefixes: about 16 B per SIMULATED query-event (stage_runs_simulated / "
+                    "stage_runs_of_the_method of the method's count), no slab")
     rec = {
         "candidates": n_cand, "queries": n, "stages": S, "query_events_per_candidate": events_per_cand,
         "kernel": kernel, "workspace_bytes": ws_bytes, "steps": steps, "warmup": warmup,
@@ -370,14 +386,14 @@ def measure(il, torch, w, dev, stream, flush, steps, warmup, e2e_steps, variant,
         "roofline_hbm": {"bound": "hbm", "kernel": kernel, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "achieved": (slab_bytes + stream_bytes) / sim_s / 1e9,
                          "frac": (slab_bytes + stream_bytes) / sim_s / 1e9 / peaks["hbm_gbs"],
-                         "bytes": "latency slab written once + every inter-stage stream record written once "
-                                  "and read once (the streams are this design's, not the method's)",
+                         "bytes": hbm_note,
                          "slab_only_achieved": slab_bytes / sim_s / 1e9,
                          "slab_only_frac": slab_bytes / sim_s / 1e9 / peaks["hbm_gbs"]},
         "roofline_select": {"bound": "hbm", "kernel": "select_kernel", "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                            "achieved": slab_bytes / sel_s / 1e9 if sel_s > 0 else None,
-                            "frac": slab_bytes / sel_s / 1e9 / peaks["hbm_gbs"] if sel_s > 0 else None,
-                            "bytes": "8 n per candidate, read once"},
+                            "achieved": slab_bytes / sel_s / 1e9 if sel_s > 0 and not shared else None,
+                            "frac": slab_bytes / sel_s / 1e9 / peaks["hbm_gbs"] if sel_s > 0 and not shared else None,
+                            "bytes": "8 n per candidate, read once" if not shared else
+                                     "shared prefixes: per-node top lists and a per-candidate combine instead"},
     }
     if clocks is not None:
         rec["clocks"] = clocks
@@ -555,11 +571,14 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5, help="host-buffer steps timed (at most --steps)")
     ap.add_argument("--no-per-workload", action="store_true",
                     help="skip the short measurements of the other workloads")
+    ap.add_argument("--lane-ctas", type=int, default=None,
+                    help="resident CTAs per SM of the lane kernel (side measurements; default 4)")
     ap.add_argument("--ring-log2", type=int, default=None,
                     help="largest stream ring of the lane kernel, log2 records (side measurements; default 13)")
     args = ap.parse_args()
-    global RING_LOG2
+    global RING_LOG2, LANE_CTAS
     RING_LOG2 = args.ring_log2
+    LANE_CTAS = args.lane_ctas
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -368,11 +368,14 @@ IL_API int il_set_variant(il_estimator *est, int variant);
  *   IL_KNOB_SHARE_PREFIXES  0: the library decides per call whether to evaluate a batch through shared
  *                           configuration prefixes (see il_estimate_device); 1: always, when the
  *                           preconditions hold; 2: never.
+ *   IL_KNOB_LANE_CTAS       value 0..16: resident CTAs (of two warps) per SM of the lane kernel; 0 restores
+ *                           the library's choice (4).  For measurements.
  * Set a knob before il_workspace_bytes / il_set_workspace: sizes depend on the ring length.
  */
 #define IL_KNOB_LANE_RING_LOG2 1
 #define IL_KNOB_ITER_LIMIT 2
 #define IL_KNOB_SHARE_PREFIXES 3
+#define IL_KNOB_LANE_CTAS 4
 IL_API int il_set_test_knob(il_estimator *est, int knob, int64_t value);
 
 /* Name of the simulation kernel the handle's next estimate call will launch

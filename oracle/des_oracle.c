@@ -31,9 +31,15 @@
  *     batch) queries from the front of the FIFO queue at once; the lowest-id
  *     idle replica goes first.
  *   - Batch-mates enter the next stage's queue in the order they had in the
- *     batch.  A query follows the one child edge whose condition its branch
- *     bits satisfy; if there is none it leaves the pipeline and its latency is
- *     clock - arrival time.  There is no delay between stages.
+ *     batch.  A query follows EVERY child edge whose condition its branch bits
+ *     satisfy (Section 2: the pipeline is a DAG whose edges are dataflow; two
+ *     unconditional children are two branches that work on the query in
+ *     parallel); where it follows none, that copy of the query leaves the
+ *     pipeline.  The query is answered when its last copy has left, and its
+ *     latency is that instant - arrival time (Section 4.3 measures the service
+ *     time along the LONGEST path of the DAG).  With mutually exclusive
+ *     conditions (the conditional control flow of Section 2) there is one copy
+ *     and one path.  There is no delay between stages.
  *   - Batch time is a dense table lookup lat[stage][hw][b-1] for the actual
  *     batch size b.
  *   - P99 is the k-th smallest latency, k = ceil(0.99 n) computed in integers
@@ -115,9 +121,8 @@ static int cmp_i64(const void *a, const void *b)
     return (x > y) - (x < y);
 }
 
-/* Checks the tree: parent[0] = -1, parent[s] < s, and the children of one
- * parent are either a single unconditional child or children guarded by the
- * same bit with distinct values (so at most one edge is taken per query). */
+/* Checks the tree: parent[0] = -1, parent[s] < s, at most two children per
+ * stage, each edge unconditional or guarded by one branch bit. */
 static int check_topology(int S, const int32_t *parent, const int8_t *cond_bit,
                           const uint8_t *cond_val)
 {
@@ -128,17 +133,9 @@ static int check_topology(int S, const int32_t *parent, const int8_t *cond_bit,
         if (cond_bit[s] >= 0 && cond_val[s] > 1) return ORC_ERR_TOPOLOGY;
     }
     for (int p = 0; p < S; p++) {
-        int nchild = 0, first = -1;
-        for (int c = 1; c < S; c++) {
-            if (parent[c] != p) continue;
-            if (nchild == 0) first = c;
-            else {
-                if (cond_bit[first] < 0 || cond_bit[c] < 0) return ORC_ERR_TOPOLOGY;
-                if (cond_bit[c] != cond_bit[first]) return ORC_ERR_TOPOLOGY;
-                if (cond_val[c] == cond_val[first]) return ORC_ERR_TOPOLOGY;
-            }
-            if (++nchild > 2) return ORC_ERR_TOPOLOGY;
-        }
+        int nchild = 0;
+        for (int c = 1; c < S; c++)
+            if (parent[c] == p && ++nchild > 2) return ORC_ERR_TOPOLOGY;
     }
     return ORC_OK;
 }
@@ -193,8 +190,9 @@ int orc_estimate_one(int32_t S, int32_t H, int32_t Bmax,
     int32_t *inflight_n[16];
     int64_t *lat = (int64_t *)malloc(sizeof(int64_t) * (size_t)n);
     uint8_t *done = (uint8_t *)calloc((size_t)n, 1);
+    int32_t *copies = (int32_t *)malloc(sizeof(int32_t) * (size_t)n);   /* copies of the query still in the pipeline */
     heap.e = (event_t *)malloc(sizeof(event_t) * (size_t)heap.cap);
-    int ok = lat && done && heap.e;
+    int ok = lat && done && copies && heap.e;
     for (int s = 0; s < S; s++) {
         queue[s] = (int32_t *)malloc(sizeof(int32_t) * (size_t)n);
         busy[s] = (uint8_t *)calloc((size_t)R[s], 1);
@@ -210,6 +208,7 @@ int orc_estimate_one(int32_t S, int32_t H, int32_t Bmax,
     for (int64_t i = 0; i < n; i++) {
         event_t ev = { arrival_us[i], i, EV_ARRIVAL, 0, 0, (int32_t)i };
         heap_push(&heap, ev);
+        copies[i] = 1;
     }
 
     while (heap.size > 0) {
@@ -222,20 +221,21 @@ int orc_estimate_one(int32_t S, int32_t H, int32_t Bmax,
             busy[s][r] = 0;
             for (int j = 0; j < inflight_n[s][r]; j++) {
                 int32_t q = inflight[s][r * MB[s] + j];
-                int child = -1;
-                for (int c = s + 1; c < S && child < 0; c++) {
+                int taken = 0;
+                for (int c = s + 1; c < S; c++) {
                     if (parent[c] != s) continue;
                     if (cond_bit[c] < 0 ||
-                        (uint8_t)((branch_bits[q] >> cond_bit[c]) & 1) == cond_val[c])
-                        child = c;
+                        (uint8_t)((branch_bits[q] >> cond_bit[c]) & 1) == cond_val[c]) {
+                        queue[c][qtail[c]++] = q;
+                        taken++;
+                    }
                 }
-                if (child < 0) {
-                    if (done[q]) { rc = ORC_ERR_INTERNAL; goto cleanup; }
+                if (done[q]) { rc = ORC_ERR_INTERNAL; goto cleanup; }
+                copies[q] += taken - 1;      /* this copy went on as `taken` copies, or left */
+                if (copies[q] == 0) {        /* the last copy has left: the query is answered now */
                     done[q] = 1;
                     lat[q] = clock - arrival_us[q];
                     n_done++;
-                } else {
-                    queue[child][qtail[child]++] = q;
                 }
             }
             inflight_n[s][r] = 0;
@@ -282,7 +282,7 @@ int orc_estimate_one(int32_t S, int32_t H, int32_t Bmax,
     }
 
 cleanup:
-    free(lat); free(done); free(heap.e);
+    free(lat); free(done); free(copies); free(heap.e);
     for (int s = 0; s < S; s++) { free(queue[s]); free(busy[s]); free(inflight[s]); free(inflight_n[s]); }
     return rc;
 }

@@ -87,7 +87,6 @@ namespace il {
 namespace {
 
 constexpr int kLaneWarps = 2;                  // warps per CTA
-constexpr int kRing = 32;                      // ring positions of a lane's slot list (>= IL_MAX_REPLICAS)
 constexpr uint32_t kDone = 0x80000000u;
 constexpr uint64_t kInf = ~0ull;
 constexpr uint32_t kAbort = 0xffffffffu;      // ring mailbox: the candidate is given up (ring overflow)
@@ -105,34 +104,56 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// Shared memory of one warp.
+// Shared memory of one warp, laid out for the launch: the batch ring has `kr` positions (a power of
+// two of at least the largest replica count of the launch's candidates; 16 or 32) and the profile copy
+// Bmax rows, so a launch pays only for what its candidates need.
 struct WarpMem {
     // Per lane a ring of batches, [pos][lane].  Positions [epos, lpos): batches whose slot has been
     // taken over, waiting to be handed on, in key order.  Positions [lpos, tpos): the slots in use,
     // sorted by key.
-    uint64_t key[kRing][32];     // (finish << q) | index of the batch's first arrival
-    uint32_t cnt[kRing][32];     // batch size
+    uint64_t (*key)[32];         // [kr] (finish << q) | index of the batch's first arrival
+    uint32_t (*cnt)[32];         // [kr] batch size
     // The lane's row of the profile, [b - 1][lane]: time of a batch of b on the stage's hardware type.
     // One copy per lane, so that lanes with different rows or batch sizes never meet in a bank.
-    uint32_t lat[IL_MAX_BATCH][32];
+    uint32_t (*lat)[32];         // [Bmax]
     // Staging rings filled by cp.async, [position][lane]: the next records of the lane's arrival stream
     // (position = record index mod kStage), and the records it is handing on with the finish << q of
     // their batch (position = iteration mod kStage)
-    uint64_t stage_x[kStage][32];
-    uint64_t stage_e[kStage][32];
-    uint64_t stage_b[kStage][32];
+    uint64_t (*stage_x)[32];     // [kStage]
+    uint64_t (*stage_e)[32];
+    uint64_t (*stage_b)[32];
     // Mailboxes, double-buffered by iteration parity: what iteration k publishes in buffer k & 1 is read
     // in iteration k + 1, while iteration k + 1 publishes into the other buffer; one warp barrier per
     // iteration then separates every write of a word from the reads of its previous value.
-    uint32_t avail[2][32];       // records written so far into the lane's arrival stream (by its parent
+    uint32_t (*avail)[32];       // [2] records written so far into the lane's arrival stream (by its parent
                                  // lane); kDone set once that is all of them
     // Ring streams only: index below which the lane needs no record of its arrival stream any more
     // (its parent may overwrite those ring positions), or kAbort.  Grows monotonically; a reader that
     // sees an older value only waits longer.
-    uint32_t freed[32];
+    uint32_t *freed;             // [32]
     // Feasibility only: queries of the group's candidate that have missed the objective so far, [group]
-    uint32_t miss[32];
+    uint32_t *miss;              // [32]
 };
+
+__host__ __device__ inline size_t warp_mem_bytes(int kr, int Bmax)
+{
+    return (size_t)kr * 32 * 12 + (size_t)3 * kStage * 32 * 8 + (size_t)(2 + 1 + 1) * 32 * 4 + (size_t)Bmax * 32 * 4;
+}
+
+__device__ __forceinline__ WarpMem warp_mem_at(unsigned char *base, int kr, int Bmax)
+{
+    WarpMem wm;
+    wm.key = reinterpret_cast<uint64_t (*)[32]>(base);          base += (size_t)kr * 256;
+    wm.stage_x = reinterpret_cast<uint64_t (*)[32]>(base);      base += (size_t)kStage * 256;
+    wm.stage_e = reinterpret_cast<uint64_t (*)[32]>(base);      base += (size_t)kStage * 256;
+    wm.stage_b = reinterpret_cast<uint64_t (*)[32]>(base);      base += (size_t)kStage * 256;
+    wm.cnt = reinterpret_cast<uint32_t (*)[32]>(base);          base += (size_t)kr * 128;
+    wm.lat = reinterpret_cast<uint32_t (*)[32]>(base);          base += (size_t)Bmax * 128;
+    wm.avail = reinterpret_cast<uint32_t (*)[32]>(base);        base += 256;
+    wm.freed = reinterpret_cast<uint32_t *>(base);              base += 128;
+    wm.miss = reinterpret_cast<uint32_t *>(base);
+    return wm;
+}
 
 }  // namespace
 
@@ -148,7 +169,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
     extern __shared__ __align__(16) unsigned char smem_raw[];
     int32_t *s_lat = reinterpret_cast<int32_t *>(smem_raw);      // the profile tables, [S][H][Bmax]
     const int n_tab = p.S * p.H * p.Bmax;
-    WarpMem *wm_all = reinterpret_cast<WarpMem *>(smem_raw + ((size_t)n_tab * 4 + 15) / 16 * 16);
+    unsigned char *wm_base = smem_raw + ((size_t)n_tab * 4 + 15) / 16 * 16;
     const int q = p.qbits;
     const uint64_t qmask = (1ull << q) - 1ull;
     for (int i = threadIdx.x; i < n_tab; i += blockDim.x)
@@ -158,7 +179,8 @@ des_lane_kernel(const __grid_constant__ DesParams p)
     const unsigned full = 0xffffffffu;
     const int wid = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    WarpMem &wm = wm_all[wid];
+    const uint32_t kr = (uint32_t)p.lane_slots, rmask = kr - 1u;      // batch ring positions of a lane
+    const WarpMem wm = warp_mem_at(wm_base + (size_t)wid * warp_mem_bytes((int)kr, p.Bmax), (int)kr, p.Bmax);
     const int S = p.S, cpw = p.cpw;
     const int j = lane / S, s = lane - j * S;
     const bool lane_used = j < cpw;
@@ -235,6 +257,9 @@ des_lane_kernel(const __grid_constant__ DesParams p)
     uint32_t lim_a = 0xffffffffu, lim_b = 0xffffffffu;
     uint32_t low_pub = 0, low_new = 0, e_first = 0;
     bool low_pending = false, aborted = false;
+    // feasibility only: a leaving record waits one iteration for the arrival time of its query
+    uint64_t late_fin = 0, late_arr = 0;
+    bool late_valid = false;
     uint32_t av = 0;             // mailbox word this iteration works with: the one read an iteration ago
     int par = 0;                 // mailbox buffer this iteration publishes into; it reads the other one
     uint32_t it = 0;
@@ -272,7 +297,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                         uint32_t lo = head;
                         if (e_left > 0) lo = min(lo, e_first);
                         for (uint32_t pp = epos; pp != tpos; pp++)
-                            lo = min(lo, (uint32_t)wm.key[pp & (kRing - 1)][lane] & (uint32_t)qmask);
+                            lo = min(lo, (uint32_t)wm.key[pp & rmask][lane] & (uint32_t)qmask);
                         low_new = lo;
                         low_pending = true;
                     }
@@ -284,8 +309,11 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                 }
             }
             if (FEAS && has && !done && wm.miss[j] > p.miss_allow) done = true;   // same word, same moment: the whole group
+            // Feasibility only: a group moves on as soon as its own lanes have finished (candidates are
+            // dropped at very different points of the trace).  Otherwise the groups of a warp start their
+            // candidates together: they then walk the trace side by side and share its cache lines.
             const unsigned dm = __ballot_sync(full, done);
-            const bool turn = !exhausted && (dm & group_mask) == group_mask;
+            const bool turn = !exhausted && (FEAS ? (dm & group_mask) == group_mask : dm == full);
             if (__any_sync(full, turn)) {
                 // a candidate that was dropped (decided, given up, out of iterations) may still have
                 // copies under way into the lane's staging rings: let them land before the rings are reused
@@ -358,6 +386,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                     lim_b = (RING && lane_b >= 0) ? K : 0xffffffffu;
                     low_pub = 0; low_new = 0; e_first = 0;
                     low_pending = false; aborted = false;
+                    late_valid = false;
                     av = avail0;
                 }
                 __syncwarp();     // the mailboxes are set before anybody reads them
@@ -374,19 +403,23 @@ des_lane_kernel(const __grid_constant__ DesParams p)
             const uint64_t h_base = wm.stage_b[h_sl][lane];
             uint32_t h_bits = 0;
             if (BRANCHY && h_valid && bit >= 0 && IL_IN_RANGE(h_qid, p.n, p.status)) h_bits = p.bits[h_qid];
-            // feasibility only: the arrival record of a query that may leave here, to test its latency
+            // feasibility only: the record that left in the previous iteration is tested now, its query's
+            // arrival record having had an iteration to come in; the arrival record of a query that may
+            // leave in this iteration is requested here
+            if (FEAS && late_valid && late_fin > (late_arr & ~qmask) + slo_q) atomicAdd(&wm.miss[j], 1u);
             uint64_t h_arr = 0;
             if (FEAS && h_valid && (da < 0 || (db < 0 && bit >= 0)) && IL_IN_RANGE(h_qid, p.n, p.status))
                 h_arr = p.ptrace[h_qid];
+            if (FEAS) late_valid = false;
             // likewise the next batch to hand on, if the one in hand is used up (a batch handed over in
             // this iteration is picked up in the next), and the table entry a close would need
             const bool f_valid = e_left == 0 && epos != lpos;
-            const uint64_t f_key = wm.key[epos & (kRing - 1)][lane];                      // unused unless f_valid
-            const uint32_t f_cnt = wm.cnt[epos & (kRing - 1)][lane];
+            const uint64_t f_key = wm.key[epos & rmask][lane];                      // unused unless f_valid
+            const uint32_t f_cnt = wm.cnt[epos & rmask][lane];
             // (latency << q) - qmask: finish key base = dispatch key + that
             const uint64_t latq = ((uint64_t)wm.lat[b > 0 ? b - 1 : 0][lane] << q) - qmask;
             // key of the second slot in use, the front after a hand-over (unused unless there are two)
-            uint64_t k2 = wm.key[(lpos + 1u) & (kRing - 1)][lane];
+            uint64_t k2 = wm.key[(lpos + 1u) & rmask][lane];
             const uint32_t written = av & ~kDone;
             const bool pdone = (av & kDone) != 0u;
             // ring streams: may this lane start handing on another record?  Not while a child's ring
@@ -400,7 +433,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
             const bool end = pdone && i >= written;
             const bool join = known && b > 0 && b < mb && ra <= tk;
             b += join ? 1 : 0;
-            const bool room = tpos - epos < (uint32_t)kRing;
+            const bool room = tpos - epos < kr;
             const bool close = b > 0 && !join && (known || end || b == mb) && room;
             // close and open as straight-line code under predicates (only the sorted insert branches),
             // so that the hand-on and request steps below can overlap with it
@@ -411,16 +444,16 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                 // a batch that finishes before one dispatched earlier
 #pragma unroll 1
                 while (pos != lpos) {
-                    const uint64_t prev = wm.key[(pos - 1) & (kRing - 1)][lane];
+                    const uint64_t prev = wm.key[(pos - 1) & rmask][lane];
                     if (prev <= key) break;
-                    wm.key[pos & (kRing - 1)][lane] = prev;
-                    wm.cnt[pos & (kRing - 1)][lane] = wm.cnt[(pos - 1) & (kRing - 1)][lane];
+                    wm.key[pos & rmask][lane] = prev;
+                    wm.cnt[pos & rmask][lane] = wm.cnt[(pos - 1) & rmask][lane];
                     pos--;
                 }
             }
             if (close) {
-                wm.key[pos & (kRing - 1)][lane] = key;
-                wm.cnt[pos & (kRing - 1)][lane] = (uint32_t)b;
+                wm.key[pos & rmask][lane] = key;
+                wm.cnt[pos & rmask][lane] = (uint32_t)b;
             }
             ktail = (close && !sorted_insert) ? key : ktail;
             const bool at_front = close && pos == lpos;
@@ -450,7 +483,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                 if (FEAS) {
                     const bool leaves = to_b ? db < 0 : da < 0;
                     if (h_valid && leaves) {
-                        if (h_base > (h_arr & ~qmask) + slo_q) atomicAdd(&wm.miss[j], 1u);
+                        late_valid = true; late_fin = h_base; late_arr = h_arr;
                     } else if (h_valid) {
                         uint64_t *dst = to_b ? out_b + (tail_b & mask_b) : out_a + (tail_a & mask_a);
                         if (IL_IN_RANGE(to_b ? (tail_b & mask_b) : (tail_a & mask_a), to_b ? size_b : size_a, p.status))
@@ -465,7 +498,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                 tail_a += (h_valid && !to_b) ? 1u : 0u;
             } else if (h_valid) {
                 if (FEAS && da < 0) {
-                    if (h_base > (h_arr & ~qmask) + slo_q) atomicAdd(&wm.miss[j], 1u);
+                    late_valid = true; late_fin = h_base; late_arr = h_arr;
                 } else if (IL_IN_RANGE(tail_a & mask_a, size_a, p.status)) {
                     out_a[tail_a & mask_a] = h_base | h_qid;
                 }
@@ -496,7 +529,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                     cp_async8(&wm.stage_x[fx & (kStage - 1)][lane], in + (fx & in_mask));
                 fx++;
             }
-            done = end && b == 0 && epos == tpos && e_left == 0 && vmask == 0u;
+            done = end && b == 0 && epos == tpos && e_left == 0 && vmask == 0u && !(FEAS && late_valid);
             if (--guard == 0) {
                 if (guard_hi == 0) { atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT); atomicOr(&p.counters[5], 1ull); done = true; }
                 else { guard_hi--; }      // guard wraps to 2^32 - 1 on the next decrement
@@ -566,9 +599,9 @@ cudaError_t launch_des_lane(const DesParams &p, int grid, size_t smem, cudaStrea
 
 int des_lane_warps_per_cta() { return kLaneWarps; }
 
-size_t des_lane_smem(int n_tab)
+size_t des_lane_smem(int n_tab, int Bmax, int ring_slots)
 {
-    return ((size_t)n_tab * 4 + 15) / 16 * 16 + (size_t)kLaneWarps * sizeof(WarpMem);
+    return ((size_t)n_tab * 4 + 15) / 16 * 16 + (size_t)kLaneWarps * warp_mem_bytes(ring_slots, Bmax);
 }
 
 int des_lane_max_ctas_per_sm(size_t smem)

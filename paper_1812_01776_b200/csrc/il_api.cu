@@ -53,7 +53,11 @@ struct il_estimator {
     int share_mode = 0;                // shared-prefix evaluation: 0 when it pays, 1 always (tests), 2 never
     int32_t parent[IL_MAX_STAGES] = {};
     int cpw = 1;                       // lane kernel: candidates per warp
-    size_t smem_lane = 0;
+    size_t smem_lane[2] = {0, 0};       // lane kernel with 16 / 32 batch ring positions per lane
+    int ctas_lane[2] = {0, 0};
+    int lane_slots = 32;               // batch ring positions used by the current call
+    int lane_ctas_knob = 0;            // test knob: resident CTAs per SM of the lane kernel (0: the library's choice)
+    int *d_maxrep = nullptr;           // device word: largest replica count of a batch
     uint8_t *d_bits = nullptr;
     int32_t *d_lat = nullptr;
     unsigned long long *d_counters = nullptr;   // [kCounters]: next candidate, batches, algorithmic ops,
@@ -136,9 +140,15 @@ size_t cand_bytes(const il_estimator *e) { return (size_t)e->n_pad * 8 + 13; }
 bool lane_fallback(const il_estimator *e) { return is_lane(e) && e->lane_wrap; }
 size_t fb_slot_bytes(const il_estimator *e) { return (size_t)e->slot_elems * 8; }
 
+int lane_ctas(const il_estimator *e)
+{
+    const int fit = e->ctas_lane[e->lane_slots == 16 ? 0 : 1];
+    return std::max(1, std::min(fit, e->lane_ctas_knob > 0 ? e->lane_ctas_knob : kLaneCtasPerSm));
+}
+
 int64_t full_slots(const il_estimator *e)
 {
-    return (int64_t)e->num_sms * e->ctas_per_sm * warps_per_cta(e);
+    return (int64_t)e->num_sms * (is_lane(e) ? lane_ctas(e) : e->ctas_per_sm) * warps_per_cta(e);
 }
 
 int64_t wanted_slots(const il_estimator *e, int64_t n_cand)
@@ -314,7 +324,7 @@ void configure_lane_rings(il_estimator *e)
 void free_device(il_estimator *e)
 {
     cudaFree(e->d_arrival); cudaFree(e->d_ptrace); cudaFree(e->d_bits); cudaFree(e->d_lat);
-    cudaFree(e->d_counters); cudaFree(e->d_status);
+    cudaFree(e->d_counters); cudaFree(e->d_status); cudaFree(e->d_maxrep);
     cudaFree(e->own_ws); cudaFree(e->d_cfg); cudaFree(e->d_out);
     if (e->h_counters) cudaFreeHost(e->h_counters);
     for (cudaEvent_t ev : e->events) cudaEventDestroy(ev);
@@ -413,7 +423,24 @@ static DesParams chunk_params(const il_estimator *e, const Plan &pl, char *ws, c
     p.order = reinterpret_cast<int32_t *>(ws + pl.off_order);
     p.ovf = reinterpret_cast<uint8_t *>(ws + pl.off_ovf);
     p.iter_limit = e->iter_limit;
+    p.lane_slots = e->lane_slots;
     return p;
+}
+
+// Batch ring positions per lane for this batch: 16 when no candidate has more than 14 replicas at any
+// stage (the ring must hold the slots in use and the batches waiting to be handed on), else 32.  One
+// small reduction over the configurations and a 4-byte read-back.
+static int choose_lane_slots(il_estimator *e, const il_stage_config *d_configs, int64_t n_cand)
+{
+    e->lane_slots = 32;
+    if (!is_lane(e)) return IL_OK;
+    int h = 0;
+    IL_CUDA(cudaMemsetAsync(e->d_maxrep, 0, sizeof(int), e->stream));
+    IL_CUDA(launch_max_replicas(d_configs, n_cand * e->S, e->d_maxrep, e->stream));
+    IL_CUDA(cudaMemcpyAsync(&h, e->d_maxrep, sizeof(int), cudaMemcpyDeviceToHost, e->stream));
+    IL_CUDA(cudaStreamSynchronize(e->stream));
+    e->lane_slots = h <= 14 ? 16 : 32;
+    return IL_OK;
 }
 
 // Enqueues the simulation of one chunk whose work counter is zero: the kernel the handle uses
@@ -425,7 +452,7 @@ static int enqueue_simulation(il_estimator *e, const DesParams &p, const Plan &p
     const int kernel = sim_kernel(e);
     const bool fb = kernel == kSimLane && e->lane_wrap;
     if (fb) IL_CUDA(cudaMemsetAsync(p.ovf, 0, (size_t)p.n_cand, st));
-    IL_CUDA(launch_simulation(p, kernel, (int)ctas, kernel == kSimLane ? e->smem_lane : e->smem, st));
+    IL_CUDA(launch_simulation(p, kernel, (int)ctas, kernel == kSimLane ? e->smem_lane[e->lane_slots == 16 ? 0 : 1] : e->smem, st));
     (*launches)++;
     if (fb) {
         IL_CUDA(launch_overflow_list(p.ovf, p.n_cand, const_cast<int32_t *>(p.order), e->d_counters, st));
@@ -742,6 +769,7 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     IL_CUDA_E(cudaMalloc(&e->d_lat, e->smem));
     IL_CUDA_E(cudaMalloc(&e->d_counters, kCounters * sizeof(unsigned long long)));
     IL_CUDA_E(cudaMalloc(&e->d_status, sizeof(int)));
+    IL_CUDA_E(cudaMalloc(&e->d_maxrep, sizeof(int)));
     IL_CUDA_E(cudaMallocHost(&e->h_counters, (kCounters + 2) * sizeof(unsigned long long)));
     e->h_status = reinterpret_cast<int *>(e->h_counters + kCounters);
     IL_CUDA_E(cudaMemcpy(e->d_arrival, tr->arrival_us, (size_t)n * 8, cudaMemcpyHostToDevice));
@@ -755,8 +783,11 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     e->ctas_per_sm_wide = des_max_ctas_per_sm(e->smem);
     e->ctas_per_sm_packed = des_packed_max_ctas_per_sm(false, e->smem);
     e->ctas_per_sm_staged = des_packed_max_ctas_per_sm(true, e->smem);
-    e->smem_lane = des_lane_smem(S * H * B);
-    e->ctas_per_sm_lane = std::min(des_lane_max_ctas_per_sm(e->smem_lane), kLaneCtasPerSm);
+    for (int k = 0; k < 2; k++) {
+        e->smem_lane[k] = des_lane_smem(S * H * B, B, k == 0 ? 16 : 32);
+        e->ctas_lane[k] = des_lane_max_ctas_per_sm(e->smem_lane[k]);
+    }
+    e->ctas_per_sm_lane = std::min(e->ctas_lane[1], kLaneCtasPerSm);
     if (e->ctas_per_sm_wide < 1 || e->ctas_per_sm_packed < 1 || e->ctas_per_sm_staged < 1 ||
         e->ctas_per_sm_lane < 1) {
         g_last_cuda_error = (int)cudaErrorLaunchOutOfResources;
@@ -805,6 +836,11 @@ int il_set_test_knob(il_estimator *e, int knob, int64_t value)
     if (knob == IL_KNOB_SHARE_PREFIXES) {
         if (value < 0 || value > 2) return IL_ERR_INVALID_ARG;
         e->share_mode = (int)value;
+        return IL_OK;
+    }
+    if (knob == IL_KNOB_LANE_CTAS) {
+        if (value < 0 || value > 16) return IL_ERR_INVALID_ARG;
+        e->lane_ctas_knob = (int)value;
         return IL_OK;
     }
     if (knob == IL_KNOB_ITER_LIMIT) {
@@ -874,6 +910,8 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
     if (!d_configs || !d_out_p99 || !d_out_miss) return IL_ERR_INVALID_ARG;
     IL_CUDA(cudaSetDevice(e->device));
 
+    int lrc = choose_lane_slots(e, d_configs, n_cand);
+    if (lrc) return lrc;
     char *ws = nullptr;
     size_t ws_bytes = 0;
     int wrc = acquire_workspace(e, n_cand, &ws, &ws_bytes);
@@ -965,6 +1003,7 @@ int il_estimate_latencies(il_estimator *e, const il_stage_config *d_config, int6
 {
     if (!e || !d_config || !d_out_latency) return IL_ERR_INVALID_ARG;
     IL_CUDA(cudaSetDevice(e->device));
+    e->lane_slots = 32;
     char *ws = nullptr;
     size_t ws_bytes = 0;
     int rc = acquire_workspace(e, 1, &ws, &ws_bytes);
@@ -1062,9 +1101,11 @@ int il_feasible_device(il_estimator *e, const il_stage_config *d_configs, int64_
     }
 
     // lane kernel: no slab and no percentile pass, so the whole batch is one chunk
+    int rc = choose_lane_slots(e, d_configs, n_cand);
+    if (rc) return rc;
     char *ws = nullptr;
     size_t ws_bytes = 0;
-    int rc = acquire_workspace(e, std::min<int64_t>(n_cand, 4096), &ws, &ws_bytes);
+    rc = acquire_workspace(e, std::min<int64_t>(n_cand, 4096), &ws, &ws_bytes);
     if (rc) return rc;
     if (e->share_mode == 1 || (e->share_mode == 0 && n_cand >= kShareMinCandidates)) {
         // a batch full of common configuration prefixes is cheaper to evaluate node by node
@@ -1108,7 +1149,7 @@ int il_feasible_device(il_estimator *e, const il_stage_config *d_configs, int64_
     const int64_t groups = (n_cand + e->cpw - 1) / e->cpw;
     const int64_t ctas = std::min<int64_t>(slots / wpc, (groups + wpc - 1) / wpc);
     IL_CUDA(cudaEventRecord(e->events[0], st));
-    IL_CUDA(launch_des_lane(p, (int)ctas, e->smem_lane, st));
+    IL_CUDA(launch_des_lane(p, (int)ctas, e->smem_lane[e->lane_slots == 16 ? 0 : 1], st));
     IL_CUDA(cudaEventRecord(e->events[1], st));
     int64_t launches = 1;
     if (e->lane_wrap) {

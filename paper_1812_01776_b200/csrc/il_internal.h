@@ -53,6 +53,8 @@ struct DesParams {
     int64_t lane_elems;           // stream records per candidate: every stage's arrival stream but the root's
     int32_t lane_off[IL_MAX_STAGES]; // record offset of stage s's arrival stream inside a candidate's block
     int32_t cpw;                  // candidates per warp, floor(32 / S)
+    int32_t lane_slots;           // positions of a lane's batch ring in shared memory: 16 or 32, at least the
+                                  // largest replica count among the launch's candidates
     int32_t lane_ring_log2;       // a stream ring holds 2^this records
     int32_t lane_wrap;            // the rings are shorter than the longest stream: positions wrap
     uint8_t *ovf;                 // [n_cand] set to 1 for a candidate given up on ring overflow (lane_wrap only)
@@ -111,7 +113,7 @@ int trace_tile_records();     // the packed trace is padded to a multiple of thi
 // lane-parallel kernel: one lane per (candidate, stage); smem from des_lane_smem
 cudaError_t launch_des_lane(const DesParams &p, int grid, size_t smem, cudaStream_t stream);
 int des_lane_warps_per_cta();
-size_t des_lane_smem(int n_tab);
+size_t des_lane_smem(int n_tab, int Bmax, int ring_slots);   // ring_slots: 16 or 32 batch ring positions per lane
 int des_lane_max_ctas_per_sm(size_t smem);
 enum SimKernel { kSimWide = 0, kSimPacked = 1, kSimPackedStaged = 2, kSimLane = 3 };
 inline cudaError_t launch_simulation(const DesParams &p, int kernel, int grid, size_t smem,
@@ -192,6 +194,7 @@ struct OrderParams {
     int32_t *order;                  // [n_cand] out
 };
 cudaError_t launch_order(const OrderParams &p, cudaStream_t stream);
+cudaError_t launch_max_replicas(const il_stage_config *configs, int64_t count, int *out, cudaStream_t stream);
 cudaError_t launch_gather_configs(const il_stage_config *configs, const int32_t *list, int64_t count, int S,
                                   il_stage_config *out, cudaStream_t stream);
 cudaError_t launch_feasible_from_p99(const int64_t *p99, const int32_t *list, int64_t count, int64_t slo_us,

@@ -84,6 +84,17 @@ __global__ void __launch_bounds__(1024) overflow_list_kernel(const uint8_t *ovf,
     }
 }
 
+// largest replica count over `count` stage configurations (values above the limit count as the limit:
+// the simulation kernel rejects them)
+__global__ void __launch_bounds__(256) max_replicas_kernel(const il_stage_config *configs, int64_t count, int *out)
+{
+    int m = 0;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
+        m = max(m, min((int)configs[i].replicas, IL_MAX_REPLICAS));
+    m = __reduce_max_sync(0xffffffffu, m);
+    if ((threadIdx.x & 31) == 0 && m > 0) atomicMax(out, m);
+}
+
 // configs of the listed candidates, packed one after the other
 __global__ void gather_configs_kernel(const il_stage_config *configs, const int32_t *list, int64_t count, int S,
                                       il_stage_config *out)
@@ -101,6 +112,13 @@ __global__ void feasible_from_p99_kernel(const int64_t *p99, const int32_t *list
 }
 
 }  // namespace
+
+cudaError_t launch_max_replicas(const il_stage_config *configs, int64_t count, int *out, cudaStream_t stream)
+{
+    const int grid = (int)std::min<int64_t>((count + 255) / 256, 1184);
+    max_replicas_kernel<<<grid, 256, 0, stream>>>(configs, count, out);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_gather_configs(const il_stage_config *configs, const int32_t *list, int64_t count, int S,
                                   il_stage_config *out, cudaStream_t stream)

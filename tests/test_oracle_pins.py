@@ -202,6 +202,7 @@ def tick_simulate(w, cfg):
     running = [dict() for _ in range(S)]     # replica -> (finish, order, [ids])
     order = 0
     lat = [None] * n
+    copies = [1] * n
     nxt = 0
     t = int(w.arrival_us[0])
     left = n
@@ -212,9 +213,10 @@ def tick_simulate(w, cfg):
             for q in ids:
                 c = [c for c in kids[s] if w.cond_bit[c] < 0
                      or ((int(w.branch_bits[q]) >> int(w.cond_bit[c])) & 1) == int(w.cond_val[c])]
-                if c:
-                    queue[c[0]].append(q)
-                else:
+                for child in c:                       # every edge whose condition holds
+                    queue[child].append(q)
+                copies[q] += len(c) - 1
+                if copies[q] == 0:                    # the last copy of the query has left
                     lat[q] = t - int(w.arrival_us[q])
                     left -= 1
         while nxt < n and int(w.arrival_us[nxt]) == t:
@@ -460,10 +462,10 @@ def test_rejects_bad_inputs(oracle):
     assert code() == 0
     bad = w.parent.copy(); bad[2] = 2
     assert code(parent=bad) == -2
-    bad = w.cond_bit.copy(); bad[3] = 1                     # siblings guarded by different bits
+    bad = w.parent.copy(); bad[2] = 0                       # three children of one stage
+    assert code(parent=bad) == -2
+    bad = w.cond_bit.copy(); bad[3] = 9                     # no such branch bit
     assert code(cond_bit=bad) == -2
-    bad = w.cond_val.copy(); bad[3] = 0                     # siblings with the same value
-    assert code(cond_val=bad) == -2
     bad = w.latency_us.copy(); bad[1, 1, 5] = 0
     assert code(latency_us=bad) == -3
     bad = w.arrival_us.copy(); bad[10] = bad[9] - 1
@@ -491,3 +493,68 @@ def test_grouped_arrivals_give_the_constructed_latency_multiset(oracle):
             w.slo_us = slo
             p99, miss = oracle.estimate_workload(w)
             assert (int(p99[0]), int(miss[0])) == (int(srt[k - 1]), int((want > slo).sum())), (case, slo)
+
+
+# --------------------------------------------------------------------------
+# fan-out: a query follows every edge whose condition holds and is answered
+# when its last copy leaves
+# --------------------------------------------------------------------------
+
+def fan_out_workload(seed, n=60, tiny=False):
+    """0 -> {1, 2}; 1 -> 3; 2 -> {4 (bit 0 = 1), 5 (always)}: an unconditional fork at the root, a chain
+    on one branch, and on the other a second fork one of whose edges is conditional."""
+    w = workloads.random_small(seed, S=6, H=2, Bmax=4, n=n, C=8, max_replicas=3, tree=False,
+                               qps=80_000.0 if tiny else 300.0, cv=2.0, lat_lo=1, lat_hi=30 if tiny else 9000,
+                               equal_stamp_every=(3 if seed % 2 == 0 else 0))
+    w.parent = np.array([-1, 0, 0, 1, 2, 2], np.int32)
+    w.cond_bit = np.array([-1, -1, -1, -1, 0, -1], np.int8)
+    w.cond_val = np.array([0, 0, 0, 0, 1, 0], np.uint8)
+    w.branch_bits = np.random.default_rng(seed).integers(0, 4, n).astype(np.uint8)
+    return w
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_fan_out_tick_brute_force(oracle, seed):
+    w = fan_out_workload(seed, n=40, tiny=True)
+    for c in range(w.n_candidates):
+        exp = tick_simulate(w, w.configs[c])
+        _, _, lat = oracle.estimate_one(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us,
+                                        w.branch_bits, w.configs[c], 40, want_latency=True)
+        assert np.array_equal(lat, exp), (seed, c)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_fan_out_is_the_maximum_over_its_branches(oracle, seed):
+    """Branches do not interact (each queue is fed by one parent), so a pipeline 0 -> {1 -> 3, 2} gives
+    every query the larger of its latencies in the two chains 0 -> 1 -> 3 and 0 -> 2 taken alone --
+    and those are linear pipelines, pinned above by the tandem and Kiefer-Wolfowitz recursions."""
+    w = workloads.random_small(50 + seed, S=4, H=2, Bmax=8, n=400, C=6, max_replicas=4, qps=300.0, cv=3.0,
+                               lat_lo=100, lat_hi=9000, equal_stamp_every=(4 if seed % 2 else 0))
+    w.parent = np.array([-1, 0, 0, 1], np.int32)
+    for c in range(w.n_candidates):
+        cfg = w.configs[c]
+        _, _, both = oracle.estimate_one(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us,
+                                         w.branch_bits, cfg, 0, want_latency=True)
+        lin = np.array([-1, 0, 1], np.int32)
+        none3, zero3 = np.full(3, -1, np.int8), np.zeros(3, np.uint8)
+        _, _, a = oracle.estimate_one(lin, none3, zero3, w.latency_us[[0, 1, 3]], w.arrival_us, None,
+                                      cfg[[0, 1, 3]], 0, want_latency=True)
+        _, _, b = oracle.estimate_one(lin[:2], none3[:2], zero3[:2], w.latency_us[[0, 2]], w.arrival_us, None,
+                                      cfg[[0, 2]], 0, want_latency=True)
+        assert np.array_equal(both, np.maximum(a, b)), (seed, c)
+
+
+def test_fan_out_never_queue_limit_is_the_longest_path(oracle):
+    """Section 4.3: the service time is the sum of the batch-1 latencies along the LONGEST path.  With
+    replicas to spare and spaced arrivals nothing queues, so every query's latency is exactly that."""
+    w = fan_out_workload(3, n=50)
+    w.arrival_us = np.arange(50, dtype=np.int64) * 200_000
+    cfg = np.array([[1, 4, 3, 0]] * 6, np.uint8)
+    d = w.latency_us[:, 1, 0].astype(np.int64)
+    _, _, lat = oracle.estimate_one(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us,
+                                    w.branch_bits, cfg, 0, want_latency=True)
+    for q in range(50):
+        paths = [d[0] + d[1] + d[3], d[0] + d[2] + d[5]]
+        if w.branch_bits[q] & 1:
+            paths.append(d[0] + d[2] + d[4])
+        assert lat[q] == max(paths)
