@@ -87,6 +87,10 @@ des_kernel(const __grid_constant__ DesParams p)
         }
 
         int64_t *slab = p.slab + c * p.slab_stride;
+        if (p.fork) {       // per-query maxima start from zero
+            for (int i = lane; i < p.n; i += 32) slab[i] = 0;
+            __syncwarp();
+        }
         int32_t exits = 0;
         uint64_t lat_or = 0;
         unsigned long long cand_batches = 0;
@@ -120,6 +124,39 @@ des_kernel(const __grid_constant__ DesParams p)
                     const bool act = j < b;
                     int32_t q = 0;
                     if (act) q = (s == 0) ? start + j : in_q[start + j];
+                    if (p.fork) {
+                        // fan-out: every edge whose condition holds; a copy that finds none leaves, and
+                        // the slab keeps the largest latency of the query's copies (the stages of a
+                        // candidate run one after the other on this warp, so a plain maximum will do)
+                        const int ca = p.child_a[s], cb = p.child_b[s];
+                        unsigned bits = 0;
+                        if (act && (p.cbit_a[s] >= 0 || p.cbit_b[s] >= 0) && IL_IN_RANGE(q, p.n, p.status)) bits = p.bits[q];
+                        const bool go_a = act && ca >= 0 && (p.cbit_a[s] < 0 || ((bits >> p.cbit_a[s]) & 1u) == p.cval_a[s]);
+                        const bool go_b = act && cb >= 0 && (p.cbit_b[s] < 0 || ((bits >> p.cbit_b[s]) & 1u) == p.cval_b[s]);
+                        const bool left = act && !go_a && !go_b;
+                        const unsigned fa = __ballot_sync(full, go_a), fb = __ballot_sync(full, go_b);
+                        const unsigned fl = __ballot_sync(full, left);
+                        if (go_a) {
+                            const int at = rt.a_tail + __popc(fa & lt_mask);
+                            if (IL_IN_RANGE(p.buf_off[ca] + at, p.slot_elems, p.status)) {
+                                (my_time + p.buf_off[ca])[at] = tfin; (my_qid + p.buf_off[ca])[at] = q;
+                            }
+                        }
+                        if (go_b) {
+                            const int at = rt.b_tail + __popc(fb & lt_mask);
+                            if (IL_IN_RANGE(p.buf_off[cb] + at, p.slot_elems, p.status)) {
+                                (my_time + p.buf_off[cb])[at] = tfin; (my_qid + p.buf_off[cb])[at] = q;
+                            }
+                        }
+                        if (left && IL_IN_RANGE(q, p.n, p.status)) {
+                            const int64_t l = tfin - p.arrival[q];
+                            if (l > slab[q]) slab[q] = l;
+                            lat_or |= (uint64_t)l;
+                        }
+                        rt.a_tail += __popc(fa); rt.b_tail += __popc(fb);
+                        exits += __popc(fl);
+                        continue;
+                    }
                     bool bitv = false;
                     if (act && rt.bit >= 0 && IL_IN_RANGE(q, p.n, p.status)) bitv = (p.bits[q] >> rt.bit) & 1;
                     const unsigned ma = __ballot_sync(full, act && !bitv);
@@ -233,7 +270,7 @@ des_kernel(const __grid_constant__ DesParams p)
         const uint32_t hi = __reduce_or_sync(full, (uint32_t)(lat_or >> 32));
         if (lane == 0) {
             p.lat_or[c] = ((uint64_t)hi << 32) | lo;
-            if (!over && exits != p.n) atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT);
+            if (!over && (int64_t)exits != (p.fork ? p.total_leaving : (int64_t)p.n)) atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT);
         }
     }
     if (lane == 0 && batches) { atomicAdd(&p.counters[1], batches); atomicAdd(&p.counters[2], alg_ops); }

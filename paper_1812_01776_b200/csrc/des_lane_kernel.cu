@@ -162,7 +162,10 @@ __device__ __forceinline__ WarpMem warp_mem_at(unsigned char *base, int kr, int 
 // FEAS: feasibility only (Section 4.3, "Feasible"): leaving queries are compared with the objective as
 //       they leave, nothing is written to a slab, and a candidate is dropped as soon as more queries
 //       have missed the objective than the P99 rule allows.
-template <bool BRANCHY, bool RING, bool FEAS>
+// FORK: fan-out -- a query goes down every edge whose condition holds, a copy that finds none leaves, and
+//       the slab keeps per query the record of the copy that left last (only with BRANCHY, without RING
+//       and FEAS).
+template <bool BRANCHY, bool RING, bool FEAS, bool FORK = false>
 __global__ void __launch_bounds__(kLaneWarps * 32)
 des_lane_kernel(const __grid_constant__ DesParams p)
 {
@@ -179,7 +182,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
     const unsigned full = 0xffffffffu;
     const int wid = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const uint32_t kr = (uint32_t)p.lane_slots, rmask = kr - 1u;      // batch ring positions of a lane
+    const uint32_t kr = p.lane_slots == 16 ? 16u : 32u, rmask = kr - 1u;      // batch ring positions of a lane
     const WarpMem wm = warp_mem_at(wm_base + (size_t)wid * warp_mem_bytes((int)kr, p.Bmax), (int)kr, p.Bmax);
     const int S = p.S, cpw = p.cpw;
     const int j = lane / S, s = lane - j * S;
@@ -194,8 +197,11 @@ des_lane_kernel(const __grid_constant__ DesParams p)
         if (b2 >= 0 && b2 != a) kids += p.n_s[b2];
         exit_off += p.n_s[u] - kids;
     }
-    const int da = p.dest_a[s], db = p.dest_b[s];
-    const int bit = p.bit[s];
+    const int da = FORK ? p.child_a[s] : p.dest_a[s], db = FORK ? p.child_b[s] : p.dest_b[s];
+    // fan-out: the guard of either edge; the branch bits are needed if one of them is conditional
+    const int cbit_a = p.cbit_a[s], cbit_b = p.cbit_b[s];
+    const unsigned cval_a = p.cval_a[s], cval_b = p.cval_b[s];
+    const int bit = FORK ? ((cbit_a >= 0 || cbit_b >= 0) ? 0 : -1) : p.bit[s];
     const uint32_t n_in = lane_used ? (uint32_t)p.n_s[s] : 0u;
     const unsigned group_mask = lane_used ? (((1u << S) - 1u) << (j * S)) : 0u;
     const int root_lane = lane_used ? j * S : 0;
@@ -236,6 +242,8 @@ des_lane_kernel(const __grid_constant__ DesParams p)
     uint32_t R = 1;
     int mb = 1;
     uint64_t *out_a = nullptr, *out_b = nullptr;
+    unsigned long long *slab_row = nullptr;   // fan-out: the candidate's slab row, indexed by query
+    uint32_t n_left = 0;                      // fan-out: copies that left the pipeline at this lane
     uint32_t epos = 0, lpos = 0, tpos = 0;   // ring positions, see WarpMem
     uint64_t kfront = kInf;      // key at lpos (kInf when no slot is in use)
     uint64_t ktail = 0;          // largest key in [lpos, tpos)
@@ -329,8 +337,9 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                     // every query of a candidate that ran to its end must have left through exactly one
                     // leaf (checked over all candidates of the warp when the kernel ends)
                     if (live && !cand_aborted && !decided)
-                        exits_seen += (da < 0 ? tail_a : 0u) + ((db < 0 && bit >= 0) ? tail_b : 0u);
-                    if (s == 0 && !cand_bad && !cand_aborted && !decided) exits_due += (unsigned)p.n;
+                        exits_seen += FORK ? n_left : (da < 0 ? tail_a : 0u) + ((db < 0 && bit >= 0) ? tail_b : 0u);
+                    if (s == 0 && !cand_bad && !cand_aborted && !decided)
+                        exits_due += FORK ? (unsigned long long)p.total_leaving : (unsigned long long)(unsigned)p.n;
                     if (FEAS && s == 0) {
                         p.out_feasible[c] = cand_aborted ? 2 : (decided || cand_bad ? 0 : 1);
                         early += (decided && head < n_in) ? 1u : 0u;     // the root had not reached the end of the trace
@@ -365,6 +374,8 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                     }
                     out_a = da < 0 ? slab + exit_off : my_block + p.lane_off[da];
                     out_b = db < 0 ? slab + exit_off : my_block + p.lane_off[db];
+                    slab_row = reinterpret_cast<unsigned long long *>(slab);
+                    n_left = 0;
                     // the root's stream is complete from the start; a stage nobody visits is finished at once
                     const uint32_t avail0 = (s == 0 || !live) ? (n_in | kDone) : 0u;
                     wm.avail[0][lane] = avail0; wm.avail[1][lane] = avail0;
@@ -475,7 +486,20 @@ des_lane_kernel(const __grid_constant__ DesParams p)
             if (end && b == 0) lpos = tpos;     // stream exhausted: everything still held leaves, in key order
 
             // ---- hand on the record picked up at the top of the iteration
-            if (BRANCHY) {
+            if (FORK) {
+                const uint64_t out = h_base | h_qid;
+                const bool go_a = da >= 0 && (cbit_a < 0 || ((h_bits >> cbit_a) & 1u) == cval_a);
+                const bool go_b = db >= 0 && (cbit_b < 0 || ((h_bits >> cbit_b) & 1u) == cval_b);
+                if (h_valid) {
+                    if (go_a && IL_IN_RANGE(tail_a, size_a, p.status)) out_a[tail_a] = out;
+                    if (go_b && IL_IN_RANGE(tail_b, size_b, p.status)) out_b[tail_b] = out;
+                    // this copy leaves: the query's slab entry keeps the latest of its copies
+                    if (!go_a && !go_b && IL_IN_RANGE(h_qid, p.n, p.status)) atomicMax(slab_row + h_qid, out);
+                }
+                tail_a += (h_valid && go_a) ? 1u : 0u;
+                tail_b += (h_valid && go_b) ? 1u : 0u;
+                n_left += (h_valid && !go_a && !go_b) ? 1u : 0u;
+            } else if (BRANCHY) {
                 // under predicates: with lanes on both sides of a branch point in one warp this measured
                 // 10 % faster than a branch around the block; without routing the branch is the faster form
                 const uint64_t out = h_base | h_qid;
@@ -571,27 +595,32 @@ bool any_branch(const DesParams &p)
 }  // namespace
 
 namespace {
-template <bool BRANCHY, bool RING, bool FEAS>
+template <bool BRANCHY, bool RING, bool FEAS, bool FORK>
 cudaError_t launch_one(const DesParams &p, int grid, size_t smem, cudaStream_t stream)
 {
-    cudaError_t e = cudaFuncSetAttribute(des_lane_kernel<BRANCHY, RING, FEAS>,
+    cudaError_t e = cudaFuncSetAttribute(des_lane_kernel<BRANCHY, RING, FEAS, FORK>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    des_lane_kernel<BRANCHY, RING, FEAS><<<grid, kLaneWarps * 32, smem, stream>>>(p);
+    des_lane_kernel<BRANCHY, RING, FEAS, FORK><<<grid, kLaneWarps * 32, smem, stream>>>(p);
     return cudaGetLastError();
 }
 
 template <bool BRANCHY, bool RING>
 cudaError_t launch_two(const DesParams &p, int grid, size_t smem, cudaStream_t stream)
 {
-    return p.out_feasible ? launch_one<BRANCHY, RING, true>(p, grid, smem, stream)
-                          : launch_one<BRANCHY, RING, false>(p, grid, smem, stream);
+    return p.out_feasible ? launch_one<BRANCHY, RING, true, false>(p, grid, smem, stream)
+                          : launch_one<BRANCHY, RING, false, false>(p, grid, smem, stream);
 }
 }  // namespace
 
-// Feasibility-only when p.out_feasible is set.
+// Feasibility-only when p.out_feasible is set; the fan-out instantiation when p.fork is (the host
+// never combines that with stream rings or feasibility-only).
 cudaError_t launch_des_lane(const DesParams &p, int grid, size_t smem, cudaStream_t stream)
 {
+    if (p.fork) {
+        if (p.lane_wrap || p.out_feasible) return cudaErrorInvalidValue;
+        return launch_one<true, false, false, true>(p, grid, smem, stream);
+    }
     const bool br = any_branch(p);
     if (p.lane_wrap) return br ? launch_two<true, true>(p, grid, smem, stream) : launch_two<false, true>(p, grid, smem, stream);
     return br ? launch_two<true, false>(p, grid, smem, stream) : launch_two<false, false>(p, grid, smem, stream);

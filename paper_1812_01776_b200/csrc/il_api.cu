@@ -42,6 +42,7 @@ struct il_estimator {
     int64_t *d_arrival = nullptr;
     uint64_t *d_ptrace = nullptr;      // packed root stream
     bool can_pack = false;             // every reachable time fits a packed record
+    bool fork = false;                 // fan-out: one query can enter two children of a stage
     bool lane_ok = false;              // the lane kernel applies (packed records, stream offsets fit 31 bits)
     int variant = IL_VARIANT_AUTO;
     int ctas_per_sm_wide = 0, ctas_per_sm_packed = 0, ctas_per_sm_staged = 0, ctas_per_sm_lane = 0;
@@ -96,11 +97,12 @@ struct Plan {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// Resident CTAs (of two warps) per SM for the lane kernel.  Two warps per scheduler keep the issue
-// slots about as busy as more would, and every further warp lengthens all chains through the
-// shared-memory pipe: on B200, workload 2 with 16,384 candidates took 101.7 / 79.2 / 68.4 / 71.1 / 85.5 ms
-// with 2 / 3 / 4 / 5 / 7 CTAs per SM; the tree workloads did not care from 4 on.
-constexpr int kLaneCtasPerSm = 4;
+// Resident CTAs (of two warps) per SM for the lane kernel, as far as shared memory lets them fit (with
+// 32 batch ring positions and 64 table rows per lane only four do).  Beyond two warps per scheduler
+// the issue slots fill only slowly: on B200 with shared memory laid out per launch, 4 / 5 / 6 / 8 CTAs
+// gave 71.0 / 71.2 / 68.9 / 70.1 ms on workload 2 with 16,384 candidates and 1,182 / 1,063 / 1,065 /
+// 1,065 ms on workload 3 (65,536 candidates).
+constexpr int kLaneCtasPerSm = 6;
 
 bool use_packed(const il_estimator *e)
 {
@@ -110,6 +112,8 @@ bool use_packed(const il_estimator *e)
 int sim_kernel(const il_estimator *e)
 {
     if (!use_packed(e)) return kSimWide;
+    // fan-out is implemented by the lane kernel and by the kernel with separate streams
+    if (e->fork) return (e->variant == IL_VARIANT_AUTO || e->variant == IL_VARIANT_LANES) && e->lane_ok ? kSimLane : kSimWide;
     if (e->variant == IL_VARIANT_LANES && e->lane_ok) return kSimLane;
     if (e->variant == IL_VARIANT_AUTO && e->lane_ok) return kSimLane;
     return e->variant == IL_VARIANT_STAGED ? kSimPackedStaged : kSimPacked;
@@ -234,16 +238,29 @@ int check_topology(const il_profiles *pr)
         if (pr->cond_bit[s] >= 0 && pr->cond_val[s] > 1) return IL_ERR_BAD_TOPOLOGY;
     }
     for (int par = 0; par < S; par++) {
-        int kids[IL_MAX_STAGES], nk = 0;
-        for (int c = 1; c < S; c++) if (pr->parent[c] == par) kids[nk++] = c;
+        int nk = 0;
+        for (int c = 1; c < S; c++) if (pr->parent[c] == par) nk++;
         if (nk > 2) return IL_ERR_BAD_TOPOLOGY;
-        if (nk == 2) {
-            const int a = kids[0], b = kids[1];
-            if (pr->cond_bit[a] < 0 || pr->cond_bit[b] != pr->cond_bit[a]) return IL_ERR_BAD_TOPOLOGY;
-            if (pr->cond_val[a] == pr->cond_val[b]) return IL_ERR_BAD_TOPOLOGY;
-        }
     }
     return IL_OK;
+}
+
+// Two children of one stage are alternatives when they are guarded by the same bit with different
+// values; otherwise one query can enter both (fan-out).
+bool has_fan_out(const il_profiles *pr)
+{
+    const int S = pr->n_stages;
+    for (int par = 0; par < S; par++) {
+        int kids[2], nk = 0;
+        for (int c = 1; c < S; c++) if (pr->parent[c] == par && nk < 2) kids[nk++] = c;
+        if (nk == 2) {
+            const int a = kids[0], b = kids[1];
+            const bool alternatives = pr->cond_bit[a] >= 0 && pr->cond_bit[b] == pr->cond_bit[a] &&
+                                      pr->cond_val[a] != pr->cond_val[b];
+            if (!alternatives) return true;
+        }
+    }
+    return false;
 }
 
 // Lays the stages' input streams out inside one warp slot.  Stage c's stream is
@@ -299,8 +316,8 @@ void configure_lane_rings(il_estimator *e)
         exact += (e->visits[s] + 3) / 4 * 4;
     }
     const int64_t resident = (int64_t)e->num_sms * kLaneCtasPerSm * des_lane_warps_per_cta() * e->cpw;
-    const bool rings = e->lane_ring_cap_log2 > 0 || exact * 8 * resident > kLaneExactBytes ||
-                       exact >= (INT64_C(1) << 31);
+    const bool rings = !e->fork && (e->lane_ring_cap_log2 > 0 || exact * 8 * resident > kLaneExactBytes ||
+                                    exact >= (INT64_C(1) << 31));
     bp.lane_off[0] = 0;
     if (!rings) {
         int64_t off = 0;
@@ -347,7 +364,7 @@ void il::set_last_cuda_error(int cuda_error) { g_last_cuda_error = cuda_error; }
 void il::bound_view(const il_estimator *e, BoundView *out)
 {
     out->base = e->base;
-    out->kernel = sim_kernel(e) == kSimLane ? (int)kSimPacked : sim_kernel(e);   // its user has no lane layout
+    out->kernel = e->fork ? (int)kSimWide : sim_kernel(e) == kSimLane ? (int)kSimPacked : sim_kernel(e);   // its user has no lane layout
     out->S = e->S;
     out->n = e->n; out->n_pad = e->n_pad; out->slot_elems = e->slot_elems;
     out->smem = e->smem;
@@ -452,6 +469,9 @@ static int enqueue_simulation(il_estimator *e, const DesParams &p, const Plan &p
     const int kernel = sim_kernel(e);
     const bool fb = kernel == kSimLane && e->lane_wrap;
     if (fb) IL_CUDA(cudaMemsetAsync(p.ovf, 0, (size_t)p.n_cand, st));
+    // fan-out: the lane kernel keeps per query the largest leaving record, starting from zero
+    if (kernel == kSimLane && e->fork)
+        IL_CUDA(cudaMemsetAsync(p.slab, 0, (size_t)p.n_cand * p.slab_stride * 8, st));
     IL_CUDA(launch_simulation(p, kernel, (int)ctas, kernel == kSimLane ? e->smem_lane[e->lane_slots == 16 ? 0 : 1] : e->smem, st));
     (*launches)++;
     if (fb) {
@@ -500,7 +520,7 @@ static int estimate_shared(il_estimator *e, const il_stage_config *d_configs, in
     const int64_t n = e->n;
     const int64_t allowed = n - (99 * n + 99) / 100;           // T: queries allowed above the P99
     const int64_t top_len = allowed + 1;
-    if (e->share_mode == 2 || !e->can_pack || e->variant != IL_VARIANT_AUTO || top_len > kShareMaxTop ||
+    if (e->share_mode == 2 || e->fork || !e->can_pack || e->variant != IL_VARIANT_AUTO || top_len > kShareMaxTop ||
         n_cand >= (INT64_C(1) << 30) || (e->share_mode == 0 && n_cand < kShareMinCandidates))
         return IL_OK;
     uint32_t cap = 1024;
@@ -722,16 +742,31 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
         }
     }
     for (int s = 0; s < S; s++) e->parent[s] = pr->parent[s];
-    e->visits[0] = n;
-    for (int64_t q = 0; q < n; q++) {   // walk every query down its path
-        int s = 0;
-        for (;;) {
-            int nxt;
-            if (bp.bit[s] < 0) nxt = bp.dest_a[s];
-            else nxt = ((tr->branch_bits[q] >> bp.bit[s]) & 1) ? bp.dest_b[s] : bp.dest_a[s];
-            if (nxt < 0) break;
-            e->visits[nxt]++;
-            s = nxt;
+    e->fork = has_fan_out(pr);
+    bp.fork = e->fork ? 1 : 0;
+    for (int s = 0; s < IL_MAX_STAGES; s++) { bp.child_a[s] = -1; bp.child_b[s] = -1; bp.cbit_a[s] = -1; bp.cbit_b[s] = -1; }
+    for (int c = 1; c < S; c++) {
+        const int par = pr->parent[c];
+        if (bp.child_a[par] < 0) { bp.child_a[par] = (int8_t)c; bp.cbit_a[par] = pr->cond_bit[c]; bp.cval_a[par] = pr->cond_val[c]; }
+        else { bp.child_b[par] = (int8_t)c; bp.cbit_b[par] = pr->cond_bit[c]; bp.cval_b[par] = pr->cond_val[c]; }
+    }
+    // walk every query down every edge it takes
+    bp.total_leaving = 0;
+    for (int64_t q = 0; q < n; q++) {
+        int stack[IL_MAX_STAGES], top = 0;
+        stack[top++] = 0;
+        while (top > 0) {
+            const int s = stack[--top];
+            e->visits[s]++;
+            int taken = 0;
+            for (int side = 0; side < 2; side++) {
+                const int c = side == 0 ? bp.child_a[s] : bp.child_b[s];
+                if (c < 0) continue;
+                const int bit = side == 0 ? bp.cbit_a[s] : bp.cbit_b[s];
+                const int val = side == 0 ? bp.cval_a[s] : bp.cval_b[s];
+                if (bit < 0 || ((tr->branch_bits[q] >> bit) & 1) == val) { stack[top++] = c; taken++; }
+            }
+            if (taken == 0) bp.total_leaving++;
         }
     }
     e->events_per_candidate = 0;
@@ -754,7 +789,7 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     IL_CUDA_E(cudaMalloc(&e->d_arrival, (size_t)n * 8));
     IL_CUDA_E(cudaMalloc(&e->d_bits, (size_t)n));
     e->can_pack = can_pack;
-    e->lane_ok = can_pack;
+    e->lane_ok = can_pack && e->lane_elems < (INT64_C(1) << 31);   // (with fan-out the streams are kept whole)
     bp.qbits = qbits;
     if (can_pack) {
         // padded with "never" records to whole tiles, so that bulk copies always move full tiles
@@ -959,9 +994,9 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
         IL_CUDA(cudaEventRecord(e->events[3 + 3 * ch], st));
         SelectParams sp = {};
         sp.slab = p.slab; sp.slab_stride = e->n_pad; sp.lat_or = p.lat_or;
-        sp.arrival = e->d_arrival; sp.qbits = p.qbits; sp.packed = use_packed(e) ? 1 : 0;
+        sp.arrival = e->d_arrival; sp.qbits = p.qbits; sp.packed = sim_kernel(e) != kSimWide ? 1 : 0;
         sp.status = e->d_status;
-        if (lane) {
+        if (lane && !e->fork) {
             slab_regions(e, sp);
             if (e->lane_wrap) sp.ovf = p.ovf;
         }
@@ -1088,8 +1123,9 @@ int il_feasible_device(il_estimator *e, const il_stage_config *d_configs, int64_
     IL_CUDA(cudaSetDevice(e->device));
     cudaStream_t st = e->stream;
 
-    if (!is_lane(e)) {
-        // the other kernels have no early exit: P99 as usual, then the comparison
+    if (!is_lane(e) || e->fork) {
+        // no early exit on the other kernels, nor with fan-out (a query is late if ANY of its copies
+        // is, so copies cannot be counted as they leave): P99 as usual, then the comparison
         int rc = ensure_staging(e, n_cand);
         if (rc) return rc;
         rc = il_estimate_device(e, d_configs, n_cand, slo_us, e->d_out, e->d_out + e->d_out_cap);
@@ -1140,6 +1176,7 @@ int il_feasible_device(il_estimator *e, const il_stage_config *d_configs, int64_
     p.lane_ws = reinterpret_cast<uint64_t *>(ws);
     p.ovf = reinterpret_cast<uint8_t *>(ws + off_ovf);
     p.iter_limit = e->iter_limit;
+    p.lane_slots = e->lane_slots;
     p.out_feasible = d_out_feasible;
     // latency > objective is tested on time fields shifted by qbits: keep the objective in that range
     // (latencies are at least 1 and every reachable time is below 2^(63 - qbits))

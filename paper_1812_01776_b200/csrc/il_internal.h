@@ -36,6 +36,15 @@ struct DesParams {
     int8_t  dest_a[IL_MAX_STAGES];   // next stage for branch bit 0 (or unconditional); -1 = leave
     int8_t  dest_b[IL_MAX_STAGES];   // next stage for branch bit 1; -1 = leave
     int8_t  bit[IL_MAX_STAGES];      // branch bit tested after stage s, -1 = none
+    // Fan-out (fork != 0): some stage has two children that one query can enter both, so the three
+    // arrays above do not describe the routing; these do.  A query goes down every edge whose
+    // condition holds; where none holds that copy of it leaves, and the slab keeps per query the
+    // record of the copy that left last.
+    int32_t fork;
+    int8_t  child_a[IL_MAX_STAGES], child_b[IL_MAX_STAGES];   // children of stage s, -1 = none
+    int8_t  cbit_a[IL_MAX_STAGES], cbit_b[IL_MAX_STAGES];     // branch bit guarding the edge, -1 = always taken
+    uint8_t cval_a[IL_MAX_STAGES], cval_b[IL_MAX_STAGES];     // the edge is taken iff the bit has this value
+    int64_t total_leaving;           // copies that leave the pipeline, all stages together (n without fan-out)
     // this launch
     const il_stage_config *configs;  // [n_cand][S], already offset to the chunk
     int64_t n_cand;

@@ -67,10 +67,10 @@ def test_create_rejects_bad_arguments_on_the_host(lib):
 
     bad = w.parent.copy(); bad[2] = 2
     assert code(parent=bad) == E.IL_ERR_BAD_TOPOLOGY
-    bad = w.cond_bit.copy(); bad[3] = 1
+    bad = w.parent.copy(); bad[2] = 0                       # three children of one stage
+    assert code(parent=bad) == E.IL_ERR_BAD_TOPOLOGY
+    bad = w.cond_bit.copy(); bad[3] = 9                     # no such branch bit
     assert code(cond_bit=bad) == E.IL_ERR_BAD_TOPOLOGY
-    bad = w.cond_val.copy(); bad[3] = 0
-    assert code(cond_val=bad) == E.IL_ERR_BAD_TOPOLOGY
     bad = w.latency_us.copy(); bad[1, 1, 5] = 0
     assert code(latency_us=bad) == E.IL_ERR_BAD_PROFILE
     bad = w.arrival_us.copy(); bad[10] = bad[9] - 1

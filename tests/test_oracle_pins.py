@@ -501,16 +501,7 @@ def test_grouped_arrivals_give_the_constructed_latency_multiset(oracle):
 # --------------------------------------------------------------------------
 
 def fan_out_workload(seed, n=60, tiny=False):
-    """0 -> {1, 2}; 1 -> 3; 2 -> {4 (bit 0 = 1), 5 (always)}: an unconditional fork at the root, a chain
-    on one branch, and on the other a second fork one of whose edges is conditional."""
-    w = workloads.random_small(seed, S=6, H=2, Bmax=4, n=n, C=8, max_replicas=3, tree=False,
-                               qps=80_000.0 if tiny else 300.0, cv=2.0, lat_lo=1, lat_hi=30 if tiny else 9000,
-                               equal_stamp_every=(3 if seed % 2 == 0 else 0))
-    w.parent = np.array([-1, 0, 0, 1, 2, 2], np.int32)
-    w.cond_bit = np.array([-1, -1, -1, -1, 0, -1], np.int8)
-    w.cond_val = np.array([0, 0, 0, 0, 1, 0], np.uint8)
-    w.branch_bits = np.random.default_rng(seed).integers(0, 4, n).astype(np.uint8)
-    return w
+    return workloads.fan_out_small(seed, n=n, C=8, max_replicas=3, Bmax=4, tiny_times=tiny)
 
 
 @pytest.mark.parametrize("seed", range(10))

@@ -311,6 +311,23 @@ def make(config_id: int, n_queries: Optional[int] = None,
                     slo_us=slo, recipe=recipe)
 
 
+def fan_out_small(seed: int, n: int = 900, C: int = 30, max_replicas: int = 4, Bmax: int = 8,
+                  tiny_times: bool = False) -> Workload:
+    """A small pipeline with fan-out (Section 2: parallel branches of a DAG): 0 -> {1, 2} both
+    unconditional; 1 -> 3; 2 -> {4 if bit 0 is 1, 5 always}.  Every query visits stages 0, 1, 2, 3, 5;
+    those with bit 0 set also stage 4."""
+    w = random_small(seed, S=6, H=2, Bmax=Bmax, n=n, C=C, max_replicas=max_replicas, tree=False,
+                     qps=80_000.0 if tiny_times else 300.0, cv=2.0, lat_lo=1,
+                     lat_hi=30 if tiny_times else 9000, equal_stamp_every=(3 if seed % 2 == 0 else 0))
+    w.parent = np.array([-1, 0, 0, 1, 2, 2], np.int32)
+    w.cond_bit = np.array([-1, -1, -1, -1, 0, -1], np.int8)
+    w.cond_val = np.array([0, 0, 0, 0, 1, 0], np.uint8)
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([BASE_SEED, 98, seed])))
+    w.branch_bits = rng.integers(0, 4, n).astype(np.uint8)
+    w.name = f"fanout{seed}"
+    return w
+
+
 def sub_batch(config_id: int, size: int, seed: int = 0, n_queries: Optional[int] = None):
     """A seeded sample of ``size`` distinct candidates of workload ``config_id``,
     drawn from its WHOLE candidate set (not a prefix of it), in increasing
