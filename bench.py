@@ -401,31 +401,39 @@ def measure(il, torch, w, dev, stream, flush, steps, warmup, e2e_steps, variant,
 
 
 def measure_feasibility(il, torch, dev, stream, flush):
-    """Feasibility-only mode against the full estimate: workload 2's 4,096 candidates (device-resident,
-    best of 3 each), and a Planner run on workload 2's trace whose questions are answered either way."""
+    """Feasibility-only mode against the full estimate on workload 2's shape (device-resident, best of 3
+    each): its 4,096 candidates (one wave of warps: a dropped candidate leaves its lanes idle) and
+    16,384 candidates of the same draw (dropped candidates make room for the next ones); and a Planner
+    run on workload 2's trace whose questions are answered either way."""
     from paper_1812_01776_b200.planner import Planner
+    out = {"workload": WORKLOADS[2], "batches": []}
+    for n_cand in (4096, 16384):
+        w = workloads.make(2, n_candidates=n_cand)
+        with il.Estimator.from_workload(w, device=dev.index) as est, torch.cuda.stream(stream):
+            est.reserve_workspace(w.n_candidates)
+            est.use_current_stream()
+            d_cfg = torch.from_numpy(w.configs).to(dev)
+            d_flag = torch.empty(w.n_candidates, dtype=torch.uint8, device=dev)
+
+            def timed(fn):
+                best = None
+                for _ in range(3):
+                    flush.fill_(1)
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record(stream); fn(); b.record(stream); b.synchronize()
+                    best = a.elapsed_time(b) if best is None else min(best, a.elapsed_time(b))
+                return best
+            full_ms = timed(lambda: est.estimate_device(d_cfg, w.slo_us))
+            feas_ms = timed(lambda: est.feasible_device(d_cfg, w.slo_us, d_flag))
+            st = est.stats()
+            out["batches"].append(dict(candidates=w.n_candidates, estimate_ms=full_ms, feasible_ms=feas_ms,
+                                       speedup=full_ms / feas_ms,
+                                       infeasible_fraction=1.0 - float(d_flag.float().mean().item()),
+                                       dropped_early=st["early_exits"]))
     w = workloads.make(2)
-    out = {"workload": WORKLOADS[2]}
     with il.Estimator.from_workload(w, device=dev.index) as est, torch.cuda.stream(stream):
         est.reserve_workspace(w.n_candidates)
         est.use_current_stream()
-        d_cfg = torch.from_numpy(w.configs).to(dev)
-        d_flag = torch.empty(w.n_candidates, dtype=torch.uint8, device=dev)
-
-        def timed(fn):
-            best = None
-            for _ in range(3):
-                flush.fill_(1)
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream); fn(); b.record(stream); b.synchronize()
-                best = a.elapsed_time(b) if best is None else min(best, a.elapsed_time(b))
-            return best
-        full_ms = timed(lambda: est.estimate_device(d_cfg, w.slo_us))
-        feas_ms = timed(lambda: est.feasible_device(d_cfg, w.slo_us, d_flag))
-        st = est.stats()
-        out.update(estimate_ms=full_ms, feasible_ms=feas_ms, speedup=full_ms / feas_ms,
-                   infeasible_fraction=1.0 - float(d_flag.float().mean().item()),
-                   dropped_early=st["early_exits"], candidates=w.n_candidates)
         prices = np.array([0.90, 0.35, 0.10])
         plans = {}
         for name, feas in (("estimate", None), ("feasible", lambda c: est.feasible(c, w.slo_us))):

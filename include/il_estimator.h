@@ -310,8 +310,13 @@ IL_API int il_set_stream(il_estimator *est, void *cuda_stream);
  *                       the given size; it stays the caller's and must outlive
  *                       its use.  NULL/0 returns to library-owned scratch.
  * Without il_set_workspace the library allocates its own scratch with
- * cudaMalloc on first use (at most il_workspace_bytes, less if the device is
- * short of memory) and keeps it until destroy.
+ * cudaMalloc inside the first estimate call that needs it: il_workspace_bytes
+ * for that call's candidate count, but never more than 80 % of the memory that
+ * is free on the device at that moment.  A later call that wants more makes the
+ * library synchronise the stream, free the buffer and allocate a larger one (by
+ * the same rule); it is kept until destroy.  Callers that share the device with
+ * other allocators should size and own the buffer themselves (il_set_workspace),
+ * or use il_estimate_device_static.
  */
 IL_API int il_workspace_bytes(const il_estimator *est, int64_t n_candidates, size_t *bytes);
 IL_API int il_workspace_min_bytes(const il_estimator *est, size_t *bytes);
