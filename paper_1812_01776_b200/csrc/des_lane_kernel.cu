@@ -601,6 +601,17 @@ cudaError_t launch_one(const DesParams &p, int grid, size_t smem, cudaStream_t s
     cudaError_t e = cudaFuncSetAttribute(des_lane_kernel<BRANCHY, RING, FEAS, FORK>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
+    // Shared memory and L1 share 256 KB per SM.  Every stream record reaches a lane through L1 (cp.async),
+    // 16 records per line, so the lines of all resident lanes must survive 16 iterations there: ask for
+    // no more shared memory than the resident CTAs use (1 KB per CTA is the system's), the rest is L1.
+    if (p.lane_ctas_per_sm > 0) {
+        const size_t need = (size_t)p.lane_ctas_per_sm * (smem + 1024);
+        int pct = (int)((need * 100 + 233472 - 1) / 233472);     // of the 228 KB an SM can give
+        pct = pct < 1 ? 1 : (pct > 100 ? 100 : pct);
+        e = cudaFuncSetAttribute(des_lane_kernel<BRANCHY, RING, FEAS, FORK>,
+                                 cudaFuncAttributePreferredSharedMemoryCarveout, pct);
+        if (e != cudaSuccess) return e;
+    }
     des_lane_kernel<BRANCHY, RING, FEAS, FORK><<<grid, kLaneWarps * 32, smem, stream>>>(p);
     return cudaGetLastError();
 }

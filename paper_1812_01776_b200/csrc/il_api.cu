@@ -97,12 +97,13 @@ struct Plan {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// Resident CTAs (of two warps) per SM for the lane kernel, as far as shared memory lets them fit (with
-// 32 batch ring positions and 64 table rows per lane only four do).  Beyond two warps per scheduler
-// the issue slots fill only slowly: on B200 with shared memory laid out per launch, 4 / 5 / 6 / 8 CTAs
-// gave 71.0 / 71.2 / 68.9 / 70.1 ms on workload 2 with 16,384 candidates and 1,182 / 1,063 / 1,065 /
-// 1,065 ms on workload 3 (65,536 candidates).
-constexpr int kLaneCtasPerSm = 6;
+// Resident CTAs (of two warps) per SM for the lane kernel.  Every stream record reaches its lane through
+// L1, and L1 is what the 256 KB of an SM have left after the shared-memory carve-out, which the launch
+// sets to what the resident CTAs use (des_lane_kernel.cu).  More CTAs mean more lanes sharing less L1:
+// on B200, 3 / 4 / 5 / 6 / 8 CTAs gave 42.8 / 39.3 / 43.0 / 46.8 / 70.4 ms on workload 2 with 16,384
+// candidates and 298 / 245 / 336 / 336 / 335 ms on workload 3 with 16,384.  (Left to the driver, the
+// carve-out was the largest one whatever the grid, and the same cases took 70 and 336 ms.)
+constexpr int kLaneCtasPerSm = 4;
 
 bool use_packed(const il_estimator *e)
 {
@@ -441,6 +442,7 @@ static DesParams chunk_params(const il_estimator *e, const Plan &pl, char *ws, c
     p.ovf = reinterpret_cast<uint8_t *>(ws + pl.off_ovf);
     p.iter_limit = e->iter_limit;
     p.lane_slots = e->lane_slots;
+    p.lane_ctas_per_sm = lane_ctas(e);
     return p;
 }
 
@@ -1177,6 +1179,7 @@ int il_feasible_device(il_estimator *e, const il_stage_config *d_configs, int64_
     p.ovf = reinterpret_cast<uint8_t *>(ws + off_ovf);
     p.iter_limit = e->iter_limit;
     p.lane_slots = e->lane_slots;
+    p.lane_ctas_per_sm = lane_ctas(e);
     p.out_feasible = d_out_feasible;
     // latency > objective is tested on time fields shifted by qbits: keep the objective in that range
     // (latencies are at least 1 and every reachable time is below 2^(63 - qbits))

@@ -64,6 +64,7 @@ struct DesParams {
     int32_t cpw;                  // candidates per warp, floor(32 / S)
     int32_t lane_slots;           // positions of a lane's batch ring in shared memory: 16 or 32, at least the
                                   // largest replica count among the launch's candidates
+    int32_t lane_ctas_per_sm;     // CTAs the host keeps resident per SM (sizes the shared-memory carve-out); 0: unknown
     int32_t lane_ring_log2;       // a stream ring holds 2^this records
     int32_t lane_wrap;            // the rings are shorter than the longest stream: positions wrap
     uint8_t *ovf;                 // [n_cand] set to 1 for a candidate given up on ring overflow (lane_wrap only)
