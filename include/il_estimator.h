@@ -129,7 +129,7 @@ typedef struct {
                                 (replica min, queue count, table add, slot update), per query-event 3 */
     int64_t chunks;          /* how many (simulate, select) launch groups the call made (the
                                 warp-per-candidate kernels add an ordering launch to each)  */
-    int64_t kernel_launches; /* kernels launched by the call                             */
+    int64_t kernel_launches; /* kernels of this library launched by the call             */
     double  sim_ms;          /* device time of the simulation kernels (CUDA events)      */
     double  select_ms;       /* device time of the percentile kernels (CUDA events)      */
     double  total_ms;        /* device time of all stream work of the call               */

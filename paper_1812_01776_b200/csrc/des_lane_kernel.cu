@@ -170,14 +170,11 @@ __global__ void __launch_bounds__(kLaneWarps * 32)
 des_lane_kernel(const __grid_constant__ DesParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    int32_t *s_lat = reinterpret_cast<int32_t *>(smem_raw);      // the profile tables, [S][H][Bmax]
-    const int n_tab = p.S * p.H * p.Bmax;
-    unsigned char *wm_base = smem_raw + ((size_t)n_tab * 4 + 15) / 16 * 16;
+    // (the profile tables stay in global memory: a lane copies its row from there once per candidate, and
+    // shared memory not spent on them is L1 for the stream records)
+    unsigned char *wm_base = smem_raw;
     const int q = p.qbits;
     const uint64_t qmask = (1ull << q) - 1ull;
-    for (int i = threadIdx.x; i < n_tab; i += blockDim.x)
-        s_lat[i] = p.lat[i];
-    __syncthreads();
 
     const unsigned full = 0xffffffffu;
     const int wid = threadIdx.x >> 5;
@@ -369,7 +366,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                     R = cfg.replicas;
                     mb = cfg.max_batch;
                     if (live) {
-                        const int32_t *row = s_lat + (s * p.H + cfg.hw) * p.Bmax;
+                        const int32_t *row = p.lat + (s * p.H + cfg.hw) * p.Bmax;
                         for (int k = 0; k < p.Bmax; k++) wm.lat[k][lane] = (uint32_t)row[k];
                     }
                     out_a = da < 0 ? slab + exit_off : my_block + p.lane_off[da];
@@ -639,9 +636,9 @@ cudaError_t launch_des_lane(const DesParams &p, int grid, size_t smem, cudaStrea
 
 int des_lane_warps_per_cta() { return kLaneWarps; }
 
-size_t des_lane_smem(int n_tab, int Bmax, int ring_slots)
+size_t des_lane_smem(int, int Bmax, int ring_slots)
 {
-    return ((size_t)n_tab * 4 + 15) / 16 * 16 + (size_t)kLaneWarps * warp_mem_bytes(ring_slots, Bmax);
+    return (size_t)kLaneWarps * warp_mem_bytes(ring_slots, Bmax);
 }
 
 int des_lane_max_ctas_per_sm(size_t smem)

@@ -57,6 +57,7 @@ struct il_estimator {
     size_t smem_lane[2] = {0, 0};       // lane kernel with 16 / 32 batch ring positions per lane
     int ctas_lane[2] = {0, 0};
     int lane_slots = 32;               // batch ring positions used by the current call
+    int64_t setup_launches = 0;        // kernels a call launched before its simulation: the replica reduction, the node probe
     int lane_ctas_knob = 0;            // test knob: resident CTAs per SM of the lane kernel (0: the library's choice)
     int *d_maxrep = nullptr;           // device word: largest replica count of a batch
     uint8_t *d_bits = nullptr;
@@ -447,12 +448,15 @@ static DesParams chunk_params(const il_estimator *e, const Plan &pl, char *ws, c
 }
 
 // Batch ring positions per lane for this batch: 16 when no candidate has more than 14 replicas at any
-// stage (the ring must hold the slots in use and the batches waiting to be handed on), else 32.  One
+// stage (the ring must hold the slots in use and the batches waiting to be handed on; with 16 replicas on
+// 16 positions a stage stalls until each batch has been handed on, and workload 4 ran 1.6x slower), else 32.  One
 // small reduction over the configurations and a 4-byte read-back.
 static int choose_lane_slots(il_estimator *e, const il_stage_config *d_configs, int64_t n_cand)
 {
     e->lane_slots = 32;
+    e->setup_launches = 0;
     if (!is_lane(e)) return IL_OK;
+    e->setup_launches = 1;
     int h = 0;
     IL_CUDA(cudaMemsetAsync(e->d_maxrep, 0, sizeof(int), e->stream));
     IL_CUDA(launch_max_replicas(d_configs, n_cand * e->S, e->d_maxrep, e->stream));
@@ -563,6 +567,7 @@ static int estimate_shared(il_estimator *e, const il_stage_config *d_configs, in
     if (*e->h_status) { *used = true; return *e->h_status; }       // an invalid candidate: the call fails here
     int64_t total_nodes = 0;
     for (int s = 0; s < S; s++) total_nodes += h_count[s];
+    e->setup_launches += 3 * S;
     if (e->share_mode == 0 && total_nodes * 4 > n_cand * S) return IL_OK;
 
     // streams between the nodes, leaving records, top lists and miss counts
@@ -587,7 +592,7 @@ static int estimate_shared(il_estimator *e, const il_stage_config *d_configs, in
     if (off > ws_bytes) return IL_OK;
     *used = true;
 
-    int64_t launches = 3 * S;
+    int64_t launches = e->setup_launches;
     for (int s = 0; s < S; s++) {
         if (e->visits[s] == 0) continue;
         const int a = e->base.dest_a[s], b = e->base.dest_b[s];
@@ -968,7 +973,7 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
     IL_CUDA(cudaMemsetAsync(e->d_status, 0, sizeof(int), st));
     IL_CUDA(cudaEventRecord(e->events[0], st));
 
-    int64_t launches = 0;
+    int64_t launches = e->setup_launches;
     for (int64_t ch = 0; ch < n_chunks; ch++) {
         const int64_t lo = ch * pl.chunk;
         const int64_t cnt = std::min(pl.chunk, n_cand - lo);
