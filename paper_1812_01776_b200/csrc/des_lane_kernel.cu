@@ -265,6 +265,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
     // feasibility only: a leaving record waits one iteration for the arrival time of its query
     uint64_t late_fin = 0, late_arr = 0;
     bool late_valid = false;
+    uint32_t miss_local = 0;     // misses seen by this lane since it last added them to the group's count
     uint32_t av = 0;             // mailbox word this iteration works with: the one read an iteration ago
     int par = 0;                 // mailbox buffer this iteration publishes into; it reads the other one
     uint32_t it = 0;
@@ -313,7 +314,11 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                     done = true;
                 }
             }
-            if (FEAS && has && !done && wm.miss[j] > p.miss_allow) done = true;   // same word, same moment: the whole group
+            if (FEAS) {
+                if (miss_local) { atomicAdd(&wm.miss[j], miss_local); miss_local = 0; }
+                __syncwarp();
+                if (has && !done && wm.miss[j] > p.miss_allow) done = true;   // same word, same moment: the whole group
+            }
             // Feasibility only: a group moves on as soon as its own lanes have finished (candidates are
             // dropped at very different points of the trace).  Otherwise the groups of a warp start their
             // candidates together: they then walk the trace side by side and share its cache lines.
@@ -395,6 +400,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                     low_pub = 0; low_new = 0; e_first = 0;
                     low_pending = false; aborted = false;
                     late_valid = false;
+                    miss_local = 0;
                     av = avail0;
                 }
                 __syncwarp();     // the mailboxes are set before anybody reads them
@@ -414,11 +420,14 @@ des_lane_kernel(const __grid_constant__ DesParams p)
             // feasibility only: the record that left in the previous iteration is tested now, its query's
             // arrival record having had an iteration to come in; the arrival record of a query that may
             // leave in this iteration is requested here
-            if (FEAS && late_valid && late_fin > (late_arr & ~qmask) + slo_q) atomicAdd(&wm.miss[j], 1u);
-            uint64_t h_arr = 0;
+            if (FEAS) {      // counted in a register; the group's shared count is brought up to date every eighth iteration
+                miss_local += (late_valid && late_fin > (late_arr & ~qmask) + slo_q) ? 1u : 0u;
+                late_valid = false;
+            }
+            // (loaded straight into the register that is carried to the next iteration: nothing in this
+            // iteration waits for it)
             if (FEAS && h_valid && (da < 0 || (db < 0 && bit >= 0)) && IL_IN_RANGE(h_qid, p.n, p.status))
-                h_arr = p.ptrace[h_qid];
-            if (FEAS) late_valid = false;
+                late_arr = __ldg(p.ptrace + h_qid);
             // likewise the next batch to hand on, if the one in hand is used up (a batch handed over in
             // this iteration is picked up in the next), and the table entry a close would need
             const bool f_valid = e_left == 0 && epos != lpos;
@@ -504,7 +513,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                 if (FEAS) {
                     const bool leaves = to_b ? db < 0 : da < 0;
                     if (h_valid && leaves) {
-                        late_valid = true; late_fin = h_base; late_arr = h_arr;
+                        late_valid = true; late_fin = h_base;
                     } else if (h_valid) {
                         uint64_t *dst = to_b ? out_b + (tail_b & mask_b) : out_a + (tail_a & mask_a);
                         if (IL_IN_RANGE(to_b ? (tail_b & mask_b) : (tail_a & mask_a), to_b ? size_b : size_a, p.status))
@@ -519,7 +528,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                 tail_a += (h_valid && !to_b) ? 1u : 0u;
             } else if (h_valid) {
                 if (FEAS && da < 0) {
-                    late_valid = true; late_fin = h_base; late_arr = h_arr;
+                    late_valid = true; late_fin = h_base;
                 } else if (IL_IN_RANGE(tail_a & mask_a, size_a, p.status)) {
                     out_a[tail_a & mask_a] = h_base | h_qid;
                 }
