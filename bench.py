@@ -46,14 +46,21 @@ WORKLOADS = {
 # proportion to the query-events processed).  Each entry names the SHA-256 of the kernel source it was taken
 # from; when the source in the tree differs, the figures that depend on the capture are reported as null.
 NCU_CAPTURES = {
+    # whole streams (workloads 1, 2, 3, 5): 16,384 candidates x 8,000 queries of workload 2, all warp slots busy
     "des_lane_kernel": {
         "source": "paper_1812_01776_b200/csrc/des_lane_kernel.cu",
-        "source_sha256": "",
-        "dram_bytes_per_query_event": 7.37, "warp_inst_per_query_event": 6.53,
+        "source_sha256": "8269d53b0207513c9937028fc0a1dff55739d786942c7232474508678458d9f7",
+        "dram_bytes_per_query_event": 8.85, "warp_inst_per_query_event": 6.60,
         "summary": "profiles/des_lane_kernel_config2.md"},
+    # stream rings (workload 4): 3,552 candidates x 20,000 queries of workload 4, all warp slots busy
+    "des_lane_kernel:rings": {
+        "source": "paper_1812_01776_b200/csrc/des_lane_kernel.cu",
+        "source_sha256": "8269d53b0207513c9937028fc0a1dff55739d786942c7232474508678458d9f7",
+        "dram_bytes_per_query_event": 9.02, "warp_inst_per_query_event": 6.76,
+        "summary": "profiles/des_lane_kernel_config4_rings.md"},
     "des_packed_kernel": {
         "source": "paper_1812_01776_b200/csrc/des_packed_kernel.cu",
-        "source_sha256": "",
+        "source_sha256": "",       # not captured again since the kernel got its node-stage entry and checks
         "dram_bytes_per_query_event": 12.24, "warp_inst_per_query_event": 32.9,
         "summary": "profiles/des_packed_kernel_config2.md"},
 }
@@ -96,10 +103,12 @@ def reduce_sum(values, dist=None, device=None):
     return t.tolist()
 
 
-def ncu_capture(kernel: str):
+def ncu_capture(kernel: str, rings: bool = False):
     """The capture record of `kernel` if it still describes the source in the tree, else None."""
     import hashlib
-    cap = NCU_CAPTURES.get(kernel.split("<")[0])
+    name = kernel.split("<")[0]
+    cap = NCU_CAPTURES.get(name + ":rings") if rings else None
+    cap = cap or NCU_CAPTURES.get(name)
     if not cap:
         return None
     try:
@@ -343,7 +352,9 @@ def measure(il, torch, w, dev, stream, flush, steps, warmup, e2e_steps, variant,
     rec_bytes = 12 if kernel == "des_kernel" else 8  # separate time/query streams, else one 64-bit record
     slab_bytes = 8 * n * n_cand                       # written once by the simulation, read once by the select
     stream_bytes = (events_per_cand - n) * 2 * rec_bytes * n_cand   # written once, read once
-    cap = None if shared else ncu_capture(kernel)
+    # the lane kernel keeps its streams in rings when whole streams of all resident candidates pass 48 GiB
+    rings = kernel == "des_lane_kernel" and (events_per_cand - n) * 8 * 148 * 8 * (32 // S) > 48 * 2**30
+    cap = None if shared else ncu_capture(kernel, rings)
     alu_peak = issue_rate * 32.0
     hbm_note = ("latency slab written once + every inter-stage stream record written once "
                 "and read once (the streams are this design's, not the method's)")
