@@ -20,10 +20,11 @@
  *     min(queue length, max batch) queries from the front at once (the
  *     lowest-id idle replica first) and is busy for
  *     latency_us[stage][hw][b-1] microseconds, b being the batch it took;
- *   - all queries of the batch leave the stage together; each follows the one
- *     child edge whose condition its branch bits satisfy, with zero delay, in
- *     batch order; a query with no such edge leaves the pipeline and its
- *     latency is that instant minus its arrival time;
+ *   - all queries of the batch leave the stage together; each follows every
+ *     child edge whose condition its branch bits satisfy (with conditional
+ *     control flow: at most one), with zero delay, in batch order; a copy with
+ *     no such edge leaves the pipeline, and the query's latency is the instant
+ *     its last copy leaves minus its arrival time;
  *   - everything at one timestamp happens as: all completions (batches
  *     dispatched earlier first), then all trace arrivals (in trace order), then
  *     dispatching;
@@ -82,13 +83,23 @@ typedef struct il_estimator il_estimator;   /* opaque; owns its device copies */
  * hardware type and batch size, how long the model takes for that batch).
  * All pointers are HOST pointers, read during il_estimator_create only.
  *
- * The pipeline is a tree.  Stage 0 is the root, parent[s] < s.  The edge
- * parent[s] -> s is taken by query q iff cond_bit[s] < 0, or
- * ((branch_bits[q] >> cond_bit[s]) & 1) == cond_val[s].  The children of one
- * stage must be either a single unconditional child, or one or two children
- * guarded by the SAME bit with different values; so a query follows at most
- * one edge, and a guarded edge without sibling is a cascade (the other queries
- * leave the pipeline there).
+ * The pipeline is a tree.  Stage 0 is the root, parent[s] < s, and a stage has
+ * at most two children.  The edge parent[s] -> s is taken by query q iff
+ * cond_bit[s] < 0, or ((branch_bits[q] >> cond_bit[s]) & 1) == cond_val[s].
+ * A query goes down EVERY edge of a stage whose condition it satisfies, and
+ * where it satisfies none, that copy of it leaves the pipeline; the query is
+ * answered when its last copy has left, and its latency is that instant minus
+ * its arrival time (Section 2: a pipeline is a DAG whose edges are dataflow;
+ * Section 4.3: the service time is taken along the longest path).  Two children
+ * guarded by the SAME bit with different values are alternatives (conditional
+ * control flow: one path per query), and a guarded edge without sibling is a
+ * cascade (the other queries leave there).  Two children that are not
+ * alternatives -- both unconditional, or guarded by different bits -- are
+ * fan-out: parallel branches.  A stage still has ONE parent: a model that waits
+ * for the outputs of two parents cannot be described.  Handles with fan-out run
+ * on the lane kernel (whole streams) or the kernel with separate streams; the
+ * other kernel choices, prefix sharing and the early exit of il_feasible fall
+ * back to those.
  */
 typedef struct {
     int32_t        n_stages;    /* S, 1..IL_MAX_STAGES                                  */
