@@ -62,6 +62,13 @@ def _load():
         lib.orc_estimate_one.argtypes = [ctypes.c_int32] * 3 + [p] * 4 + [ctypes.c_int64, p, p,
                                          p, ctypes.c_int64, ctypes.c_int32, p, p, p, p,
                                          ctypes.c_int64, p]
+        lib.orc_estimate_one_dag.restype = ctypes.c_int
+        lib.orc_estimate_one_dag.argtypes = [ctypes.c_int32] * 3 + [p] * 7 + [ctypes.c_int64, p, p,
+                                             p, ctypes.c_int64, ctypes.c_int32, p, p, p, p,
+                                             ctypes.c_int64, p]
+        lib.orc_estimate_many_dag.restype = ctypes.c_int
+        lib.orc_estimate_many_dag.argtypes = [ctypes.c_int32] * 3 + [p] * 7 + [ctypes.c_int64, p, p,
+                                              p, ctypes.c_int64, ctypes.c_int64, p, p]
         lib.orc_estimate_many.restype = ctypes.c_int
         lib.orc_estimate_many.argtypes = [ctypes.c_int32] * 3 + [p] * 4 + [ctypes.c_int64, p, p,
                                           p, ctypes.c_int64, ctypes.c_int64, p, p]
@@ -90,9 +97,20 @@ def _prep(parent, cond_bit, cond_val, latency_us, arrival_us, branch_bits):
     return parent, cond_bit, cond_val, latency_us, arrival_us, branch_bits, S, H, B
 
 
+def _prep_join(join, S):
+    """join = None or (parent2, cond_bit2, cond_val2): per stage the second incoming edge."""
+    if join is None:
+        return None, None, None
+    parent2 = np.ascontiguousarray(join[0], dtype=np.int32)
+    cond_bit2 = np.ascontiguousarray(join[1], dtype=np.int8)
+    cond_val2 = np.ascontiguousarray(join[2], dtype=np.uint8)
+    assert parent2.shape == (S,) and cond_bit2.shape == (S,) and cond_val2.shape == (S,)
+    return parent2, cond_bit2, cond_val2
+
+
 def estimate_one(parent, cond_bit, cond_val, latency_us, arrival_us, branch_bits,
                  config, slo_us: int, replica_pref: int = 0, want_latency: bool = False,
-                 want_log: bool = False):
+                 want_log: bool = False, join=None):
     """Simulate one candidate; returns (p99_us, miss[, latency][, dispatch log])."""
     lib = _load()
     parent, cond_bit, cond_val, latency_us, arrival_us, branch_bits, S, H, B = _prep(
@@ -104,7 +122,9 @@ def estimate_one(parent, cond_bit, cond_val, latency_us, arrival_us, branch_bits
     lat = np.empty(n, dtype=np.int64) if want_latency else None
     cap = int(n) * S if want_log else 0
     log = np.zeros(cap, dtype=DISPATCH_DTYPE) if want_log else None
-    rc = lib.orc_estimate_one(S, H, B, _ptr(parent), _ptr(cond_bit), _ptr(cond_val),
+    parent2, cond_bit2, cond_val2 = _prep_join(join, S)
+    rc = lib.orc_estimate_one_dag(S, H, B, _ptr(parent), _ptr(cond_bit), _ptr(cond_val),
+                              _ptr(parent2), _ptr(cond_bit2), _ptr(cond_val2),
                               _ptr(latency_us), n, _ptr(arrival_us), _ptr(branch_bits),
                               _ptr(config), int(slo_us), int(replica_pref),
                               ctypes.addressof(p99), ctypes.addressof(miss), _ptr(lat),
@@ -120,7 +140,7 @@ def estimate_one(parent, cond_bit, cond_val, latency_us, arrival_us, branch_bits
 
 
 def estimate_many(parent, cond_bit, cond_val, latency_us, arrival_us, branch_bits,
-                  configs, slo_us: int) -> Tuple[np.ndarray, np.ndarray]:
+                  configs, slo_us: int, join=None) -> Tuple[np.ndarray, np.ndarray]:
     """Simulate configs[c] for every c, one after the other, on this thread."""
     lib = _load()
     parent, cond_bit, cond_val, latency_us, arrival_us, branch_bits, S, H, B = _prep(
@@ -130,7 +150,9 @@ def estimate_many(parent, cond_bit, cond_val, latency_us, arrival_us, branch_bit
     C = configs.shape[0]
     p99 = np.zeros(C, dtype=np.int64)
     miss = np.zeros(C, dtype=np.int64)
-    rc = lib.orc_estimate_many(S, H, B, _ptr(parent), _ptr(cond_bit), _ptr(cond_val),
+    parent2, cond_bit2, cond_val2 = _prep_join(join, S)
+    rc = lib.orc_estimate_many_dag(S, H, B, _ptr(parent), _ptr(cond_bit), _ptr(cond_val),
+                               _ptr(parent2), _ptr(cond_bit2), _ptr(cond_val2),
                                _ptr(latency_us), arrival_us.shape[0], _ptr(arrival_us),
                                _ptr(branch_bits), _ptr(configs), C, int(slo_us),
                                _ptr(p99), _ptr(miss))
@@ -143,7 +165,7 @@ def estimate_workload(w, lo: int = 0, hi: Optional[int] = None):
     """estimate_many over candidates [lo, hi) of a workloads.Workload-like object."""
     hi = w.configs.shape[0] if hi is None else hi
     return estimate_many(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us,
-                         w.branch_bits, w.configs[lo:hi], w.slo_us)
+                         w.branch_bits, w.configs[lo:hi], w.slo_us, join=getattr(w, "join", None))
 
 
 def _worker(args):

@@ -40,6 +40,10 @@
  *     time along the LONGEST path of the DAG).  With mutually exclusive
  *     conditions (the conditional control flow of Section 2) there is one copy
  *     and one path.  There is no delay between stages.
+ *   - A stage may have a SECOND incoming edge (a join: Section 2 draws pipelines as DAGs whose edges
+ *     are dataflow, so a model that consumes two models' outputs needs both).  A query enters the
+ *     join's queue at the instant the last of the incoming edges it follows delivers it -- one edge if
+ *     its branch bits switch the other one off -- and is processed there once.
  *   - Batch time is a dense table lookup lat[stage][hw][b-1] for the actual
  *     batch size b.
  *   - P99 is the k-th smallest latency, k = ceil(0.99 n) computed in integers
@@ -71,10 +75,15 @@ typedef struct {
     int32_t query;   /* arrival: trace index */
 } event_t;
 
+/* Completions of one instant are taken stage by stage (lower stage index first) and, within a stage, in
+ * the order their batches were dispatched.  While every stage has one parent the order between stages
+ * cannot matter; with a join it decides who enters the join's queue first, and a rule that a stage-wise
+ * formulation can follow as well is needed. */
 static int ev_less(const event_t *a, const event_t *b)
 {
     if (a->time != b->time) return a->time < b->time;
     if (a->kind != b->kind) return a->kind < b->kind;
+    if (a->kind == EV_COMPLETION && a->stage != b->stage) return a->stage < b->stage;
     return a->seq < b->seq;
 }
 
@@ -121,23 +130,38 @@ static int cmp_i64(const void *a, const void *b)
     return (x > y) - (x < y);
 }
 
-/* Checks the tree: parent[0] = -1, parent[s] < s, at most two children per
- * stage, each edge unconditional or guarded by one branch bit. */
+/* Checks the graph: parent[0] = -1, parent[s] < s, an optional second parent with
+ * parent[s] < parent2[s] < s, at most two outgoing edges per stage, each edge
+ * unconditional or guarded by one branch bit. */
 static int check_topology(int S, const int32_t *parent, const int8_t *cond_bit,
-                          const uint8_t *cond_val)
+                          const uint8_t *cond_val, const int32_t *parent2,
+                          const int8_t *cond_bit2, const uint8_t *cond_val2)
 {
     if (parent[0] != -1) return ORC_ERR_TOPOLOGY;
+    if (parent2 && parent2[0] != -1) return ORC_ERR_TOPOLOGY;
     for (int s = 1; s < S; s++) {
         if (parent[s] < 0 || parent[s] >= s) return ORC_ERR_TOPOLOGY;
         if (cond_bit[s] < -1 || cond_bit[s] > 7) return ORC_ERR_TOPOLOGY;
         if (cond_bit[s] >= 0 && cond_val[s] > 1) return ORC_ERR_TOPOLOGY;
+        if (parent2 && parent2[s] != -1) {
+            if (parent2[s] <= parent[s] || parent2[s] >= s) return ORC_ERR_TOPOLOGY;
+            if (cond_bit2[s] < -1 || cond_bit2[s] > 7) return ORC_ERR_TOPOLOGY;
+            if (cond_bit2[s] >= 0 && cond_val2[s] > 1) return ORC_ERR_TOPOLOGY;
+        }
     }
     for (int p = 0; p < S; p++) {
         int nchild = 0;
-        for (int c = 1; c < S; c++)
+        for (int c = 1; c < S; c++) {
             if (parent[c] == p && ++nchild > 2) return ORC_ERR_TOPOLOGY;
+            if (parent2 && parent2[c] == p && ++nchild > 2) return ORC_ERR_TOPOLOGY;
+        }
     }
     return ORC_OK;
+}
+
+static int edge_on(int8_t bit, uint8_t val, const uint8_t *branch_bits, int64_t q)
+{
+    return bit < 0 || (uint8_t)((branch_bits[q] >> bit) & 1) == val;
 }
 
 /*
@@ -150,9 +174,13 @@ static int check_topology(int S, const int32_t *parent, const int8_t *cond_bit,
  *   out_latency     NULL or int64[n]: latency of every query, by trace index
  *   out_log         NULL or room for log_cap dispatch records; *out_nlog gets
  *                   the number of batches dispatched (may exceed log_cap)
+ *   parent2, cond_bit2, cond_val2
+ *                   NULL (no joins), or per stage the second incoming edge: its
+ *                   source stage (-1: none) and its guard
  */
-int orc_estimate_one(int32_t S, int32_t H, int32_t Bmax,
+int orc_estimate_one_dag(int32_t S, int32_t H, int32_t Bmax,
                      const int32_t *parent, const int8_t *cond_bit, const uint8_t *cond_val,
+                     const int32_t *parent2, const int8_t *cond_bit2, const uint8_t *cond_val2,
                      const int32_t *latency_us,
                      int64_t n, const int64_t *arrival_us, const uint8_t *branch_bits,
                      const uint8_t *config, int64_t slo_us, int32_t replica_pref,
@@ -162,10 +190,14 @@ int orc_estimate_one(int32_t S, int32_t H, int32_t Bmax,
 {
     if (S < 1 || S > 16 || H < 1 || H > 8 || Bmax < 1 || Bmax > 64 || n < 1) return ORC_ERR_ARG;
     if (!parent || !cond_bit || !cond_val || !latency_us || !arrival_us || !config) return ORC_ERR_ARG;
-    int rc = check_topology(S, parent, cond_bit, cond_val);
+    if (parent2 && (!cond_bit2 || !cond_val2)) return ORC_ERR_ARG;
+    int rc = check_topology(S, parent, cond_bit, cond_val, parent2, cond_bit2, cond_val2);
     if (rc) return rc;
-    int any_cond = 0;
-    for (int s = 1; s < S; s++) any_cond |= (cond_bit[s] >= 0);
+    int any_cond = 0, any_join = 0;
+    for (int s = 1; s < S; s++) {
+        any_cond |= (cond_bit[s] >= 0);
+        if (parent2 && parent2[s] >= 0) { any_join = 1; any_cond |= (cond_bit2[s] >= 0); }
+    }
     if (any_cond && !branch_bits) return ORC_ERR_ARG;
     for (int64_t i = 0; i < (int64_t)S * H * Bmax; i++)
         if (latency_us[i] < 1) return ORC_ERR_PROFILE;
@@ -192,7 +224,12 @@ int orc_estimate_one(int32_t S, int32_t H, int32_t Bmax,
     uint8_t *done = (uint8_t *)calloc((size_t)n, 1);
     int32_t *copies = (int32_t *)malloc(sizeof(int32_t) * (size_t)n);   /* copies of the query still in the pipeline */
     heap.e = (event_t *)malloc(sizeof(event_t) * (size_t)heap.cap);
-    int ok = lat && done && copies && heap.e;
+    /* joins only: reach[s][q] = the query visits stage s; need[s][q] = how many of the stage's incoming
+     * edges deliver it; arrived[s][q] = how many have so far */
+    uint8_t *reach = any_join ? (uint8_t *)calloc((size_t)n * S, 1) : NULL;
+    uint8_t *need = any_join ? (uint8_t *)calloc((size_t)n * S, 1) : NULL;
+    uint8_t *arrived = any_join ? (uint8_t *)calloc((size_t)n * S, 1) : NULL;
+    int ok = lat && done && copies && heap.e && (!any_join || (reach && need && arrived));
     for (int s = 0; s < S; s++) {
         queue[s] = (int32_t *)malloc(sizeof(int32_t) * (size_t)n);
         busy[s] = (uint8_t *)calloc((size_t)R[s], 1);
@@ -210,6 +247,19 @@ int orc_estimate_one(int32_t S, int32_t H, int32_t Bmax,
         heap_push(&heap, ev);
         copies[i] = 1;
     }
+    if (any_join) {
+        /* which stages a query visits follows from its branch bits alone; parents come first in index order */
+        for (int64_t q = 0; q < n; q++) {
+            reach[q] = 1;
+            for (int c = 1; c < S; c++) {
+                int a = reach[(size_t)parent[c] * n + q] && edge_on(cond_bit[c], cond_val[c], branch_bits, q);
+                int b = parent2[c] >= 0 && reach[(size_t)parent2[c] * n + q] &&
+                        edge_on(cond_bit2[c], cond_val2[c], branch_bits, q);
+                need[(size_t)c * n + q] = (uint8_t)(a + b);
+                reach[(size_t)c * n + q] = (uint8_t)(a || b);
+            }
+        }
+    }
 
     while (heap.size > 0) {
         const int64_t clock = heap.e[0].time;
@@ -221,17 +271,18 @@ int orc_estimate_one(int32_t S, int32_t H, int32_t Bmax,
             busy[s][r] = 0;
             for (int j = 0; j < inflight_n[s][r]; j++) {
                 int32_t q = inflight[s][r * MB[s] + j];
-                int taken = 0;
+                int taken = 0;       /* copies that enter a queue now */
                 for (int c = s + 1; c < S; c++) {
-                    if (parent[c] != s) continue;
-                    if (cond_bit[c] < 0 ||
-                        (uint8_t)((branch_bits[q] >> cond_bit[c]) & 1) == cond_val[c]) {
-                        queue[c][qtail[c]++] = q;
-                        taken++;
-                    }
+                    int on = (parent[c] == s && edge_on(cond_bit[c], cond_val[c], branch_bits, q)) ||
+                             (any_join && parent2[c] == s && edge_on(cond_bit2[c], cond_val2[c], branch_bits, q));
+                    if (!on) continue;
+                    /* at a join the copy waits for the other input; the one that completes the set goes on */
+                    if (any_join && ++arrived[(size_t)c * n + q] < need[(size_t)c * n + q]) continue;
+                    queue[c][qtail[c]++] = q;
+                    taken++;
                 }
                 if (done[q]) { rc = ORC_ERR_INTERNAL; goto cleanup; }
-                copies[q] += taken - 1;      /* this copy went on as `taken` copies, or left */
+                copies[q] += taken - 1;      /* this copy went on as `taken` copies, was absorbed, or left */
                 if (copies[q] == 0) {        /* the last copy has left: the query is answered now */
                     done[q] = 1;
                     lat[q] = clock - arrival_us[q];
@@ -282,13 +333,45 @@ int orc_estimate_one(int32_t S, int32_t H, int32_t Bmax,
     }
 
 cleanup:
-    free(lat); free(done); free(copies); free(heap.e);
+    free(lat); free(done); free(copies); free(heap.e); free(reach); free(need); free(arrived);
     for (int s = 0; s < S; s++) { free(queue[s]); free(busy[s]); free(inflight[s]); free(inflight_n[s]); }
     return rc;
 }
 
+/* The same for a pipeline without joins. */
+int orc_estimate_one(int32_t S, int32_t H, int32_t Bmax,
+                     const int32_t *parent, const int8_t *cond_bit, const uint8_t *cond_val,
+                     const int32_t *latency_us,
+                     int64_t n, const int64_t *arrival_us, const uint8_t *branch_bits,
+                     const uint8_t *config, int64_t slo_us, int32_t replica_pref,
+                     int64_t *out_p99_us, int64_t *out_miss,
+                     int64_t *out_latency,
+                     orc_dispatch_t *out_log, int64_t log_cap, int64_t *out_nlog)
+{
+    return orc_estimate_one_dag(S, H, Bmax, parent, cond_bit, cond_val, NULL, NULL, NULL, latency_us,
+                                n, arrival_us, branch_bits, config, slo_us, replica_pref,
+                                out_p99_us, out_miss, out_latency, out_log, log_cap, out_nlog);
+}
+
 /* Plain loop over candidates [0, C): configs is [C][S][4] bytes.  Stops at the
  * first error and returns it. */
+int orc_estimate_many_dag(int32_t S, int32_t H, int32_t Bmax,
+                      const int32_t *parent, const int8_t *cond_bit, const uint8_t *cond_val,
+                      const int32_t *parent2, const int8_t *cond_bit2, const uint8_t *cond_val2,
+                      const int32_t *latency_us,
+                      int64_t n, const int64_t *arrival_us, const uint8_t *branch_bits,
+                      const uint8_t *configs, int64_t C, int64_t slo_us,
+                      int64_t *out_p99_us, int64_t *out_miss)
+{
+    for (int64_t c = 0; c < C; c++) {
+        int rc = orc_estimate_one_dag(S, H, Bmax, parent, cond_bit, cond_val, parent2, cond_bit2, cond_val2,
+                                      latency_us, n, arrival_us, branch_bits, configs + c * S * 4, slo_us, 0,
+                                      out_p99_us + c, out_miss + c, NULL, NULL, 0, NULL);
+        if (rc) return rc;
+    }
+    return ORC_OK;
+}
+
 int orc_estimate_many(int32_t S, int32_t H, int32_t Bmax,
                       const int32_t *parent, const int8_t *cond_bit, const uint8_t *cond_val,
                       const int32_t *latency_us,

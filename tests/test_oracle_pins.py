@@ -178,8 +178,11 @@ def test_hand_traces(oracle, case):
     topo = (np.array(case["parent"], np.int32), np.array(case["cond_bit"], np.int8),
             np.array(case["cond_val"], np.uint8), np.array(case["latency_us"], np.int32))
     bits = np.array(case["branch_bits"], np.uint8) if "branch_bits" in case else None
+    kw = {}
+    if "join" in case:
+        kw["join"] = (case["join"]["parent2"], case["join"]["cond_bit2"], case["join"]["cond_val2"])
     p99, miss, lat = run(oracle, topo, case["arrival_us"], np.array(case["config"], np.uint8),
-                         slo=case["slo_us"], bits=bits, want_latency=True)
+                         slo=case["slo_us"], bits=bits, want_latency=True, **kw)
     assert lat.tolist() == case["latency"]
     assert p99 == case["p99_us"]
     assert miss == case["miss"]
@@ -197,7 +200,31 @@ def tick_simulate(w, cfg):
     heap, no event records): usable only when all times are tiny."""
     S = w.n_stages
     n = w.n_queries
-    kids = [[c for c in range(S) if w.parent[c] == s] for s in range(S)]
+    join = getattr(w, "join", None)
+    # edges[s] = [(child, guard bit, guard value)], child by child
+    edges = [[] for _ in range(S)]
+    for c in range(1, S):
+        edges[int(w.parent[c])].append((c, int(w.cond_bit[c]), int(w.cond_val[c])))
+        if join is not None and int(join[0][c]) >= 0:
+            edges[int(join[0][c])].append((c, int(join[1][c]), int(join[2][c])))
+    for e in edges:
+        e.sort()
+
+    def follows(q, bit, val):
+        return bit < 0 or ((int(w.branch_bits[q]) >> bit) & 1) == val
+
+    def inputs_of(q):
+        """per stage, how many of its incoming edges carry query q"""
+        seen = [0] * S
+        seen[0] = 1
+        for s in range(S):                     # parents come before children
+            if seen[s]:
+                for c, bit, val in edges[s]:
+                    seen[c] += follows(q, bit, val)
+        return seen
+
+    wanted = [inputs_of(q) for q in range(n)]
+    got = [[0] * S for _ in range(n)]
     queue = [[] for _ in range(S)]
     running = [dict() for _ in range(S)]     # replica -> (finish, order, [ids])
     order = 0
@@ -207,15 +234,20 @@ def tick_simulate(w, cfg):
     t = int(w.arrival_us[0])
     left = n
     while left:
-        fin = sorted((f, o, s, r) for s in range(S) for r, (f, o, _) in running[s].items() if f == t)
-        for _, _, s, r in fin:
+        # batches that finish now: stage by stage, within a stage in dispatch order
+        fin = sorted((s, o, r) for s in range(S) for r, (f, o, _) in running[s].items() if f == t)
+        for s, _, r in fin:
             ids = running[s].pop(r)[2]
             for q in ids:
-                c = [c for c in kids[s] if w.cond_bit[c] < 0
-                     or ((int(w.branch_bits[q]) >> int(w.cond_bit[c])) & 1) == int(w.cond_val[c])]
-                for child in c:                       # every edge whose condition holds
-                    queue[child].append(q)
-                copies[q] += len(c) - 1
+                went_on = 0
+                for child, bit, val in edges[s]:      # every edge whose condition holds
+                    if not follows(q, bit, val):
+                        continue
+                    got[q][child] += 1
+                    if got[q][child] == wanted[q][child]:   # the stage has all its inputs for q
+                        queue[child].append(q)
+                        went_on += 1
+                copies[q] += went_on - 1
                 if copies[q] == 0:                    # the last copy of the query has left
                     lat[q] = t - int(w.arrival_us[q])
                     left -= 1
@@ -549,3 +581,82 @@ def test_fan_out_never_queue_limit_is_the_longest_path(oracle):
         if w.branch_bits[q] & 1:
             paths.append(d[0] + d[2] + d[4])
         assert lat[q] == max(paths)
+
+
+# --------------------------------------------------------------------------
+# joins: a stage with two incoming edges takes a query when the last of the
+# edges the query follows has delivered it
+# --------------------------------------------------------------------------
+
+def _one(oracle, w, cfg, **kw):
+    return oracle.estimate_one(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us, w.branch_bits,
+                               cfg, 0, want_latency=True, join=w.join, **kw)[2]
+
+
+@pytest.mark.parametrize("shape", ["diamond", "guarded", "two_joins"])
+@pytest.mark.parametrize("seed", range(8))
+def test_join_tick_brute_force(oracle, seed, shape):
+    w = workloads.join_small(seed, n=40, C=6, max_replicas=3, Bmax=4, tiny_times=True, shape=shape)
+    for c in range(w.n_candidates):
+        assert np.array_equal(_one(oracle, w, w.configs[c]), tick_simulate(w, w.configs[c])), (seed, c)
+
+
+@pytest.mark.parametrize("fast", [1, 2])
+@pytest.mark.parametrize("seed", range(5))
+def test_join_with_an_instant_branch_is_the_other_chain(oracle, seed, fast):
+    """Diamond 0 -> {1, 2} -> 3 in which one branch takes 1 us and never queues (32 replicas, at most
+    32 queries leave stage 0 in one instant) while the other needs at least 2 us: the slow branch always
+    delivers last, so stage 3 sees exactly what it sees in the linear chain 0 -> slow -> 3, which the
+    tandem recursions above pin."""
+    slow = 3 - fast
+    w = workloads.join_small(20 + seed, n=500, C=6, max_replicas=4, Bmax=8)
+    w.latency_us = np.maximum(w.latency_us, 2)
+    w.latency_us[fast] = 1
+    lin = np.array([-1, 0, 1], np.int32)
+    for c in range(w.n_candidates):
+        cfg = w.configs[c].copy()
+        cfg[fast] = (0, 1, 32, 0)
+        a = _one(oracle, w, cfg)
+        _, _, b = oracle.estimate_one(lin, np.full(3, -1, np.int8), np.zeros(3, np.uint8),
+                                      w.latency_us[[0, slow, 3]], w.arrival_us, None, cfg[[0, slow, 3]], 0,
+                                      want_latency=True)
+        assert np.array_equal(a, b), (seed, c)
+
+
+def test_join_never_queue_limit_is_the_longest_path(oracle):
+    """Section 4.3 again: with replicas to spare and spaced arrivals the latency is the sum of batch-1
+    times along the longest path, here d0 + max(d1, d2) + d3 (+ d4 behind the join)."""
+    w = workloads.join_small(4, n=60, shape="guarded")
+    w.arrival_us = np.arange(60, dtype=np.int64) * 200_000
+    cfg = np.array([[1, 4, 3, 0]] * 5, np.uint8)
+    d = w.latency_us[:, 1, 0].astype(np.int64)
+    lat = _one(oracle, w, cfg)
+    for q in range(60):
+        mid = max(d[1], d[2]) if w.branch_bits[q] & 1 else d[1]     # bit 0 clear: stage 2 is skipped
+        assert lat[q] == d[0] + mid + d[3] + d[4]
+
+
+def test_join_guard_that_is_never_true_is_no_join(oracle):
+    """If no query follows the second edge the join has one input and the graph is the tree without it."""
+    w = workloads.join_small(9, n=300, shape="guarded")
+    w.branch_bits[:] &= 0xFE                                        # bit 0 clear everywhere: nobody visits 2
+    lin = np.array([-1, 0, 1, 2], np.int32)
+    for c in range(4):
+        a = _one(oracle, w, w.configs[c])
+        _, _, b = oracle.estimate_one(lin, np.full(4, -1, np.int8), np.zeros(4, np.uint8),
+                                      w.latency_us[[0, 1, 3, 4]], w.arrival_us, None, w.configs[c][[0, 1, 3, 4]],
+                                      0, want_latency=True)
+        assert np.array_equal(a, b)
+
+
+def test_join_rejects_bad_second_parents(oracle):
+    w = workloads.join_small(1, n=20)
+    for p2 in ([-1, -1, -1, 1], [-1, -1, -1, 3], [-1, -1, -1, 0], [0, -1, -1, 2]):
+        with pytest.raises(oracle.OracleError) as e:       # not above the first parent / not below the stage
+            oracle.estimate_one(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us, w.branch_bits,
+                                w.configs[0], 0, join=(p2, w.join[1], w.join[2]))
+        assert e.value.code == -2
+    # a third outgoing edge from stage 0
+    with pytest.raises(oracle.OracleError):
+        oracle.estimate_one(np.array([-1, 0, 0, 0], np.int32), w.cond_bit, w.cond_val, w.latency_us, w.arrival_us,
+                            w.branch_bits, w.configs[0], 0, join=w.join)

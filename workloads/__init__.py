@@ -51,6 +51,8 @@ class Workload:
     arrival_us     int64 [n], non-decreasing
     branch_bits    uint8 [n]
     configs        uint8 [C][S][4] = (hw, max_batch, replicas, 0) per stage
+    join           None, or (parent2, cond_bit2, cond_val2): per stage a second incoming
+                   edge (parent2[s] = -1: none; else parent[s] < parent2[s] < s) and its guard
     """
 
     name: str
@@ -63,6 +65,7 @@ class Workload:
     configs: np.ndarray
     slo_us: int
     recipe: Dict[str, object] = field(default_factory=dict)
+    join: Optional[tuple] = None
 
     @property
     def n_stages(self) -> int:
@@ -325,6 +328,40 @@ def fan_out_small(seed: int, n: int = 900, C: int = 30, max_replicas: int = 4, B
     rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([BASE_SEED, 98, seed])))
     w.branch_bits = rng.integers(0, 4, n).astype(np.uint8)
     w.name = f"fanout{seed}"
+    return w
+
+
+def join_small(seed: int, n: int = 900, C: int = 30, max_replicas: int = 4, Bmax: int = 8,
+               tiny_times: bool = False, shape: str = "diamond") -> Workload:
+    """A small pipeline with a join (Section 2: a DAG in which a model consumes two models' outputs).
+
+    diamond     0 -> {1, 2} -> 3: every query runs 1 and 2 in parallel and enters 3 when both are done.
+    guarded     0 -> {1, 2 if bit 0 is 1}; 3 joins 1 and 2; 3 -> 4.  A query with bit 0 clear reaches 3
+                through stage 1 alone.
+    two_joins   0 -> {1, 2}; 3 joins 1 and 2; 1 is a fork as well: 1 -> {3, 4 if bit 1 is 1}; 5 joins 3 and 4
+                (the second edge, 4 -> 5, only exists for queries that visited 4)."""
+    S = {"diamond": 4, "guarded": 5, "two_joins": 6}[shape]
+    w = random_small(seed, S=S, H=2, Bmax=Bmax, n=n, C=C, max_replicas=max_replicas, tree=False,
+                     qps=80_000.0 if tiny_times else 300.0, cv=2.0, lat_lo=1,
+                     lat_hi=30 if tiny_times else 9000, equal_stamp_every=(3 if seed % 2 == 0 else 0))
+    if shape == "diamond":
+        w.parent = np.array([-1, 0, 0, 1], np.int32)
+        w.cond_bit = np.array([-1, -1, -1, -1], np.int8)
+        w.cond_val = np.zeros(4, np.uint8)
+        w.join = (np.array([-1, -1, -1, 2], np.int32), np.full(4, -1, np.int8), np.zeros(4, np.uint8))
+    elif shape == "guarded":
+        w.parent = np.array([-1, 0, 0, 1, 3], np.int32)
+        w.cond_bit = np.array([-1, -1, 0, -1, -1], np.int8)
+        w.cond_val = np.array([0, 0, 1, 0, 0], np.uint8)
+        w.join = (np.array([-1, -1, -1, 2, -1], np.int32), np.full(5, -1, np.int8), np.zeros(5, np.uint8))
+    else:
+        w.parent = np.array([-1, 0, 0, 1, 1, 3], np.int32)
+        w.cond_bit = np.array([-1, -1, -1, -1, 1, -1], np.int8)
+        w.cond_val = np.array([0, 0, 0, 0, 1, 0], np.uint8)
+        w.join = (np.array([-1, -1, -1, 2, -1, 4], np.int32), np.full(6, -1, np.int8), np.zeros(6, np.uint8))
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([BASE_SEED, 97, seed])))
+    w.branch_bits = rng.integers(0, 4, n).astype(np.uint8)
+    w.name = f"join_{shape}{seed}"
     return w
 
 
