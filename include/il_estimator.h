@@ -95,11 +95,11 @@ typedef struct il_estimator il_estimator;   /* opaque; owns its device copies */
  * control flow: one path per query), and a guarded edge without sibling is a
  * cascade (the other queries leave there).  Two children that are not
  * alternatives -- both unconditional, or guarded by different bits -- are
- * fan-out: parallel branches.  A stage still has ONE parent: a model that waits
- * for the outputs of two parents cannot be described.  Handles with fan-out run
- * on the lane kernel (whole streams) or the kernel with separate streams; the
- * other kernel choices, prefix sharing and the early exit of il_feasible fall
- * back to those.
+ * fan-out: parallel branches.  Handles with fan-out run on the lane kernel
+ * (whole streams) or the kernel with separate streams; the other kernel
+ * choices, prefix sharing and the early exit of il_feasible fall back to those.
+ * A stage that waits for the outputs of TWO stages (a join) is described with
+ * il_join_edges and il_estimator_create_dag below.
  */
 typedef struct {
     int32_t        n_stages;    /* S, 1..IL_MAX_STAGES                                  */
@@ -166,6 +166,38 @@ typedef struct {
  * 62 bits), NOMEM, CUDA.
  */
 IL_API int il_estimator_create(const il_profiles *profiles, const il_trace *trace, il_estimator **out);
+
+/*
+ * Joins (Section 2: the pipeline is a DAG whose edges are dataflow, so a model
+ * may consume the outputs of two models).  Per stage s an optional SECOND
+ * incoming edge parent2[s] -> s, with parent[s] < parent2[s] < s, guarded like
+ * the first one by (cond_bit2[s], cond_val2[s]); parent2[s] = -1: none.  A query
+ * enters the queue of stage s at the instant the LAST of the incoming edges it
+ * follows delivers it (both, or the only one its branch bits leave on) and is
+ * processed there once.  Queries that become ready in the same instant queue in
+ * the order (delivering stage, that stage's completion order).  A stage still
+ * has at most two outgoing edges, counting both kinds.  HOST pointers, [S] each,
+ * read during the call only.
+ */
+typedef struct {
+    const int32_t *parent2;     /* [S], -1 or parent[s] < parent2[s] < s                */
+    const int8_t  *cond_bit2;   /* [S], -1 or 0..7                                      */
+    const uint8_t *cond_val2;   /* [S], 0 or 1 (ignored where cond_bit2 < 0)            */
+} il_join_edges;
+
+/*
+ * il_estimator_create for a pipeline with joins; `joins` may be NULL (then the
+ * two calls are the same).  A handle with a join runs on the kernel with
+ * separate streams (kernel name "des_kernel") whatever variant is set: that
+ * kernel builds the join's arrival stream from the two incoming streams before
+ * it simulates the stage.  Every entry point works on such a handle and gives
+ * the same results as on any other; il_feasible* evaluate it without early exit.
+ * Errors: as il_estimator_create; BAD_TOPOLOGY also for a second edge outside
+ * the form above or a third outgoing edge; TOO_LARGE if the streams of one
+ * candidate exceed 2^31 - 1 elements.
+ */
+IL_API int il_estimator_create_dag(const il_profiles *profiles, const il_join_edges *joins,
+                                   const il_trace *trace, il_estimator **out);
 
 /* Frees the handle and everything the library allocated for it.  Memory given
  * through il_set_workspace stays the caller's.  NULL is allowed. */

@@ -48,6 +48,77 @@ struct Route {
     bool a_exit, b_exit;
 };
 
+// Number of leading elements of the sorted array t[0 .. len) that are < key (strict) or <= key.
+__device__ __forceinline__ int count_below(const int64_t *t, int len, int64_t key, bool or_equal)
+{
+    int a = 0, b = len;
+    while (a < b) {
+        const int m = (a + b) >> 1;
+        const int64_t v = t[m];
+        if (v < key || (or_equal && v == key)) a = m + 1; else b = m;
+    }
+    return a;
+}
+
+// Arrival stream of a join (a stage with two incoming edges), built by one warp from the two incoming
+// streams A (edge from the first parent, na records) and B (edge from the second parent, nb records), both
+// sorted by time.  A query is ready at the join when the last of its inputs has arrived, and queries that
+// become ready in the same instant queue in the order (delivering stage, that stage's completion order);
+// the first parent has the smaller stage index.  So the stream is the merge of
+//   Y: the records of A whose query has no record in B, or an earlier one   (made ready by the first parent)
+//   X: the records of B whose query has no record in A, or one that is not later (made ready by the second)
+// with Y before X at equal times; both halves are subsequences of sorted streams, hence sorted, and an
+// element's place in the merge is its index in its own half plus the number of elements of the other half
+// that go before it, found by bisection.  Returns the length of the merged stream.
+__device__ int build_join_stream(const DesParams &p, int s, int64_t *my_time, int32_t *my_qid, int lane)
+{
+    const unsigned full = 0xffffffffu;
+    const unsigned lt_mask = (1u << lane) - 1u;
+    const int na = p.join_na[s], nb = p.join_nb[s];
+    const int64_t *ta = my_time + p.join_in_a[s]; const int32_t *qa = my_qid + p.join_in_a[s];
+    const int64_t *tb = my_time + p.join_in_b[s]; const int32_t *qb = my_qid + p.join_in_b[s];
+    const int64_t n_pad = (p.n + 31) / 32 * 32;
+    int64_t *seen_a = my_time + p.join_t_off, *seen_b = seen_a + n_pad;     // time of the query's record, -1: none
+    for (int i = lane; i < p.n; i += 32) { seen_a[i] = -1; seen_b[i] = -1; }
+    __syncwarp();
+    for (int i = lane; i < na; i += 32) { const int32_t q = qa[i]; if (IL_IN_RANGE(q, p.n, p.status)) seen_a[q] = ta[i]; }
+    for (int i = lane; i < nb; i += 32) { const int32_t q = qb[i]; if (IL_IN_RANGE(q, p.n, p.status)) seen_b[q] = tb[i]; }
+    __syncwarp();
+    int64_t *ty = my_time + p.join_tmp_off; int32_t *qy = my_qid + p.join_tmp_off;
+    int64_t *tx = ty + (na + 31) / 32 * 32; int32_t *qx = qy + (na + 31) / 32 * 32;
+    int ny = 0, nx = 0;
+    for (int i0 = 0; i0 < na; i0 += 32) {
+        const int i = i0 + lane;
+        bool keep = false; int64_t t = 0; int32_t q = 0;
+        if (i < na) { t = ta[i]; q = qa[i]; if (IL_IN_RANGE(q, p.n, p.status)) keep = t > seen_b[q]; }   // -1: no record in B
+        const unsigned m = __ballot_sync(full, keep);
+        if (keep) { const int at = ny + __popc(m & lt_mask); ty[at] = t; qy[at] = q; }
+        ny += __popc(m);
+    }
+    for (int i0 = 0; i0 < nb; i0 += 32) {
+        const int i = i0 + lane;
+        bool keep = false; int64_t t = 0; int32_t q = 0;
+        if (i < nb) { t = tb[i]; q = qb[i]; if (IL_IN_RANGE(q, p.n, p.status)) keep = t >= seen_a[q]; }
+        const unsigned m = __ballot_sync(full, keep);
+        if (keep) { const int at = nx + __popc(m & lt_mask); tx[at] = t; qx[at] = q; }
+        nx += __popc(m);
+    }
+    __syncwarp();
+    int64_t *out_t = my_time + p.buf_off[s]; int32_t *out_q = my_qid + p.buf_off[s];
+    const int total = nx + ny;
+    if (total != p.n_s[s]) return -1;          // the host counted something else: give up before writing
+    for (int i = lane; i < ny; i += 32) {
+        const int at = i + count_below(tx, nx, ty[i], false);
+        out_t[at] = ty[i]; out_q[at] = qy[i];
+    }
+    for (int i = lane; i < nx; i += 32) {
+        const int at = i + count_below(ty, ny, tx[i], true);
+        out_t[at] = tx[i]; out_q[at] = qx[i];
+    }
+    __syncwarp();
+    return total;
+}
+
 }  // namespace
 
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
@@ -99,6 +170,11 @@ des_kernel(const __grid_constant__ DesParams p)
         for (int s = 0; s < p.S; s++) {
             const int n_in = p.n_s[s];
             if (n_in == 0) continue;
+            if (p.fork && p.join_b[s] >= 0 && build_join_stream(p, s, my_time, my_qid, lane) != n_in) {
+                if (lane == 0) { atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT); atomicOr(&p.counters[5], 16ull); }
+                over = true;
+                break;
+            }
             const int hw = __shfl_sync(full, (int)my_cfg.hw, s);
             const int mb = __shfl_sync(full, (int)my_cfg.max_batch, s);
             const int R = __shfl_sync(full, (int)my_cfg.replicas, s);
@@ -138,14 +214,14 @@ des_kernel(const __grid_constant__ DesParams p)
                         const unsigned fl = __ballot_sync(full, left);
                         if (go_a) {
                             const int at = rt.a_tail + __popc(fa & lt_mask);
-                            if (IL_IN_RANGE(p.buf_off[ca] + at, p.slot_elems, p.status)) {
-                                (my_time + p.buf_off[ca])[at] = tfin; (my_qid + p.buf_off[ca])[at] = q;
+                            if (IL_IN_RANGE(p.out_off_a[s] + at, p.slot_elems, p.status)) {
+                                (my_time + p.out_off_a[s])[at] = tfin; (my_qid + p.out_off_a[s])[at] = q;
                             }
                         }
                         if (go_b) {
                             const int at = rt.b_tail + __popc(fb & lt_mask);
-                            if (IL_IN_RANGE(p.buf_off[cb] + at, p.slot_elems, p.status)) {
-                                (my_time + p.buf_off[cb])[at] = tfin; (my_qid + p.buf_off[cb])[at] = q;
+                            if (IL_IN_RANGE(p.out_off_b[s] + at, p.slot_elems, p.status)) {
+                                (my_time + p.out_off_b[s])[at] = tfin; (my_qid + p.out_off_b[s])[at] = q;
                             }
                         }
                         if (left && IL_IN_RANGE(q, p.n, p.status)) {

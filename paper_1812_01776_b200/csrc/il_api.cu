@@ -43,6 +43,7 @@ struct il_estimator {
     uint64_t *d_ptrace = nullptr;      // packed root stream
     bool can_pack = false;             // every reachable time fits a packed record
     bool fork = false;                 // fan-out: one query can enter two children of a stage
+    bool join = false;                 // some stage has two incoming edges (implies fork: copies of a query exist)
     bool lane_ok = false;              // the lane kernel applies (packed records, stream offsets fit 31 bits)
     int variant = IL_VARIANT_AUTO;
     int ctas_per_sm_wide = 0, ctas_per_sm_packed = 0, ctas_per_sm_staged = 0, ctas_per_sm_lane = 0;
@@ -113,7 +114,7 @@ bool use_packed(const il_estimator *e)
 
 int sim_kernel(const il_estimator *e)
 {
-    if (!use_packed(e)) return kSimWide;
+    if (!use_packed(e) || e->join) return kSimWide;     // joins: only the kernel with separate streams merges them
     // fan-out is implemented by the lane kernel and by the kernel with separate streams
     if (e->fork) return (e->variant == IL_VARIANT_AUTO || e->variant == IL_VARIANT_LANES) && e->lane_ok ? kSimLane : kSimWide;
     if (e->variant == IL_VARIANT_LANES && e->lane_ok) return kSimLane;
@@ -230,18 +231,24 @@ bool make_plan(const il_estimator *e, size_t bytes, int64_t n_cand, Plan &pl)
     return pl.chunk >= 1;
 }
 
-int check_topology(const il_profiles *pr)
+int check_topology(const il_profiles *pr, const il_join_edges *jn)
 {
     const int S = pr->n_stages;
     if (pr->parent[0] != -1) return IL_ERR_BAD_TOPOLOGY;
+    if (jn && jn->parent2[0] != -1) return IL_ERR_BAD_TOPOLOGY;
     for (int s = 1; s < S; s++) {
         if (pr->parent[s] < 0 || pr->parent[s] >= s) return IL_ERR_BAD_TOPOLOGY;
         if (pr->cond_bit[s] < -1 || pr->cond_bit[s] > 7) return IL_ERR_BAD_TOPOLOGY;
         if (pr->cond_bit[s] >= 0 && pr->cond_val[s] > 1) return IL_ERR_BAD_TOPOLOGY;
+        if (jn && jn->parent2[s] != -1) {
+            if (jn->parent2[s] <= pr->parent[s] || jn->parent2[s] >= s) return IL_ERR_BAD_TOPOLOGY;
+            if (jn->cond_bit2[s] < -1 || jn->cond_bit2[s] > 7) return IL_ERR_BAD_TOPOLOGY;
+            if (jn->cond_bit2[s] >= 0 && jn->cond_val2[s] > 1) return IL_ERR_BAD_TOPOLOGY;
+        }
     }
     for (int par = 0; par < S; par++) {
         int nk = 0;
-        for (int c = 1; c < S; c++) if (pr->parent[c] == par) nk++;
+        for (int c = 1; c < S; c++) nk += (pr->parent[c] == par) + (jn && jn->parent2[c] == par);
         if (nk > 2) return IL_ERR_BAD_TOPOLOGY;
     }
     return IL_OK;
@@ -690,19 +697,29 @@ int il_last_cuda_error(void) { return g_last_cuda_error; }
 
 int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator **out)
 {
+    return il_estimator_create_dag(pr, nullptr, tr, out);
+}
+
+int il_estimator_create_dag(const il_profiles *pr, const il_join_edges *jn, const il_trace *tr, il_estimator **out)
+{
     if (!pr || !tr || !out) return IL_ERR_INVALID_ARG;
+    if (jn && (!jn->parent2 || !jn->cond_bit2 || !jn->cond_val2)) return IL_ERR_INVALID_ARG;
     if (pr->n_stages < 1 || pr->n_stages > IL_MAX_STAGES || pr->n_hw < 1 || pr->n_hw > IL_MAX_HW ||
         pr->max_batch < 1 || pr->max_batch > IL_MAX_BATCH)
         return IL_ERR_INVALID_ARG;
     if (!pr->parent || !pr->cond_bit || !pr->cond_val || !pr->latency_us || !tr->arrival_us)
         return IL_ERR_INVALID_ARG;
     if (tr->n_queries < 1 || tr->n_queries > INT32_MAX) return IL_ERR_INVALID_ARG;
-    int rc = check_topology(pr);
+    int rc = check_topology(pr, jn);
     if (rc) return rc;
     const int S = pr->n_stages, H = pr->n_hw, B = pr->max_batch;
     const int64_t n = tr->n_queries;
-    bool any_cond = false;
-    for (int s = 1; s < S; s++) any_cond |= pr->cond_bit[s] >= 0;
+    bool any_cond = false, any_join = false;
+    for (int s = 1; s < S; s++) {
+        any_cond |= pr->cond_bit[s] >= 0;
+        if (jn && jn->parent2[s] >= 0) { any_join = true; any_cond |= jn->cond_bit2[s] >= 0; }
+    }
+    if (!any_join) jn = nullptr;
     if (any_cond && !tr->branch_bits) return IL_ERR_INVALID_ARG;
 
     int64_t worst = 0;   // bound on how far the clock can run past the last arrival
@@ -749,36 +766,85 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
         }
     }
     for (int s = 0; s < S; s++) e->parent[s] = pr->parent[s];
-    e->fork = has_fan_out(pr);
+    e->join = any_join;
+    e->fork = any_join || has_fan_out(pr);
     bp.fork = e->fork ? 1 : 0;
-    for (int s = 0; s < IL_MAX_STAGES; s++) { bp.child_a[s] = -1; bp.child_b[s] = -1; bp.cbit_a[s] = -1; bp.cbit_b[s] = -1; }
-    for (int c = 1; c < S; c++) {
-        const int par = pr->parent[c];
-        if (bp.child_a[par] < 0) { bp.child_a[par] = (int8_t)c; bp.cbit_a[par] = pr->cond_bit[c]; bp.cval_a[par] = pr->cond_val[c]; }
-        else { bp.child_b[par] = (int8_t)c; bp.cbit_b[par] = pr->cond_bit[c]; bp.cval_b[par] = pr->cond_val[c]; }
+    for (int s = 0; s < IL_MAX_STAGES; s++) {
+        bp.child_a[s] = -1; bp.child_b[s] = -1; bp.cbit_a[s] = -1; bp.cbit_b[s] = -1; bp.join_b[s] = -1;
     }
-    // walk every query down every edge it takes
+    // outgoing edges of every stage, first-parent and second-parent edges alike
+    auto add_edge = [&](int par, int c, int bit, int val) {
+        if (bp.child_a[par] < 0) { bp.child_a[par] = (int8_t)c; bp.cbit_a[par] = (int8_t)bit; bp.cval_a[par] = (uint8_t)val; }
+        else { bp.child_b[par] = (int8_t)c; bp.cbit_b[par] = (int8_t)bit; bp.cval_b[par] = (uint8_t)val; }
+    };
+    for (int c = 1; c < S; c++) {
+        add_edge(pr->parent[c], c, pr->cond_bit[c], pr->cond_val[c]);
+        if (jn && jn->parent2[c] >= 0) {
+            add_edge(jn->parent2[c], c, jn->cond_bit2[c], jn->cond_val2[c]);
+            bp.join_b[c] = (int8_t)jn->parent2[c];
+        }
+    }
+    // Which stages a query visits follows from its branch bits alone (parents have smaller indices):
+    // count the visits per stage, the records on each edge into a join, and the copies that leave.
     bp.total_leaving = 0;
+    int64_t edge_a[IL_MAX_STAGES] = {}, edge_b[IL_MAX_STAGES] = {};
     for (int64_t q = 0; q < n; q++) {
-        int stack[IL_MAX_STAGES], top = 0;
-        stack[top++] = 0;
-        while (top > 0) {
-            const int s = stack[--top];
+        const unsigned bits = tr->branch_bits ? tr->branch_bits[q] : 0u;
+        bool reach[IL_MAX_STAGES] = {};
+        reach[0] = true;
+        for (int c = 1; c < S; c++) {
+            const bool a = reach[pr->parent[c]] && (pr->cond_bit[c] < 0 || ((bits >> pr->cond_bit[c]) & 1u) == pr->cond_val[c]);
+            const bool b = jn && jn->parent2[c] >= 0 && reach[jn->parent2[c]] &&
+                           (jn->cond_bit2[c] < 0 || ((bits >> jn->cond_bit2[c]) & 1u) == jn->cond_val2[c]);
+            reach[c] = a || b;
+            edge_a[c] += a; edge_b[c] += b;
+        }
+        for (int s = 0; s < S; s++) {
+            if (!reach[s]) continue;
             e->visits[s]++;
             int taken = 0;
             for (int side = 0; side < 2; side++) {
                 const int c = side == 0 ? bp.child_a[s] : bp.child_b[s];
                 if (c < 0) continue;
                 const int bit = side == 0 ? bp.cbit_a[s] : bp.cbit_b[s];
-                const int val = side == 0 ? bp.cval_a[s] : bp.cval_b[s];
-                if (bit < 0 || ((tr->branch_bits[q] >> bit) & 1) == val) { stack[top++] = c; taken++; }
+                const unsigned val = side == 0 ? bp.cval_a[s] : bp.cval_b[s];
+                taken += (bit < 0 || ((bits >> bit) & 1u) == val);
             }
             if (taken == 0) bp.total_leaving++;
         }
     }
     e->events_per_candidate = 0;
     for (int s = 0; s < S; s++) e->events_per_candidate += e->visits[s];
-    e->slot_elems = std::max<int64_t>(32, plan_stream_buffers(pr, e->visits, bp.buf_off));
+    if (!e->join) {
+        e->slot_elems = std::max<int64_t>(32, plan_stream_buffers(pr, e->visits, bp.buf_off));
+    } else {
+        // joins: every stream gets memory of its own (arrival stream per stage, the two incoming streams of
+        // a join), then the scratch of the merge: its two halves and the per-query input times
+        auto pad = [](int64_t v) { return (v + 31) / 32 * 32; };
+        int64_t off = 0, tmp = 0;
+        bp.buf_off[0] = 0;
+        for (int c = 1; c < S; c++) {
+            bp.buf_off[c] = (int32_t)std::min<int64_t>(off, INT32_MAX); off += pad(e->visits[c]);
+            if (bp.join_b[c] < 0) continue;
+            bp.join_in_a[c] = (int32_t)std::min<int64_t>(off, INT32_MAX); off += pad(edge_a[c]);
+            bp.join_in_b[c] = (int32_t)std::min<int64_t>(off, INT32_MAX); off += pad(edge_b[c]);
+            bp.join_na[c] = (int32_t)edge_a[c]; bp.join_nb[c] = (int32_t)edge_b[c];
+            tmp = std::max(tmp, pad(edge_a[c]) + pad(edge_b[c]));
+        }
+        bp.join_tmp_off = (int32_t)std::min<int64_t>(off, INT32_MAX); off += tmp;
+        bp.join_t_off = (int32_t)std::min<int64_t>(off, INT32_MAX); off += 2 * e->n_pad;
+        if (off > INT32_MAX) { delete e; return IL_ERR_TOO_LARGE; }
+        e->slot_elems = std::max<int64_t>(32, off);
+    }
+    // where each stage writes the records of its two outgoing edges (kernel with separate streams)
+    for (int s = 0; s < S; s++) {
+        for (int side = 0; side < 2; side++) {
+            const int c = side == 0 ? bp.child_a[s] : bp.child_b[s];
+            int32_t at = 0;
+            if (c >= 0) at = bp.join_b[c] < 0 ? bp.buf_off[c] : (bp.join_b[c] == s ? bp.join_in_b[c] : bp.join_in_a[c]);
+            (side == 0 ? bp.out_off_a : bp.out_off_b)[s] = at;
+        }
+    }
     for (int s = 0; s < S; s++) bp.n_s[s] = (int32_t)e->visits[s];
     // lane kernel: every stage but the root reads its arrival stream from a ring
     e->cpw = 32 / S;
@@ -796,7 +862,7 @@ int il_estimator_create(const il_profiles *pr, const il_trace *tr, il_estimator 
     IL_CUDA_E(cudaMalloc(&e->d_arrival, (size_t)n * 8));
     IL_CUDA_E(cudaMalloc(&e->d_bits, (size_t)n));
     e->can_pack = can_pack;
-    e->lane_ok = can_pack && e->lane_elems < (INT64_C(1) << 31);   // (with fan-out the streams are kept whole)
+    e->lane_ok = can_pack && !e->join && e->lane_elems < (INT64_C(1) << 31);   // (with fan-out the streams are kept whole)
     bp.qbits = qbits;
     if (can_pack) {
         // padded with "never" records to whole tiles, so that bulk copies always move full tiles

@@ -45,6 +45,17 @@ struct DesParams {
     int8_t  cbit_a[IL_MAX_STAGES], cbit_b[IL_MAX_STAGES];     // branch bit guarding the edge, -1 = always taken
     uint8_t cval_a[IL_MAX_STAGES], cval_b[IL_MAX_STAGES];     // the edge is taken iff the bit has this value
     int64_t total_leaving;           // copies that leave the pipeline, all stages together (n without fan-out)
+    int32_t out_off_a[IL_MAX_STAGES], out_off_b[IL_MAX_STAGES];   // fan-out, separate streams: where stage s writes
+                                     // the records for child_a / child_b inside a warp slot
+    // Joins (kernel with separate streams only): stage s with join_b[s] >= 0 has two incoming edges.  Its
+    // parents write to in_a[s] (edge parent -> s, na[s] records) and in_b[s] (edge join_b[s] -> s, nb[s]
+    // records); before the stage is simulated the warp merges them into the stage's arrival stream at
+    // buf_off[s], one record per query at the time its last input arrived.
+    int8_t  join_b[IL_MAX_STAGES];   // second parent, -1 = none
+    int32_t join_in_a[IL_MAX_STAGES], join_in_b[IL_MAX_STAGES];
+    int32_t join_na[IL_MAX_STAGES], join_nb[IL_MAX_STAGES];
+    int32_t join_tmp_off;            // scratch for the two sorted halves of a merge
+    int32_t join_t_off;              // scratch: per query the times of its two inputs, 2 x n_pad elements
     // this launch
     const il_stage_config *configs;  // [n_cand][S], already offset to the chunk
     int64_t n_cand;

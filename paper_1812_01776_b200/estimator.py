@@ -33,7 +33,7 @@ EXPORTS = ["il_estimator_create", "il_estimator_destroy", "il_estimate", "il_est
            "il_set_stream", "il_workspace_bytes", "il_workspace_min_bytes", "il_set_workspace",
            "il_get_stats", "il_stage_visits", "il_strerror", "il_last_cuda_error",
            "il_measure_int_issue", "il_estimate_device_static", "il_set_variant", "il_estimate_latencies", "il_traffic_envelope", "il_kernel_name",
-           "il_set_test_knob", "il_feasible", "il_feasible_device"]
+           "il_set_test_knob", "il_feasible", "il_feasible_device", "il_estimator_create_dag"]
 
 
 class ILError(RuntimeError):
@@ -51,6 +51,10 @@ class _Profiles(ctypes.Structure):
                 ("max_batch", ctypes.c_int32), ("parent", ctypes.c_void_p),
                 ("cond_bit", ctypes.c_void_p), ("cond_val", ctypes.c_void_p),
                 ("latency_us", ctypes.c_void_p)]
+
+
+class _JoinEdges(ctypes.Structure):
+    _fields_ = [("parent2", ctypes.c_void_p), ("cond_bit2", ctypes.c_void_p), ("cond_val2", ctypes.c_void_p)]
 
 
 class _Trace(ctypes.Structure):
@@ -93,6 +97,9 @@ def load_library():
     lib.il_estimator_create.restype = ctypes.c_int
     lib.il_estimator_create.argtypes = [ctypes.POINTER(_Profiles), ctypes.POINTER(_Trace),
                                         ctypes.POINTER(vp)]
+    lib.il_estimator_create_dag.restype = ctypes.c_int
+    lib.il_estimator_create_dag.argtypes = [ctypes.POINTER(_Profiles), ctypes.POINTER(_JoinEdges),
+                                            ctypes.POINTER(_Trace), ctypes.POINTER(vp)]
     lib.il_estimator_destroy.restype = None
     lib.il_estimator_destroy.argtypes = [vp]
     lib.il_estimate.restype = ctypes.c_int
@@ -149,7 +156,15 @@ def il_strerror(code: int) -> str:
 
 # ---- one-to-one wrappers (host numpy arrays / raw device pointers) ----------
 
-def il_estimator_create(parent, cond_bit, cond_val, latency_us, arrival_us, branch_bits=None):
+def il_estimator_create_dag(parent, cond_bit, cond_val, latency_us, arrival_us, branch_bits=None, join=None):
+    """il_estimator_create_dag: as il_estimator_create, with join = (parent2, cond_bit2, cond_val2),
+    per stage the second incoming edge (parent2[s] = -1: none), or None."""
+    return il_estimator_create(parent, cond_bit, cond_val, latency_us, arrival_us, branch_bits, _join=join,
+                               _dag=True)
+
+
+def il_estimator_create(parent, cond_bit, cond_val, latency_us, arrival_us, branch_bits=None, _join=None,
+                        _dag=False):
     """il_estimator_create: host arrays in, opaque handle out."""
     lib = load_library()
     parent = np.ascontiguousarray(parent, dtype=np.int32)
@@ -171,6 +186,18 @@ def il_estimator_create(parent, cond_bit, cond_val, latency_us, arrival_us, bran
     tr = _Trace(arrival_us.shape[0], arrival_us.ctypes.data,
                 None if branch_bits is None else branch_bits.ctypes.data)
     handle = ctypes.c_void_p()
+    if _dag:
+        jn = None
+        if _join is not None:
+            parent2 = np.ascontiguousarray(_join[0], dtype=np.int32)
+            cond_bit2 = np.ascontiguousarray(_join[1], dtype=np.int8)
+            cond_val2 = np.ascontiguousarray(_join[2], dtype=np.uint8)
+            if parent2.shape != (S,) or cond_bit2.shape != (S,) or cond_val2.shape != (S,):
+                raise ValueError("the join arrays must have one entry per stage")
+            jn = ctypes.byref(_JoinEdges(parent2.ctypes.data, cond_bit2.ctypes.data, cond_val2.ctypes.data))
+        _check(lib.il_estimator_create_dag(ctypes.byref(pr), jn, ctypes.byref(tr), ctypes.byref(handle)),
+               "il_estimator_create_dag")
+        return handle
     _check(lib.il_estimator_create(ctypes.byref(pr), ctypes.byref(tr), ctypes.byref(handle)),
            "il_estimator_create")
     return handle
@@ -307,7 +334,7 @@ class Estimator:
     """
 
     def __init__(self, parent, cond_bit, cond_val, latency_us, arrival_us, branch_bits=None,
-                 device: Optional[int] = None):
+                 device: Optional[int] = None, join=None):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("the Estimator needs a CUDA device (sm_100a); there is no CPU path")
@@ -316,15 +343,19 @@ class Estimator:
         self.n_stages = int(np.asarray(latency_us).shape[0])
         self.n_queries = int(np.asarray(arrival_us).shape[0])
         with torch.cuda.device(self.device):
-            self._h = il_estimator_create(parent, cond_bit, cond_val, latency_us, arrival_us,
-                                          branch_bits)
+            if join is None:
+                self._h = il_estimator_create(parent, cond_bit, cond_val, latency_us, arrival_us,
+                                              branch_bits)
+            else:
+                self._h = il_estimator_create_dag(parent, cond_bit, cond_val, latency_us, arrival_us,
+                                                  branch_bits, join=join)
         self._ws = None
         self.visits = il_stage_visits(self._h, self.n_stages)
 
     @classmethod
     def from_workload(cls, w, device: Optional[int] = None) -> "Estimator":
         return cls(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us, w.branch_bits,
-                   device=device)
+                   device=device, join=getattr(w, "join", None))
 
     def close(self) -> None:
         if getattr(self, "_h", None):

@@ -48,6 +48,27 @@ def test_strerror_covers_codes(lib):
     assert lib.il_strerror(-99).decode() == "unknown error"
 
 
+def test_create_dag_rejects_bad_joins_on_the_host(lib):
+    """A second incoming edge must come from a stage above the first parent and below the stage itself,
+    and a stage keeps at most two outgoing edges; checked before any CUDA call."""
+    from paper_1812_01776_b200 import estimator as E
+    import workloads
+    w = workloads.join_small(1, n=32)
+    for p2 in ([-1, -1, -1, 1], [-1, -1, -1, 3], [-1, -1, -1, 0], [0, -1, -1, 2]):
+        with pytest.raises(E.ILError) as e:
+            E.il_estimator_create_dag(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us, w.branch_bits,
+                                      join=(p2, w.join[1], w.join[2]))
+        assert e.value.code == E.IL_ERR_BAD_TOPOLOGY
+    with pytest.raises(E.ILError) as e:                     # stage 0 would have three outgoing edges
+        E.il_estimator_create_dag(np.array([-1, 0, 0, 0], np.int32), w.cond_bit, w.cond_val, w.latency_us,
+                                  w.arrival_us, w.branch_bits, join=w.join)
+    assert e.value.code == E.IL_ERR_BAD_TOPOLOGY
+    with pytest.raises(E.ILError) as e:                     # no such branch bit on the second edge
+        E.il_estimator_create_dag(w.parent, w.cond_bit, w.cond_val, w.latency_us, w.arrival_us, w.branch_bits,
+                                  join=(w.join[0], np.array([-1, -1, -1, 8], np.int8), w.join[2]))
+    assert e.value.code == E.IL_ERR_BAD_TOPOLOGY
+
+
 def test_create_rejects_bad_arguments_on_the_host(lib):
     """Validation comes before any CUDA call, so these run without a device."""
     from paper_1812_01776_b200 import estimator as E

@@ -31,8 +31,8 @@ def test_parity_slice_on_the_checked_build():
                            cwd=ROOT, env=env, capture_output=True, text=True)
     assert "libil_estimator_checked.so" in probe.stdout, probe.stdout + probe.stderr
     run = subprocess.run([sys.executable, "-m", "pytest", "tests/test_gpu_parity.py", "tests/test_shared_prefix.py",
-                          "tests/test_feasible.py", "-m", "gpu", "-x", "-q", "-k",
+                          "tests/test_feasible.py", "tests/test_join.py", "-m", "gpu", "-x", "-q", "-k",
                           "random_small or deep_pipelines or edge_cases or short_stream_rings or forced_sharing "
-                          "or feasible_random_small or largest_table"],
+                          "or feasible_random_small or largest_table or join_parity or join_equal_instants"],
                          cwd=ROOT, env=env, capture_output=True, text=True)
     assert run.returncode == 0, run.stdout[-3000:] + run.stderr[-2000:]

@@ -60,9 +60,12 @@ def _hand_cases():
 @pytest.mark.parametrize("case", _hand_cases(), ids=lambda c: c["name"])
 def test_hand_traces(il, case):
     bits = np.array(case["branch_bits"], np.uint8) if "branch_bits" in case else None
+    join = None
+    if "join" in case:
+        join = (case["join"]["parent2"], case["join"]["cond_bit2"], case["join"]["cond_val2"])
     with il.Estimator(np.array(case["parent"], np.int32), np.array(case["cond_bit"], np.int8),
                       np.array(case["cond_val"], np.uint8), np.array(case["latency_us"], np.int32),
-                      np.array(case["arrival_us"], np.int64), bits) as est:
+                      np.array(case["arrival_us"], np.int64), bits, join=join) as est:
         p99, miss = est.estimate(np.array([case["config"]], np.uint8), case["slo_us"])
     assert (int(p99[0]), int(miss[0])) == (case["p99_us"], case["miss"])
 
