@@ -25,8 +25,9 @@
  *
  * Readings taken where the paper is silent (each is pinned by a test):
  *   - Everything that happens at one timestamp happens in three phases: all
- *     completions (in the order their batches were dispatched), then all
- *     external arrivals (in trace order), then dispatching, stage by stage.
+ *     completions (stage by stage, within a stage in the order their batches
+ *     were dispatched), then all external arrivals (in trace order), then
+ *     dispatching, stage by stage.
  *   - An idle replica with a non-empty queue takes min(queue length, max
  *     batch) queries from the front of the FIFO queue at once; the lowest-id
  *     idle replica goes first.
@@ -264,7 +265,7 @@ int orc_estimate_one_dag(int32_t S, int32_t H, int32_t Bmax,
     while (heap.size > 0) {
         const int64_t clock = heap.e[0].time;
 
-        /* phase 1: every completion at this instant, earliest-dispatched batch first */
+        /* phase 1: every completion at this instant: by stage, then earliest-dispatched batch first */
         while (heap.size > 0 && heap.e[0].time == clock && heap.e[0].kind == EV_COMPLETION) {
             event_t ev = heap_pop(&heap);
             int s = ev.stage, r = ev.replica;
