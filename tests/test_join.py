@@ -8,7 +8,7 @@ import workloads
 
 pytestmark = pytest.mark.gpu
 
-SHAPES = ["diamond", "guarded", "two_joins"]
+SHAPES = ["diamond", "guarded", "two_joins", "skip"]
 
 
 @pytest.fixture(scope="module")
@@ -52,6 +52,27 @@ def test_join_equal_instants(il, oracle, shape):
                                                 w.branch_bits, w.configs[c], w.slo_us, want_latency=True,
                                                 join=w.join)
                 assert np.array_equal(est.latencies(w.configs[c]), lat), (seed, c)
+
+
+def test_join_edges_nobody_follows(il, oracle):
+    """A join one of whose incoming streams is empty (no query has the bit that opens the edge), and one
+    that no query reaches at all."""
+    w = workloads.join_small(8, n=800, C=12, shape="guarded")
+    w.branch_bits[:] &= 0xFE                       # nobody visits stage 2: the join has one input
+    exp = oracle.estimate_workload(w)
+    with il.Estimator.from_workload(w) as est:
+        assert est.visits.tolist() == [800, 800, 0, 800, 800]
+        p99, miss = est.estimate(w.configs, w.slo_us)
+        assert np.array_equal(p99, exp[0]) and np.array_equal(miss, exp[1])
+    w = workloads.join_small(8, n=800, C=12, shape="two_joins")
+    w.cond_bit = np.array([-1, 0, 0, -1, 1, -1], np.int8)      # bit 0 decides between 1 and 2 ...
+    w.cond_val = np.array([0, 0, 1, 0, 1, 0], np.uint8)
+    w.branch_bits[:] |= 1                          # ... and everyone takes 2: stages 1 and 4 stay empty
+    exp = oracle.estimate_workload(w)
+    with il.Estimator.from_workload(w) as est:
+        assert est.visits.tolist() == [800, 0, 800, 800, 0, 800]
+        p99, miss = est.estimate(w.configs, w.slo_us)
+        assert np.array_equal(p99, exp[0]) and np.array_equal(miss, exp[1])
 
 
 def test_join_hand_trace_and_visits(il):

@@ -593,7 +593,7 @@ def _one(oracle, w, cfg, **kw):
                                cfg, 0, want_latency=True, join=w.join, **kw)[2]
 
 
-@pytest.mark.parametrize("shape", ["diamond", "guarded", "two_joins"])
+@pytest.mark.parametrize("shape", ["diamond", "guarded", "two_joins", "skip"])
 @pytest.mark.parametrize("seed", range(8))
 def test_join_tick_brute_force(oracle, seed, shape):
     w = workloads.join_small(seed, n=40, C=6, max_replicas=3, Bmax=4, tiny_times=True, shape=shape)

@@ -339,8 +339,9 @@ def join_small(seed: int, n: int = 900, C: int = 30, max_replicas: int = 4, Bmax
     guarded     0 -> {1, 2 if bit 0 is 1}; 3 joins 1 and 2; 3 -> 4.  A query with bit 0 clear reaches 3
                 through stage 1 alone.
     two_joins   0 -> {1, 2}; 3 joins 1 and 2; 1 is a fork as well: 1 -> {3, 4 if bit 1 is 1}; 5 joins 3 and 4
-                (the second edge, 4 -> 5, only exists for queries that visited 4)."""
-    S = {"diamond": 4, "guarded": 5, "two_joins": 6}[shape]
+                (the second edge, 4 -> 5, only exists for queries that visited 4).
+    skip        0 -> 1 -> 2 with a skip connection 0 -> 2 (guarded by bit 1): stage 2 joins 0 and 1; 2 -> 3."""
+    S = {"diamond": 4, "guarded": 5, "two_joins": 6, "skip": 4}[shape]
     w = random_small(seed, S=S, H=2, Bmax=Bmax, n=n, C=C, max_replicas=max_replicas, tree=False,
                      qps=80_000.0 if tiny_times else 300.0, cv=2.0, lat_lo=1,
                      lat_hi=30 if tiny_times else 9000, equal_stamp_every=(3 if seed % 2 == 0 else 0))
@@ -354,6 +355,11 @@ def join_small(seed: int, n: int = 900, C: int = 30, max_replicas: int = 4, Bmax
         w.cond_bit = np.array([-1, -1, 0, -1, -1], np.int8)
         w.cond_val = np.array([0, 0, 1, 0, 0], np.uint8)
         w.join = (np.array([-1, -1, -1, 2, -1], np.int32), np.full(5, -1, np.int8), np.zeros(5, np.uint8))
+    elif shape == "skip":
+        w.parent = np.array([-1, 0, 0, 2], np.int32)
+        w.cond_bit = np.array([-1, -1, 1, -1], np.int8)
+        w.cond_val = np.array([0, 0, 1, 0], np.uint8)
+        w.join = (np.array([-1, -1, 1, -1], np.int32), np.full(4, -1, np.int8), np.zeros(4, np.uint8))
     else:
         w.parent = np.array([-1, 0, 0, 1, 1, 3], np.int32)
         w.cond_bit = np.array([-1, -1, -1, -1, 1, -1], np.int8)
