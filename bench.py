@@ -345,7 +345,8 @@ def measure(il, torch, w, dev, stream, flush, steps, warmup, e2e_steps, variant,
     n, S = w.n_queries, w.n_stages
     shared = bool(st.get("stage_runs")) and st["stage_runs"] < n_cand * S
     if shared:
-        kernel = "des_node_stage_kernel (shared configuration prefixes: every distinct stage run simulated once)"
+        kernel = ("shared configuration prefixes: a covering set of whole candidates on des_lane_kernel "
+                  "(des_node_stage_kernel, node by node, where that does not apply)")
     sim_s = statistics.mean(sim_ms) * 1e-3
     sel_s = statistics.mean(sel_ms) * 1e-3
     total_events = events_per_cand * n_cand
@@ -359,13 +360,13 @@ def measure(il, torch, w, dev, stream, flush, steps, warmup, e2e_steps, variant,
     hbm_note = ("latency slab written once + every inter-stage stream record written once "
                 "and read once (the streams are this design's, not the method's)")
     if shared:
-        # only the distinct stage runs move data: per run its arrival stream read and its output written
+        # only the simulated stage runs move data: per run its arrival stream read and its output written
         # (about 16 B per simulated query-event); the method's own count does not apply
         simulated_events = total_events * st["stage_runs"] / float(n_cand * S)
         stream_bytes = 16.0 * simulated_events
         slab_bytes = 0
         hbm_note = ("shared prefixes: about 16 B per SIMULATED query-event (stage_runs_simulated / "
-                    "stage_runs_of_the_method of the method's count), no slab")
+                    "stage_runs_of_the_method of the method's count)")
     rec = {
         "candidates": n_cand, "queries": n, "stages": S, "query_events_per_candidate": events_per_cand,
         "kernel": kernel, "workspace_bytes": ws_bytes, "steps": steps, "warmup": warmup,

@@ -233,10 +233,11 @@ IL_API int il_estimate(il_estimator *est, const il_stage_config *configs, int64_
  * 16,384 and enough workspace, the call first builds the set of distinct (stage,
  * configuration, parent) nodes on the device; if there are at most a quarter as
  * many nodes as candidates x stages (an exhaustive sweep over per-stage choices,
- * not a uniform random draw) it simulates every node once and assembles each
- * candidate's P99 and miss count from the nodes where its queries leave.  Results
- * are the same integers; il_stats.stage_runs tells how many stage simulations
- * were carried out.
+ * not a uniform random draw) it simulates the nodes instead of the candidates --
+ * through a small set of whole candidates that between them contain every node
+ * queries leave after, or node by node -- and assembles each candidate's P99 and
+ * miss count from the nodes where its queries leave.  Results are the same
+ * integers; il_stats.stage_runs tells how many stage simulations were carried out.
  */
 IL_API int il_estimate_device(il_estimator *est, const il_stage_config *d_configs, int64_t n,
                               int64_t slo_us, int64_t *d_out_p99_us, int64_t *d_out_miss);
@@ -415,7 +416,9 @@ IL_API int il_set_variant(il_estimator *est, int variant);
  *                           return IL_ERR_ITER_LIMIT; the handle stays usable.
  *   IL_KNOB_SHARE_PREFIXES  0: the library decides per call whether to evaluate a batch through shared
  *                           configuration prefixes (see il_estimate_device); 1: always, when the
- *                           preconditions hold; 2: never.
+ *                           preconditions hold; 2: never; 3: always, and the distinct stage runs are
+ *                           simulated one by one even where a covering set of whole candidates on
+ *                           the lane kernel would do.
  *   IL_KNOB_LANE_CTAS       value 0..16: resident CTAs (of two warps) per SM of the lane kernel; 0 restores
  *                           the library's choice (4).  For measurements.
  * Set a knob before il_workspace_bytes / il_set_workspace: sizes depend on the ring length.

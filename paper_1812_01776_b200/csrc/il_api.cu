@@ -52,7 +52,7 @@ struct il_estimator {
     int lane_ring_cap_log2 = 0;        // test knob: force rings of at most 2^this records (0: the library's choice)
     bool lane_wrap = false;            // the rings are shorter than the longest stream
     unsigned long long iter_limit = 0; // test knob: iteration bound of the device loops (0 = their own)
-    int share_mode = 0;                // shared-prefix evaluation: 0 when it pays, 1 always (tests), 2 never
+    int share_mode = 0;                // shared-prefix evaluation: 0 when it pays, 1 always (tests), 2 never, 3 always and node by node
     int32_t parent[IL_MAX_STAGES] = {};
     int cpw = 1;                       // lane kernel: candidates per warp
     size_t smem_lane[2] = {0, 0};       // lane kernel with 16 / 32 batch ring positions per lane
@@ -515,6 +515,137 @@ static void slab_regions(const il_estimator *e, SelectParams &sp)
 }
 
 
+// End of a shared-prefix call: events[0], events[1] and the work in between are on the stream.
+static int finish_shared(il_estimator *e, int64_t n_cand, int64_t launches, int64_t stage_runs)
+{
+    cudaStream_t st = e->stream;
+    IL_CUDA(cudaEventRecord(e->events[2], st));
+    IL_CUDA(cudaMemcpyAsync(e->h_counters, e->d_counters, kCounters * sizeof(unsigned long long),
+                            cudaMemcpyDeviceToHost, st));
+    IL_CUDA(cudaMemcpyAsync(e->h_status, e->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+    IL_CUDA(cudaStreamSynchronize(st));
+    float ms = 0.f;
+    IL_CUDA(cudaEventElapsedTime(&ms, e->events[0], e->events[1]));
+    e->stats.sim_ms = ms;
+    IL_CUDA(cudaEventElapsedTime(&ms, e->events[1], e->events[2]));
+    e->stats.select_ms = ms;
+    e->stats.total_ms = e->stats.sim_ms + e->stats.select_ms;
+    e->stats.candidates = n_cand;
+    e->stats.query_events = n_cand * e->events_per_candidate;
+    e->stats.batches = (int64_t)e->h_counters[1];
+    e->stats.algorithmic_ops = (int64_t)e->h_counters[2];
+    e->stats.chunks = 1;
+    e->stats.kernel_launches = launches;
+    e->stats.error_detail = (int64_t)e->h_counters[5];
+    e->stats.stage_runs = stage_runs;
+    return *e->h_status;
+}
+
+// Shared-prefix evaluation, simulation by the lane kernel.  The nodes that queries leave after are
+// covered by a set of whole candidates of the batch (per node the candidate with the smallest index
+// that contains it); those are simulated like any batch, and a node's leaving records are the region
+// of its stage in the slab row of its candidate.  Candidates of the set repeat the work of the
+// prefixes they share, but they run on the kernel that is an order of magnitude faster per stage run
+// than the node-by-node one, and all at once instead of level by level.  Needs whole streams (no
+// rings, so that every row has the region layout) and room for all rows in one chunk; *done stays
+// false when that is not so, and the caller simulates the nodes one by one.
+// On entry `off` bytes of the workspace are in use; events[0] has been recorded.
+struct SharedCommon {
+    const il_stage_config *d_configs;
+    int64_t n_cand, slo_us, allowed, top_len;
+    int64_t *d_out_p99, *d_out_miss;
+    const int32_t *node_of;
+    const int *h_count;
+    const int64_t *leaving;
+};
+
+static int shared_by_cover(il_estimator *e, const SharedCommon &c, char *ws, size_t ws_bytes, size_t off,
+                           int64_t *launches, int64_t *stage_runs, bool *done)
+{
+    *done = false;
+    if (e->share_mode == 3 || !is_lane(e) || e->lane_wrap) return IL_OK;
+    const int S = e->S;
+    const int64_t n_cand = c.n_cand;
+    auto take = [&](size_t bytes) { const size_t at = off; off = align_up(off + bytes, 256); return at; };
+    int64_t exit_nodes = 0;
+    size_t o_rep[IL_MAX_STAGES] = {}, o_row[IL_MAX_STAGES] = {}, o_top[IL_MAX_STAGES] = {}, o_miss[IL_MAX_STAGES] = {};
+    for (int s = 0; s < S; s++) {
+        if (c.leaving[s] <= 0) continue;
+        exit_nodes += c.h_count[s];
+        o_rep[s] = take((size_t)c.h_count[s] * 4); o_row[s] = take((size_t)c.h_count[s] * 4);
+        o_top[s] = take((size_t)c.h_count[s] * c.top_len * 8); o_miss[s] = take((size_t)c.h_count[s] * 8);
+    }
+    const int64_t most = std::min(n_cand, exit_nodes);
+    const size_t o_flags = take((size_t)n_cand), o_pos = take((size_t)n_cand * 4), o_list = take((size_t)most * 4);
+    const size_t o_cnt = take(4), o_cfg = take((size_t)most * S * sizeof(il_stage_config));
+    if (off > ws_bytes) return IL_OK;
+    Plan pl;
+    if (!make_plan(e, ws_bytes - off, most, pl) || pl.chunk < most) return IL_OK;   // all rows must be there at once
+
+    cudaStream_t st = e->stream;
+    uint8_t *flags = reinterpret_cast<uint8_t *>(ws + o_flags);
+    int32_t *pos = reinterpret_cast<int32_t *>(ws + o_pos), *list = reinterpret_cast<int32_t *>(ws + o_list);
+    int *d_cnt = reinterpret_cast<int *>(ws + o_cnt);
+    il_stage_config *cfg = reinterpret_cast<il_stage_config *>(ws + o_cfg);
+    IL_CUDA(cudaMemsetAsync(flags, 0, (size_t)n_cand, st));
+    IL_CUDA(cudaMemsetAsync(d_cnt, 0, 4, st));
+    for (int s = 0; s < S; s++)
+        if (c.leaving[s] > 0) {
+            IL_CUDA(launch_cover_rep(c.node_of + (size_t)s * n_cand, n_cand, reinterpret_cast<int32_t *>(ws + o_rep[s]),
+                                     c.h_count[s], flags, st));
+            *launches += 2;
+        }
+    IL_CUDA(launch_cover_list(flags, n_cand, list, pos, d_cnt, st));
+    for (int s = 0; s < S; s++)
+        if (c.leaving[s] > 0) {
+            IL_CUDA(launch_cover_rows(reinterpret_cast<int32_t *>(ws + o_rep[s]), pos, c.h_count[s],
+                                      reinterpret_cast<int32_t *>(ws + o_row[s]), st));
+            (*launches)++;
+        }
+    int m = 0;
+    IL_CUDA(cudaMemcpyAsync(&m, d_cnt, 4, cudaMemcpyDeviceToHost, st));
+    IL_CUDA(cudaStreamSynchronize(st));
+    if (m < 1 || m > most) return IL_ERR_ITER_LIMIT;      // cannot happen: every node has a candidate
+    IL_CUDA(launch_gather_configs(c.d_configs, list, m, S, cfg, st));
+    *launches += 2;
+    *done = true;
+
+    char *sim_ws = ws + off;
+    DesParams p = chunk_params(e, pl, sim_ws, cfg, m);
+    const int64_t wpc = warps_per_cta(e);
+    const int64_t groups = (m + cands_per_slot(e) - 1) / cands_per_slot(e);
+    const int64_t ctas = std::min<int64_t>(pl.slots / wpc, (groups + wpc - 1) / wpc);
+    int rc = enqueue_simulation(e, p, pl, sim_ws, ctas, st, launches);
+    if (rc) return rc;
+    IL_CUDA(cudaEventRecord(e->events[1], st));
+
+    CombineParams cp = {};
+    cp.n_cand = n_cand; cp.node_of = c.node_of; cp.top_len = (int32_t)c.top_len; cp.allowed = c.allowed;
+    cp.out_p99 = c.d_out_p99; cp.out_miss = c.d_out_miss;
+    int64_t region = 0;
+    for (int s = 0; s < S; s++) {
+        if (c.leaving[s] <= 0) continue;
+        NodeTopParams tp = {};
+        tp.records = reinterpret_cast<uint64_t *>(p.slab);
+        tp.stride = e->n_pad; tp.len = (int32_t)c.leaving[s];
+        tp.row_of = reinterpret_cast<int32_t *>(ws + o_row[s]);
+        tp.offset = region;
+        tp.arrival = e->d_arrival; tp.qbits = e->base.qbits; tp.slo_us = c.slo_us;
+        tp.top_len = (int32_t)c.top_len;
+        tp.top = reinterpret_cast<int64_t *>(ws + o_top[s]);
+        tp.miss = reinterpret_cast<int64_t *>(ws + o_miss[s]);
+        tp.n_nodes = c.h_count[s];
+        IL_CUDA(launch_node_top(tp, st));
+        (*launches)++;
+        cp.exit_stage[cp.n_exit] = s; cp.top[cp.n_exit] = tp.top; cp.miss[cp.n_exit] = tp.miss; cp.n_exit++;
+        region += c.leaving[s];
+    }
+    IL_CUDA(launch_prefix_combine(cp, st));
+    (*launches)++;
+    *stage_runs = (int64_t)m * S;
+    return IL_OK;
+}
+
 // ---- shared-prefix evaluation -------------------------------------------------------------------
 // Candidates that agree on the configurations of all stages on a path from the root have the same
 // completion stream at the end of that path; the batch is turned into the set of distinct (stage,
@@ -577,15 +708,29 @@ static int estimate_shared(il_estimator *e, const il_stage_config *d_configs, in
     e->setup_launches += 3 * S;
     if (e->share_mode == 0 && total_nodes * 4 > n_cand * S) return IL_OK;
 
-    // streams between the nodes, leaving records, top lists and miss counts
     int64_t leaving[IL_MAX_STAGES], stride_in[IL_MAX_STAGES], stride_ex[IL_MAX_STAGES];
-    size_t o_in[IL_MAX_STAGES] = {}, o_ex[IL_MAX_STAGES] = {}, o_top[IL_MAX_STAGES] = {}, o_miss[IL_MAX_STAGES] = {};
     for (int s = 0; s < S; s++) {
         const int a = e->base.dest_a[s], b = e->base.dest_b[s];
         int64_t kids = 0;
         if (a >= 0) kids += e->visits[a];
         if (b >= 0 && b != a) kids += e->visits[b];
         leaving[s] = e->visits[s] - kids;
+    }
+    int64_t launches = e->setup_launches, stage_runs = total_nodes;
+    {
+        // the fast way first: the nodes covered by whole candidates on the lane kernel
+        SharedCommon sc = {d_configs, n_cand, slo_us, allowed, top_len, d_out_p99, d_out_miss, node_of, h_count, leaving};
+        bool done = false;
+        rc = shared_by_cover(e, sc, ws, ws_bytes, off, &launches, &stage_runs, &done);
+        if (rc) { *used = true; return rc; }
+        if (done) {
+            *used = true;
+            return finish_shared(e, n_cand, launches, stage_runs);
+        }
+    }
+    // streams between the nodes, leaving records, top lists and miss counts
+    size_t o_in[IL_MAX_STAGES] = {}, o_ex[IL_MAX_STAGES] = {}, o_top[IL_MAX_STAGES] = {}, o_miss[IL_MAX_STAGES] = {};
+    for (int s = 0; s < S; s++) {
         stride_in[s] = (e->visits[s] + 3) / 4 * 4;
         stride_ex[s] = (leaving[s] + 3) / 4 * 4;
         if (s > 0 && e->visits[s] > 0)
@@ -599,7 +744,6 @@ static int estimate_shared(il_estimator *e, const il_stage_config *d_configs, in
     if (off > ws_bytes) return IL_OK;
     *used = true;
 
-    int64_t launches = e->setup_launches;
     for (int s = 0; s < S; s++) {
         if (e->visits[s] == 0) continue;
         const int a = e->base.dest_a[s], b = e->base.dest_b[s];
@@ -651,26 +795,7 @@ static int estimate_shared(il_estimator *e, const il_stage_config *d_configs, in
     }
     IL_CUDA(launch_prefix_combine(cp, st));
     launches++;
-    IL_CUDA(cudaEventRecord(e->events[2], st));
-    IL_CUDA(cudaMemcpyAsync(e->h_counters, e->d_counters, kCounters * sizeof(unsigned long long),
-                            cudaMemcpyDeviceToHost, st));
-    IL_CUDA(cudaMemcpyAsync(e->h_status, e->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
-    IL_CUDA(cudaStreamSynchronize(st));
-    float ms = 0.f;
-    IL_CUDA(cudaEventElapsedTime(&ms, e->events[0], e->events[1]));
-    e->stats.sim_ms = ms;
-    IL_CUDA(cudaEventElapsedTime(&ms, e->events[1], e->events[2]));
-    e->stats.select_ms = ms;
-    e->stats.total_ms = e->stats.sim_ms + e->stats.select_ms;
-    e->stats.candidates = n_cand;
-    e->stats.query_events = n_cand * e->events_per_candidate;
-    e->stats.batches = (int64_t)e->h_counters[1];
-    e->stats.algorithmic_ops = (int64_t)e->h_counters[2];
-    e->stats.chunks = 1;
-    e->stats.kernel_launches = launches;
-    e->stats.error_detail = (int64_t)e->h_counters[5];
-    e->stats.stage_runs = total_nodes;
-    return *e->h_status;
+    return finish_shared(e, n_cand, launches, stage_runs);
 }
 
 extern "C" {
@@ -942,7 +1067,7 @@ int il_set_test_knob(il_estimator *e, int knob, int64_t value)
         return IL_OK;
     }
     if (knob == IL_KNOB_SHARE_PREFIXES) {
-        if (value < 0 || value > 2) return IL_ERR_INVALID_ARG;
+        if (value < 0 || value > 3) return IL_ERR_INVALID_ARG;
         e->share_mode = (int)value;
         return IL_OK;
     }
@@ -1216,7 +1341,7 @@ int il_feasible_device(il_estimator *e, const il_stage_config *d_configs, int64_
     size_t ws_bytes = 0;
     rc = acquire_workspace(e, std::min<int64_t>(n_cand, 4096), &ws, &ws_bytes);
     if (rc) return rc;
-    if (e->share_mode == 1 || (e->share_mode == 0 && n_cand >= kShareMinCandidates)) {
+    if (e->share_mode == 1 || e->share_mode == 3 || (e->share_mode == 0 && n_cand >= kShareMinCandidates)) {
         // a batch full of common configuration prefixes is cheaper to evaluate node by node
         rc = ensure_staging(e, n_cand);
         if (rc) return rc;

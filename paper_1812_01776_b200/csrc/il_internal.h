@@ -177,8 +177,10 @@ cudaError_t launch_prefix_stage(const il_stage_config *configs, int64_t n_cand, 
                                 int32_t *node_of, int *status, cudaStream_t stream);
 // Largest latencies of every node of a stage that queries leave after (select_kernel.cu).
 struct NodeTopParams {
-    uint64_t *records;            // [n_nodes][stride] leaving records (finish << qbits | query); overwritten
+    uint64_t *records;            // [rows][stride] leaving records (finish << qbits | query); overwritten
     int64_t stride;
+    const int32_t *row_of;        // row of node k (nullptr: row k)
+    int64_t offset;               // a node's records start this far into its row
     int32_t len;                  // records per node
     const int64_t *arrival;
     int32_t qbits;
@@ -202,6 +204,13 @@ struct CombineParams {
     int64_t *out_p99, *out_miss;
 };
 cudaError_t launch_prefix_combine(const CombineParams &p, cudaStream_t stream);
+// Covering candidates (prefix_kernel.cu): per node of a stage the smallest candidate that contains it
+// (marked in flags), the list of marked candidates with their positions, and per node its candidate's position.
+cudaError_t launch_cover_rep(const int32_t *node_of, int64_t n_cand, int32_t *rep, int64_t n_nodes, uint8_t *flags,
+                             cudaStream_t stream);
+cudaError_t launch_cover_list(const uint8_t *flags, int64_t n_cand, int32_t *list, int32_t *pos, int *count,
+                              cudaStream_t stream);
+cudaError_t launch_cover_rows(const int32_t *rep, const int32_t *pos, int64_t n_nodes, int32_t *row, cudaStream_t stream);
 
 // Fills order[0..n_cand) with the chunk's candidate indices, costliest first
 // (longest-processing-time-first scheduling over the warps).

@@ -92,6 +92,47 @@ prefix_lookup_kernel(const int32_t *slot_of, const int32_t *vals, int64_t n_cand
         node_of[c] = vals[slot_of[c]];
 }
 
+// ---- covering candidates ------------------------------------------------------------------------
+// The nodes can be simulated by the lane kernel, which only knows whole candidates: pick a set of
+// candidates of the batch that between them contain every node that queries leave after (the
+// candidate with the smallest index for each such node), simulate those, and read each node's leaving
+// records from the slab row of its candidate.
+
+// rep[k] = smallest candidate index whose node of this stage is k (rep filled with a large value).
+__global__ void __launch_bounds__(256)
+cover_rep_kernel(const int32_t *node_of, int64_t n_cand, int32_t *rep)
+{
+    for (int64_t c = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; c < n_cand; c += (int64_t)gridDim.x * blockDim.x)
+        atomicMin(&rep[node_of[c]], (int32_t)c);
+}
+
+__global__ void __launch_bounds__(256)
+cover_mark_kernel(const int32_t *rep, int64_t n_nodes, uint8_t *flags)
+{
+    for (int64_t k = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; k < n_nodes; k += (int64_t)gridDim.x * blockDim.x)
+        flags[rep[k]] = 1;
+}
+
+// The marked candidates, in any order: list[i] = candidate, pos[candidate] = i.
+__global__ void __launch_bounds__(256)
+cover_list_kernel(const uint8_t *flags, int64_t n_cand, int32_t *list, int32_t *pos, int *count)
+{
+    for (int64_t c = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; c < n_cand; c += (int64_t)gridDim.x * blockDim.x) {
+        if (!flags[c]) continue;
+        const int i = atomicAdd(count, 1);
+        list[i] = (int32_t)c;
+        pos[c] = i;
+    }
+}
+
+// row[k] = slab row of the candidate that stands for node k.
+__global__ void __launch_bounds__(256)
+cover_rows_kernel(const int32_t *rep, const int32_t *pos, int64_t n_nodes, int32_t *row)
+{
+    for (int64_t k = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; k < n_nodes; k += (int64_t)gridDim.x * blockDim.x)
+        row[k] = pos[rep[k]];
+}
+
 // P99 and miss count of every candidate from the nodes where its queries leave the pipeline.
 // Node i of leaving stage e has its `top` largest latencies in top_e[i][0 .. top), sorted in
 // descending order (entries beyond the node's own count are 0, below every latency), and its miss
@@ -152,6 +193,31 @@ cudaError_t launch_prefix_stage(const il_stage_config *configs, int64_t n_cand, 
                                                      slot_of, status);
     prefix_number_kernel<<<grid_t, 256, 0, stream>>>(keys, cap, vals, count, node_cfg, node_parent);
     prefix_lookup_kernel<<<grid_c, 256, 0, stream>>>(slot_of, vals, n_cand, node_of);
+    return cudaGetLastError();
+}
+
+static int cover_grid(int64_t items) { return (int)std::max<int64_t>(1, std::min<int64_t>((items + 255) / 256, 2368)); }
+
+cudaError_t launch_cover_rep(const int32_t *node_of, int64_t n_cand, int32_t *rep, int64_t n_nodes, uint8_t *flags,
+                             cudaStream_t stream)
+{
+    cudaError_t e = cudaMemsetAsync(rep, 0x7f, (size_t)n_nodes * 4, stream);
+    if (e != cudaSuccess) return e;
+    cover_rep_kernel<<<cover_grid(n_cand), 256, 0, stream>>>(node_of, n_cand, rep);
+    cover_mark_kernel<<<cover_grid(n_nodes), 256, 0, stream>>>(rep, n_nodes, flags);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_cover_list(const uint8_t *flags, int64_t n_cand, int32_t *list, int32_t *pos, int *count,
+                              cudaStream_t stream)
+{
+    cover_list_kernel<<<cover_grid(n_cand), 256, 0, stream>>>(flags, n_cand, list, pos, count);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_cover_rows(const int32_t *rep, const int32_t *pos, int64_t n_nodes, int32_t *row, cudaStream_t stream)
+{
+    cover_rows_kernel<<<cover_grid(n_nodes), 256, 0, stream>>>(rep, pos, n_nodes, row);
     return cudaGetLastError();
 }
 

@@ -201,7 +201,7 @@ node_top_kernel(const __grid_constant__ NodeTopParams p)
     while (pow2 < p.top_len) pow2 <<= 1;
     const uint64_t qmask = (1ull << p.qbits) - 1ull;
     for (int64_t node = blockIdx.x; node < p.n_nodes; node += gridDim.x) {
-        int64_t *lat = reinterpret_cast<int64_t *>(p.records + node * p.stride);
+        int64_t *lat = reinterpret_cast<int64_t *>(p.records + (p.row_of ? (int64_t)p.row_of[node] : node) * p.stride + p.offset);
         if (threadIdx.x == 0) { s_or = 0; s_miss = 0; s_fill = 0; s_prefix = 0; }
         __syncthreads();
         unsigned miss = 0;

@@ -38,10 +38,12 @@ def product_configs(rng, S, H, Bmax, max_replicas, per_stage):
     return cfg
 
 
+@pytest.mark.parametrize("mode", [1, 3], ids=["covering-candidates", "node-by-node"])
 @pytest.mark.parametrize("seed", range(10))
-def test_forced_sharing_on_random_pipelines(il, oracle, seed):
+def test_forced_sharing_on_random_pipelines(il, oracle, seed, mode):
     """Random chains and trees (cascades included), candidate sets with a lot of sharing (products of
-    2-3 choices per stage) and with hardly any (independent draws), equal stamps, R up to 32."""
+    2-3 choices per stage) and with hardly any (independent draws), equal stamps, R up to 32; the nodes
+    simulated by the lane kernel through a covering set of candidates, and one by one."""
     S = 1 + seed % 6
     w = workloads.random_small(seed, S=S, H=3, Bmax=[4, 33, 64][seed % 3], n=700 + 37 * seed, C=24,
                                max_replicas=[3, 8, 32][seed % 3], tree=(seed % 2 == 1), qps=400.0, cv=3.0,
@@ -51,11 +53,13 @@ def test_forced_sharing_on_random_pipelines(il, oracle, seed):
     w.configs = np.ascontiguousarray(np.concatenate([prod, w.configs, prod[:5]]))
     exp = oracle.estimate_workload(w)
     with il.Estimator.from_workload(w) as est:
-        est.set_test_knob(KNOB_SHARE, 1)
+        est.set_test_knob(KNOB_SHARE, mode)
         p99, miss = est.estimate(w.configs, w.slo_us)
         st = est.stats()
         assert np.array_equal(p99, exp[0]) and np.array_equal(miss, exp[1]), np.nonzero(p99 != exp[0])[0][:5]
         assert st["stage_runs"] < w.n_candidates * S and st["candidates"] == w.n_candidates
+        if mode == 1:
+            assert st["stage_runs"] % S == 0          # whole candidates
         assert np.array_equal(est.feasible(w.configs, w.slo_us), exp[0] <= w.slo_us)
         est.set_test_knob(KNOB_SHARE, 2)
         p99, miss = est.estimate(w.configs, w.slo_us)
@@ -76,6 +80,11 @@ def test_sharing_is_chosen_for_a_product_sweep(il, oracle, oracle_pool):
         st = est.stats()
         assert np.array_equal(a.cpu().numpy(), exp[0]) and np.array_equal(b.cpu().numpy(), exp[1])
         assert st["stage_runs"] * 4 <= w.n_candidates * w.n_stages
+        est.set_test_knob(KNOB_SHARE, 3)              # the same nodes one by one
+        a, b = est.estimate_device(torch.from_numpy(w.configs).cuda(), w.slo_us)
+        assert np.array_equal(a.cpu().numpy(), exp[0]) and np.array_equal(b.cpu().numpy(), exp[1])
+        assert est.stats()["stage_runs"] == 8 + 64 + 64 + 512 + 3 * 64 + 512
+        est.set_test_knob(KNOB_SHARE, 0)
         got = est.feasible_device(torch.from_numpy(w.configs).cuda(), w.slo_us).cpu().numpy().astype(bool)
         assert np.array_equal(got, exp[0] <= w.slo_us)
     w = workloads.make(3, n_queries=3000, n_candidates=2500)
