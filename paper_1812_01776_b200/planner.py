@@ -7,12 +7,19 @@ compared.  Where the paper's loops ask one question at a time and the answers
 do not depend on each other, the questions are put to the estimator as ONE
 batch of candidates:
 
-* Algorithm 2 evaluates, per iteration, three actions for every model; all
-  resulting configurations go out in one call;
-* the hardware downgrade re-initialises one model on the next cheaper
-  hardware (add replicas until feasible) and then minimises that model's cost
-  locally; both loops walk a small grid (replicas x batch sizes of that one
-  model), which is evaluated in one call and then walked on the host.
+* Algorithm 2 evaluates, per iteration, three actions for every model.  The
+  hardware downgrade re-initialises one model on the next cheaper hardware (add
+  replicas until feasible) and then minimises that model's cost locally; both
+  loops walk a small grid (replicas x batch sizes of that one model).  The
+  grids of all models and the two simple actions of all models go out in ONE
+  call per iteration (a few hundred to a few thousand configurations, which
+  cost the GPU the same one wave as a single configuration) and are then walked
+  on the host;
+* Algorithm 1 adds a replica to the throughput bottleneck until the Estimator
+  says feasible.  Which model is the bottleneck follows from the profiles, not
+  from the Estimator's answers, so the next configurations of that sequence are
+  known in advance: they are evaluated a run at a time, and the first feasible
+  one is taken.
 
 Rules taken from the paper:
 
@@ -140,40 +147,58 @@ class Planner:
             steps.append("initialize: service time exceeds the objective")
             return None
         while True:
-            ok, _ = self.feasible_many(cfg[None])
-            if ok[0]:
+            # the next configurations of the sequence "add a replica to the bottleneck", this one first
+            run = [cfg.copy()]
+            stuck = False
+            while len(run) < self.INIT_RUN:
+                nxt = self._grow_bottleneck(run[-1])
+                if nxt is None:
+                    stuck = True
+                    break
+                run.append(nxt)
+            ok, _ = self.feasible_many(np.stack(run))
+            hit = np.nonzero(ok)[0]
+            if hit.size:
+                cfg = run[int(hit[0])]
                 steps.append(f"initialize: feasible with replicas {cfg[:, 2].tolist()}")
                 return cfg
-            thr = self.throughput(cfg)
-            # the bottleneck among the models that can still grow
-            order = np.argsort(thr, kind="stable")
-            grown = False
-            for s in order:
-                if cfg[s, 2] < MAX_REPLICAS:
-                    cfg[s, 2] += 1
-                    grown = True
-                    break
-            if not grown:
+            nxt = None if stuck else self._grow_bottleneck(run[-1])
+            if nxt is None:
                 steps.append("initialize: every model at the replica limit, still infeasible")
                 return None
+            cfg = nxt
+
+    INIT_RUN = 32      # configurations of the Initialize sequence evaluated per call
+
+    def _grow_bottleneck(self, cfg: np.ndarray) -> Optional[np.ndarray]:
+        """cfg with one more replica for the throughput bottleneck among the models that can still grow."""
+        thr = self.throughput(cfg)
+        for s in np.argsort(thr, kind="stable"):
+            if cfg[s, 2] < MAX_REPLICAS:
+                new = cfg.copy()
+                new[s, 2] += 1
+                return new
+        return None
 
     # ---- Algorithm 2 -------------------------------------------------------
 
-    def _downgrade(self, cfg: np.ndarray, s: int) -> Optional[np.ndarray]:
-        """Model s on the next cheaper hardware, other models frozen: initialise
-        (batch 1, add replicas until feasible), then minimise locally (increase
-        batch / remove replica while feasible).  Accepted only if cheaper."""
+    def _downgrade_grid(self, cfg: np.ndarray, s: int) -> Optional[Tuple[int, np.ndarray]]:
+        """Every (batch, replicas) of model s on the next cheaper hardware, other models as in cfg."""
         hw = self.next_cheaper(int(cfg[s, 0]))
         if hw is None:
             return None
-        # every (batch, replicas) of this one model on the new hardware, in one call
         grid = np.repeat(cfg[None], len(self.batches) * MAX_REPLICAS, axis=0)
         k = 0
         for b in self.batches:
             for r in range(1, MAX_REPLICAS + 1):
                 grid[k, s] = (hw, b, r, 0)
                 k += 1
-        ok, _ = self.feasible_many(grid)
+        return hw, grid
+
+    def _downgrade_pick(self, cfg: np.ndarray, s: int, hw: int, ok: np.ndarray) -> Optional[np.ndarray]:
+        """Model s on hardware hw, other models frozen: initialise (batch 1, add
+        replicas until feasible), then minimise locally (increase batch / remove
+        replica while feasible), walking the grid's answers.  Accepted only if cheaper."""
         ok = ok.reshape(len(self.batches), MAX_REPLICAS)
         # initialise: batch 1, replicas 1, 2, ... until feasible
         feas_r = np.nonzero(ok[0])[0]
@@ -192,6 +217,14 @@ class Planner:
         new[s] = (hw, self.batches[bi], r, 0)
         return new if self.cost(new) < self.cost(cfg) else None
 
+    def _downgrade(self, cfg: np.ndarray, s: int) -> Optional[np.ndarray]:
+        """The downgrade action of model s, with a call of its own."""
+        g = self._downgrade_grid(cfg, s)
+        if g is None:
+            return None
+        ok, _ = self.feasible_many(g[1])
+        return self._downgrade_pick(cfg, s, g[0], ok)
+
     def minimize_cost(self) -> PlanResult:
         steps: List[str] = []
         cfg = self.initialize(steps)
@@ -199,30 +232,51 @@ class Planner:
             return PlanResult(False, None, float("inf"), -1, self.calls, self.evaluated, steps, [])
         trajectory = [cfg.copy()]
         while True:
-            cands, labels = [], []
+            # one call per iteration: the simple actions of every model and every model's downgrade grid
+            simple, simple_labels, simple_model, grids = [], [], [], {}
             for s in range(self.S):
                 if cfg[s, 2] > 1:
                     new = cfg.copy(); new[s, 2] -= 1
-                    cands.append(new); labels.append(f"remove replica of model {s}")
-                down = self._downgrade(cfg, s)      # feasible by construction, cheaper than cfg
-                if down is not None:
-                    cands.append(down); labels.append(f"downgrade model {s} to hw {int(down[s, 0])} "
-                                                      f"(batch {int(down[s, 1])}, replicas {int(down[s, 2])})")
+                    simple.append(new); simple_labels.append(f"remove replica of model {s}"); simple_model.append((s, 0))
                 if int(cfg[s, 1]) * 2 <= self.Bmax:
                     new = cfg.copy(); new[s, 1] = int(cfg[s, 1]) * 2
-                    cands.append(new); labels.append(f"double batch of model {s} to {int(new[s, 1])}")
-            if not cands:
+                    simple.append(new); simple_labels.append(f"double batch of model {s} to {int(new[s, 1])}")
+                    simple_model.append((s, 2))
+                g = self._downgrade_grid(cfg, s)
+                if g is not None:
+                    grids[s] = g
+            if not simple and not grids:
                 break
-            ok, _ = self.feasible_many(np.stack(cands))
+            parts = ([np.stack(simple)] if simple else []) + [grids[s][1] for s in sorted(grids)]
+            ok, _ = self.feasible_many(np.concatenate(parts))
+            # candidates in the order (model, remove replica, downgrade, double batch), as ties are broken
+            cands = []
+            at = len(simple)
+            downs = {}
+            for s in sorted(grids):
+                n_grid = grids[s][1].shape[0]
+                downs[s] = self._downgrade_pick(cfg, s, grids[s][0], ok[at:at + n_grid])   # feasible by construction
+                at += n_grid
+            for s in range(self.S):
+                for i, (m, kind) in enumerate(simple_model):
+                    if m == s and kind == 0 and ok[i]:
+                        cands.append((simple[i], simple_labels[i]))
+                if downs.get(s) is not None:
+                    d = downs[s]
+                    cands.append((d, f"downgrade model {s} to hw {int(d[s, 0])} "
+                                     f"(batch {int(d[s, 1])}, replicas {int(d[s, 2])})"))
+                for i, (m, kind) in enumerate(simple_model):
+                    if m == s and kind == 2 and ok[i]:
+                        cands.append((simple[i], simple_labels[i]))
             best = None
             for i in range(len(cands)):
-                if ok[i] and (best is None or self.cost(cands[i]) < self.cost(cands[best])):
+                if best is None or self.cost(cands[i][0]) < self.cost(cands[best][0]):
                     best = i
             if best is None:
                 break
-            cfg = cands[best]
+            cfg = cands[best][0]
             trajectory.append(cfg.copy())
-            steps.append(f"{labels[best]} -> cost {self.cost(cfg):.4f}")
+            steps.append(f"{cands[best][1]} -> cost {self.cost(cfg):.4f}")
         p99, _ = self._estimate(np.ascontiguousarray(cfg[None], dtype=np.uint8))
         self.calls += 1
         self.evaluated += 1
