@@ -498,23 +498,6 @@ static int enqueue_simulation(il_estimator *e, const DesParams &p, const Plan &p
     return IL_OK;
 }
 
-// Where each stage's leaving queries end in a slab row written by the lane kernel.
-static void slab_regions(const il_estimator *e, SelectParams &sp)
-{
-    sp.n_regions = 0;
-    int32_t off = 0;
-    for (int s = 0; s < e->S; s++) {
-        const int a = e->base.dest_a[s], b = e->base.dest_b[s];
-        int32_t kids = 0;
-        if (a >= 0) kids += e->base.n_s[a];
-        if (b >= 0 && b != a) kids += e->base.n_s[b];
-        const int32_t leaving = e->base.n_s[s] - kids;
-        off += leaving;
-        if (leaving > 0) sp.region_end[sp.n_regions++] = off;
-    }
-}
-
-
 // End of a shared-prefix call: events[0], events[1] and the work in between are on the stream.
 static int finish_shared(il_estimator *e, int64_t n_cand, int64_t launches, int64_t stage_runs)
 {
@@ -1191,13 +1174,9 @@ int il_estimate_device(il_estimator *e, const il_stage_config *d_configs, int64_
         if (rc) return rc;
         IL_CUDA(cudaEventRecord(e->events[3 + 3 * ch], st));
         SelectParams sp = {};
-        sp.slab = p.slab; sp.slab_stride = e->n_pad; sp.lat_or = p.lat_or;
+        sp.slab = p.slab; sp.slab_stride = e->n_pad;
         sp.arrival = e->d_arrival; sp.qbits = p.qbits; sp.packed = sim_kernel(e) != kSimWide ? 1 : 0;
         sp.status = e->d_status;
-        if (lane && !e->fork) {
-            slab_regions(e, sp);
-            if (e->lane_wrap) sp.ovf = p.ovf;
-        }
         sp.n = (int32_t)e->n; sp.n_cand = cnt; sp.slo_us = slo_us;
         sp.out_p99 = d_out_p99 + lo; sp.out_miss = d_out_miss + lo;
         IL_CUDA(launch_select(sp, st));

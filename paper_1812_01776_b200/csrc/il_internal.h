@@ -95,13 +95,6 @@ struct SelectParams {
     const int64_t *arrival;       // [n], to turn packed records into latencies
     int32_t qbits;
     int32_t packed;               // slab holds packed records (from a packed-record simulation kernel)
-    // Packed slabs of the lane kernel: the queries that leave after stage s fill one region of the row,
-    // in finish order, so the last record of each region carries that region's largest finish time.
-    int32_t n_regions;            // 0: not known
-    int32_t region_end[IL_MAX_STAGES];   // one past the last record of each non-empty region
-    const uint64_t *lat_or;       // [n_cand]: OR of the latencies (wide kernel)
-    const uint8_t *ovf;           // if set: candidates whose row does not have the region layout (they were
-                                  // evaluated by the warp-per-candidate kernel after a ring overflow)
     int *status;                  // checked build: where an index out of range is recorded
     int32_t n;
     int64_t n_cand;

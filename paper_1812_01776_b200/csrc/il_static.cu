@@ -77,10 +77,9 @@ static int enqueue_static(const BoundView &v, unsigned char *base, const il_stag
     IL_ST(launch_simulation(p, v.kernel, (int)(slots / kWarpsPerCta), v.smem, st));
 
     SelectParams sp = {};
-    sp.slab = p.slab; sp.slab_stride = v.n_pad; sp.lat_or = p.lat_or;
+    sp.slab = p.slab; sp.slab_stride = v.n_pad;
     sp.arrival = p.arrival; sp.qbits = p.qbits; sp.packed = v.kernel != kSimWide ? 1 : 0;
     sp.status = p.status;
-    sp.n_regions = 0;
     sp.n = (int32_t)v.n; sp.n_cand = n_cand; sp.slo_us = slo_us;
     sp.out_p99 = d_out_p99; sp.out_miss = d_out_miss;
     IL_ST(launch_select(sp, st));

@@ -2,184 +2,220 @@
 //
 // P99 is the k-th smallest of the candidate's n latencies with
 // k = ceil(0.99 n) = (99 n + 99) / 100 (Section 2: 99% of the query latencies
-// must lie below the objective); a query misses iff latency > slo.  The k-th
-// smallest is found by most-significant-digit radix select: each pass
-// histograms one 8-bit digit of the keys that still match the prefix found so
-// far, then descends into the bucket that holds rank k.  Digits above the
-// highest set bit of any latency (known from the simulation kernel's OR) are
-// skipped.  One CTA per candidate.
+// must lie below the objective); a query misses iff latency > slo.  One CTA per
+// candidate.  The row is never rewritten: a slab of packed (finish time, query)
+// records is turned into latencies on the fly, latency = finish - arrival[query]
+// (the trace stays in L2), in every pass that needs them.
 //
-// When the slab comes from a packed-record simulation kernel it holds
-// (finish time, query) records; a first sweep replaces each by
-// latency = finish - arrival[query], ORs the latencies and counts the misses.
-// When the slab's regions are known (lane kernel: one region per stage that
-// queries leave after, each in finish order), the last record of each region
-// gives the candidate's largest finish time, and largest finish - first arrival
-// bounds every latency before the sweep: if that is below 2^32 the sweep writes 32-bit latencies (into the front
-// half of the row; one barrier per 256 records keeps the writes behind the
-// reads) and histograms the top digit on the way, and the remaining passes read
-// half the bytes.
+// The k-th smallest is found by a radix select whose FIRST digit needs no bound
+// on the latencies: a latency falls into one of 8,192 bins by its bit length and
+// the seven bits below its leading one (values below 256 have a bin each), which
+// is monotone in the value and resolves it to better than 1 %.  The pass that
+// fills this histogram also counts the misses.  The bin that holds rank k spans
+// 2^e consecutive values.  If it holds at most 4,096 latencies (the rule, since
+// rank k sits in the thin upper tail), a second pass over the row collects them
+// into shared memory, in the space of the histogram, and the select ends there;
+// otherwise passes with plain 13-bit digits over the bin's offsets narrow it
+// until that holds or no bit is left (all latencies equal: two passes).  A
+// thread requests the records of its next round before it uses those of the
+// current one (eight independent 8-byte loads in flight), which is what the row
+// passes need to run near memory speed.
 #include "il_internal.h"
 
 namespace il {
 
-__global__ void __launch_bounds__(kSelectThreads)
-select_kernel(const __grid_constant__ SelectParams p)
+namespace {
+
+constexpr int kSelBins = 8192;       // bins of a histogram pass
+constexpr int kSelCap = 4096;        // latencies the shared-memory list holds (the same 32 KB)
+// Records a thread requests per round (it has two rounds in flight) and resident CTAs per SM.  Measured on
+// 50,000- to 1,000,000-record rows: 4 x 4 as here 0.68 / 40.4 / 50.2 ms on three workloads, 8 x 4 0.70 / 40.8 /
+// 52.4, 4 x 6 (40 registers) 0.81 / 62.2 / 67.0, 2 x 6 0.74 / 56.1 / 62.3, 8 x 3 0.92 / 49.8 / 60.6.
+constexpr int kSelUnroll = 4;
+constexpr int kSelCtasPerSm = 4;
+constexpr int kSelDigit = 13;        // bits of a refinement digit: 2^13 = kSelBins
+
+// Bin of the first pass.  Monotone in l; bin B >= 128 holds the values [m << e, (m + 1) << e) with
+// e = (B >> 7) - 1 and m = B - (e << 7) in [128, 256); B < 128 holds the value B alone.
+__device__ __forceinline__ unsigned first_bin(uint64_t l)
 {
-    __shared__ unsigned hist[256];
-    __shared__ unsigned long long s_prefix;
-    __shared__ unsigned s_rank;
-    __shared__ unsigned s_miss;
-    __shared__ unsigned long long s_or;
+    if (l < 128u) return (unsigned)l;
+    const int e = 56 - __clzll((long long)l);
+    return ((unsigned)e << 7) + (unsigned)(l >> e);
+}
 
-    for (int64_t c = blockIdx.x; c < p.n_cand; c += gridDim.x) {
-        int64_t *lat = p.slab + c * p.slab_stride;
-        unsigned miss = 0;
-        bool counted_miss = false;
-        uint64_t bits_used;
-        if (p.packed && p.n_regions > 0 && !(p.ovf && p.ovf[c])) {
-            uint64_t last = 0;
+struct SelectShared {
+    unsigned warp_sum[kSelectThreads / 32];
+    unsigned bin, rank, count;       // result of find_rank
+    unsigned fill, miss;
+    unsigned long long prefix;
+};
+
+// The bin of h[0 .. PER * 256) that holds the rank-th smallest element (1-based), the rank inside
+// that bin and the bin's count, left in sh.bin / sh.rank / sh.count.  Thread t owns bins
+// [PER * t, PER * (t + 1)); it reads them in a rotated order so that the threads of a warp never meet in
+// a bank.  Called by all threads; ends with a barrier.
+template <int PER>
+__device__ __forceinline__ void find_rank(const unsigned *h, unsigned rank, SelectShared &sh)
+{
+    const int t = threadIdx.x, lane = t & 31, w = t >> 5;
+    unsigned mine = 0;
 #pragma unroll
-            for (int r = 0; r < IL_MAX_STAGES; r++)      // unrolled: constant indices into the parameter block
-                if (r < p.n_regions) last = max(last, (uint64_t)lat[p.region_end[r] - 1] >> p.qbits);
-            const int64_t bound64 = (int64_t)last - p.arrival[0];
-            if (bound64 < (INT64_C(1) << 32)) {
-                const uint32_t bound = bound64 > 0 ? (uint32_t)bound64 : 0u;
-                int top32 = 0;
-                while (top32 < 4 && (bound >> (8 * top32)) != 0) top32++;
-                hist[threadIdx.x] = 0;
-                if (threadIdx.x == 0) {
-                    s_prefix = 0;
-                    s_rank = (unsigned)((99ll * p.n + 99) / 100);
-                    s_miss = 0;
-                }
-                __syncthreads();
-                uint32_t *lat32 = reinterpret_cast<uint32_t *>(lat);
-                const uint64_t qmask = (1ull << p.qbits) - 1ull;
-                const int sh_top = top32 > 0 ? 8 * (top32 - 1) : 0;
-                for (int base = 0; base < p.n; base += kSelectThreads) {
-                    const int i = base + (int)threadIdx.x;
-                    uint32_t l = 0;
-                    if (i < p.n) {
-                        const uint64_t rec = (uint64_t)lat[i];
-                        if (IL_IN_RANGE(rec & qmask, p.n, p.status))
-                            l = (uint32_t)((int64_t)(rec >> p.qbits) - p.arrival[rec & qmask]);
-                        miss += ((int64_t)l > p.slo_us);
-                    }
-                    __syncthreads();        // all records of this block are read before their row space is reused
-                    if (i < p.n) {
-                        lat32[i] = l;
-                        atomicAdd(&hist[(l >> sh_top) & 0xff], 1u);
-                    }
-                }
-                __syncthreads();
-                for (int d = top32 - 1; d >= 0; d--) {
-                    const int shift = 8 * d;
-                    if (d != top32 - 1) {
-                        hist[threadIdx.x] = 0;
-                        __syncthreads();
-                        const uint32_t prefix = (uint32_t)s_prefix;
-                        const uint32_t himask = ~0u << (shift + 8);     // d <= 2 here
-                        for (int i = threadIdx.x; i < p.n; i += kSelectThreads) {
-                            const uint32_t v = lat32[i];
-                            if ((v & himask) == prefix) atomicAdd(&hist[(v >> shift) & 0xff], 1u);
-                        }
-                        __syncthreads();
-                    }
-                    if (threadIdx.x == 0) {
-                        unsigned r = s_rank, acc = 0;
-                        int b = 0;
-                        for (; b < 255; b++) {
-                            if (acc + hist[b] >= r) break;
-                            acc += hist[b];
-                        }
-                        s_rank = r - acc;
-                        s_prefix = s_prefix | ((unsigned long long)b << shift);
-                    }
-                    __syncthreads();
-                }
-                if (miss) atomicAdd(&s_miss, miss);
-                __syncthreads();
-                if (threadIdx.x == 0) {
-                    p.out_p99[c] = (int64_t)s_prefix;
-                    p.out_miss[c] = (int64_t)s_miss;
-                }
-                __syncthreads();
-                continue;
-            }
+    for (int j = 0; j < PER; j++) mine += h[PER * t + ((j + t) & (PER - 1))];
+    unsigned incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) sh.warp_sum[w] = incl;
+    __syncthreads();
+    unsigned before = incl - mine;
+    for (int k = 0; k < w; k++) before += sh.warp_sum[k];
+    if (before < rank && rank <= before + mine) {      // exactly one thread
+        unsigned acc = before;
+        for (int j = 0; j < PER; j++) {
+            const unsigned c = h[PER * t + j];
+            if (acc + c >= rank) { sh.bin = (unsigned)(PER * t + j); sh.rank = rank - acc; sh.count = c; break; }
+            acc += c;
         }
-        if (p.packed) {
-            if (threadIdx.x == 0) s_or = 0;
-            __syncthreads();
-            const uint64_t qmask = (1ull << p.qbits) - 1ull;
-            unsigned long long my_or = 0;
-            for (int i = threadIdx.x; i < p.n; i += kSelectThreads) {
-                const uint64_t rec = (uint64_t)lat[i];
-                int64_t l = 0;
-                if (IL_IN_RANGE(rec & qmask, p.n, p.status)) l = (int64_t)(rec >> p.qbits) - p.arrival[rec & qmask];
-                lat[i] = l;
-                my_or |= (unsigned long long)l;
-                miss += (l > p.slo_us);
-            }
-            counted_miss = true;
-            my_or |= __shfl_xor_sync(0xffffffffu, my_or, 16);
-            my_or |= __shfl_xor_sync(0xffffffffu, my_or, 8);
-            my_or |= __shfl_xor_sync(0xffffffffu, my_or, 4);
-            my_or |= __shfl_xor_sync(0xffffffffu, my_or, 2);
-            my_or |= __shfl_xor_sync(0xffffffffu, my_or, 1);
-            if ((threadIdx.x & 31) == 0 && my_or) atomicOr(&s_or, my_or);
-            __syncthreads();   // also orders the latency writes before the passes below
-            bits_used = s_or;
-        } else {
-            bits_used = p.lat_or[c];
-        }
-        int top = 0;                                   // number of 8-bit digits that matter
-        while (top < 8 && (bits_used >> (8 * top)) != 0) top++;
+    }
+    __syncthreads();
+}
 
-        if (threadIdx.x == 0) {
-            s_prefix = 0;
-            s_rank = (unsigned)((99ll * p.n + 99) / 100);   // 1-indexed rank still to find
-            s_miss = 0;
+// One pass over a row.  MODE 0: first-bin histogram of every latency, misses counted.  MODE 1:
+// histogram of ((latency - lo) >> sh) over the latencies in [lo, lo + 2^e).  MODE 2: the offsets
+// latency - lo of those latencies appended to the list.
+template <bool PACKED, int MODE>
+__device__ __forceinline__ void row_pass(const SelectParams &p, const uint64_t *__restrict__ row, unsigned *hist,
+                                         SelectShared &sh, uint64_t lo, int e, int shift, unsigned &miss)
+{
+    const uint64_t qmask = (1ull << p.qbits) - 1ull;
+    const uint64_t width_m1 = e >= 64 ? ~0ull : ((1ull << e) - 1ull);
+    uint64_t *list = reinterpret_cast<uint64_t *>(hist);
+    const int n = p.n;
+    // software pipeline: the records of the next round are requested before this round's are used
+    uint64_t nx[kSelUnroll];
+#pragma unroll
+    for (int u = 0; u < kSelUnroll; u++) {
+        const int i = u * kSelectThreads + (int)threadIdx.x;
+        nx[u] = i < n ? __ldg(row + i) : 0ull;
+    }
+    for (int base = 0; base < n; base += kSelectThreads * kSelUnroll) {
+        uint64_t v[kSelUnroll];
+#pragma unroll
+        for (int u = 0; u < kSelUnroll; u++) {
+            const int i = base + (kSelUnroll + u) * kSelectThreads + (int)threadIdx.x;
+            v[u] = nx[u];
+            nx[u] = i < n ? __ldg(row + i) : 0ull;
         }
-        __syncthreads();
-
-        for (int d = top - 1; d >= 0; d--) {
-            hist[threadIdx.x] = 0;                     // kSelectThreads == 256 bins
-            __syncthreads();
-            const unsigned long long prefix = s_prefix;
-            const int shift = 8 * d;
-            // keys whose digits above d equal the prefix are still in the running
-            const unsigned long long himask = (d == 7) ? 0ull : (~0ull << (shift + 8));
-            for (int i = threadIdx.x; i < p.n; i += kSelectThreads) {
-                const unsigned long long v = (unsigned long long)lat[i];
-                if (!counted_miss) miss += ((int64_t)v > p.slo_us);
-                if ((v & himask) == prefix) atomicAdd(&hist[(v >> shift) & 0xff], 1u);
+        if (PACKED) {
+#pragma unroll
+            for (int u = 0; u < kSelUnroll; u++) {
+                const int i = base + u * kSelectThreads + (int)threadIdx.x;
+                const uint64_t q = v[u] & qmask;
+                if (i < n && IL_IN_RANGE(q, p.n, p.status))
+                    v[u] = (v[u] >> p.qbits) - (uint64_t)__ldg(p.arrival + q);
+                else
+                    v[u] = 0ull;
             }
-            counted_miss = true;
-            __syncthreads();
-            if (threadIdx.x == 0) {
-                unsigned r = s_rank, acc = 0;
-                int b = 0;
-                for (; b < 255; b++) {
-                    if (acc + hist[b] >= r) break;
-                    acc += hist[b];
+        }
+#pragma unroll
+        for (int u = 0; u < kSelUnroll; u++) {
+            const int i = base + u * kSelectThreads + (int)threadIdx.x;
+            if (i >= n) continue;
+            if (MODE == 0) {
+                miss += ((int64_t)v[u] > p.slo_us) ? 1u : 0u;
+                atomicAdd(&hist[first_bin(v[u])], 1u);
+            } else {
+                const uint64_t off = v[u] - lo;
+                if (off <= width_m1) {
+                    if (MODE == 1) {
+                        atomicAdd(&hist[(unsigned)(off >> shift)], 1u);
+                    } else {
+                        const unsigned pos = atomicAdd(&sh.fill, 1u);
+                        if (pos < (unsigned)kSelCap) list[pos] = off;
+                    }
                 }
-                s_rank = r - acc;
-                s_prefix = prefix | ((unsigned long long)b << shift);
             }
-            __syncthreads();
         }
-        if (!counted_miss) {   // every latency is zero: cannot happen (tables >= 1); kept for safety
-            for (int i = threadIdx.x; i < p.n; i += kSelectThreads) miss += (lat[i] > p.slo_us);
-        }
-        if (miss) atomicAdd(&s_miss, miss);
+    }
+}
+
+template <bool PACKED>
+__device__ __forceinline__ void select_rows(const SelectParams &p, unsigned *hist, unsigned *hist256, SelectShared &sh)
+{
+    uint64_t *list = reinterpret_cast<uint64_t *>(hist);
+    for (int64_t c = blockIdx.x; c < p.n_cand; c += gridDim.x) {
+        const uint64_t *row = reinterpret_cast<const uint64_t *>(p.slab + c * p.slab_stride);
+        for (int i = threadIdx.x; i < kSelBins; i += kSelectThreads) hist[i] = 0u;
+        if (threadIdx.x == 0) sh.miss = 0u;
         __syncthreads();
+        unsigned miss = 0, unused = 0;
+        row_pass<PACKED, 0>(p, row, hist, sh, 0ull, 0, 0, miss);
+        for (int o = 16; o > 0; o >>= 1) miss += __shfl_xor_sync(0xffffffffu, miss, o);
+        if ((threadIdx.x & 31) == 0 && miss) atomicAdd(&sh.miss, miss);
+        __syncthreads();
+        find_rank<kSelBins / kSelectThreads>(hist, (unsigned)((99ll * p.n + 99) / 100), sh);
+        unsigned rank = sh.rank, count = sh.count;
+        int e = sh.bin < 128u ? 0 : (int)(sh.bin >> 7) - 1;
+        uint64_t lo = sh.bin < 128u ? (uint64_t)sh.bin : (uint64_t)(sh.bin - ((unsigned)e << 7)) << e;
+        // narrow [lo, lo + 2^e) until its latencies fit the list
+        while (e > 0 && count > (unsigned)kSelCap) {
+            const int d = e < kSelDigit ? e : kSelDigit;
+            __syncthreads();                 // everybody has read sh.bin / sh.rank / sh.count
+            for (int i = threadIdx.x; i < kSelBins; i += kSelectThreads) hist[i] = 0u;
+            __syncthreads();
+            row_pass<PACKED, 1>(p, row, hist, sh, lo, e, e - d, unused);
+            __syncthreads();
+            find_rank<kSelBins / kSelectThreads>(hist, rank, sh);
+            lo += (uint64_t)sh.bin << (e - d);
+            e -= d;
+            rank = sh.rank; count = sh.count;
+        }
+        if (e > 0) {
+            // the rest in shared memory: collect the offsets, then 8-bit digits over the list
+            __syncthreads();
+            if (threadIdx.x == 0) sh.fill = 0u;
+            __syncthreads();
+            row_pass<PACKED, 2>(p, row, hist, sh, lo, e, 0, unused);
+            __syncthreads();
+            const unsigned got = sh.fill < (unsigned)kSelCap ? sh.fill : (unsigned)kSelCap;
+            uint64_t prefix = 0;
+            for (int shift = ((e - 1) >> 3) << 3; shift >= 0; shift -= 8) {
+                hist256[threadIdx.x] = 0u;
+                __syncthreads();
+                const uint64_t himask = shift + 8 >= 64 ? 0ull : (~0ull << (shift + 8));
+                for (unsigned i = threadIdx.x; i < got; i += kSelectThreads) {
+                    const uint64_t v = list[i];
+                    if ((v & himask) == prefix) atomicAdd(&hist256[(unsigned)(v >> shift) & 0xffu], 1u);
+                }
+                __syncthreads();
+                find_rank<1>(hist256, rank, sh);
+                prefix |= (uint64_t)sh.bin << shift;
+                rank = sh.rank;
+                __syncthreads();
+            }
+            lo += prefix;
+        }
         if (threadIdx.x == 0) {
-            p.out_p99[c] = (int64_t)s_prefix;
-            p.out_miss[c] = (int64_t)s_miss;
+            p.out_p99[c] = (int64_t)lo;
+            p.out_miss[c] = (int64_t)sh.miss;
         }
         __syncthreads();
     }
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(kSelectThreads, kSelCtasPerSm)
+select_kernel(const __grid_constant__ SelectParams p)
+{
+    __shared__ __align__(16) unsigned hist[kSelBins];
+    __shared__ unsigned hist256[kSelectThreads];
+    __shared__ SelectShared sh;
+    if (p.packed) select_rows<true>(p, hist, hist256, sh);
+    else select_rows<false>(p, hist, hist256, sh);
 }
 
 // Shared-prefix evaluation: the largest latencies of one node of a stage that queries leave after.

@@ -43,4 +43,11 @@ SELECT_CASES = {
     "p99_above_2_32": ([1] * 90 + [5, 3, 2], {1: 40, 5: 3 * 2 ** 31 - 9, 3: 2 ** 32 + 1, 2: 2 ** 32}, 3),
     "byte_boundaries": ([1 + g % 8 for g in range(400)], {1: 255, 2: 256, 3: 65535, 4: 65536, 5: 2 ** 24 - 1,
                                                            6: 2 ** 24, 7: 2 ** 31 - 1, 8: 257}, 1),
+    # more than 4,096 latencies that agree in their bit length and the seven bits below the leading one (what a
+    # radix select with a logarithmic first digit must narrow down before it can finish on a short list):
+    # all equal; the rank among 1,280 equal values 2^14 above 4,640 others; the rank inside those 4,640
+    "all_equal_n6400": ([64] * 100, {64: 1000003}, 1),
+    "crowded_then_few": ([64] * 70 + [32] * 40 + [16] * 10,
+                         {64: 2 ** 33 + 5, 32: 2 ** 33 + 5 + 2 ** 14, 16: 2 ** 33 + 8}, 6),
+    "crowded_twice": ([64] * 70 + [32] + [16] * 10, {64: 2 ** 33 + 5, 32: 2 ** 33 + 5 + 2 ** 14, 16: 2 ** 33 + 8}, 6),
 }
