@@ -421,12 +421,16 @@ IL_API int il_set_variant(il_estimator *est, int variant);
  *                           the lane kernel would do.
  *   IL_KNOB_LANE_CTAS       value 0..16: resident CTAs (of two warps) per SM of the lane kernel; 0 restores
  *                           the library's choice (4).  For measurements.
+ *   IL_KNOB_BITS_IN_RECORDS value 0 or 1: whether the lane kernel's stream records carry the queries' branch
+ *                           bits (1, the default where the time range leaves room) or every stage looks
+ *                           them up by query index (0).  Same results either way.
  * Set a knob before il_workspace_bytes / il_set_workspace: sizes depend on the ring length.
  */
 #define IL_KNOB_LANE_RING_LOG2 1
 #define IL_KNOB_ITER_LIMIT 2
 #define IL_KNOB_SHARE_PREFIXES 3
 #define IL_KNOB_LANE_CTAS 4
+#define IL_KNOB_BITS_IN_RECORDS 5
 IL_API int il_set_test_knob(il_estimator *est, int knob, int64_t value);
 
 /* Name of the simulation kernel the handle's next estimate call will launch

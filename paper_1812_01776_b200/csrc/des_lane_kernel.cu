@@ -173,8 +173,14 @@ des_lane_kernel(const __grid_constant__ DesParams p)
     // (the profile tables stay in global memory: a lane copies its row from there once per candidate, and
     // shared memory not spent on them is L1 for the stream records)
     unsigned char *wm_base = smem_raw;
-    const int q = p.qbits;
+    // A stream record is (time << q) | low part; the low part is the query index, below the query's
+    // branch bits when the records carry them (rb > 0: no stage then looks the bits up).  Keys of batches
+    // use the same q, with the index of the batch's first arrival in the low part.
+    const int qi = p.qbits, rb = BRANCHY ? p.rec_bits : 0;
+    const int q = qi + rb;
     const uint64_t qmask = (1ull << q) - 1ull;
+    const uint32_t imask = (uint32_t)((1ull << qi) - 1ull);
+    const uint64_t *trace = rb > 0 ? p.ptrace_b : p.ptrace;
 
     const unsigned full = 0xffffffffu;
     const int wid = threadIdx.x >> 5;
@@ -209,7 +215,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
 
     const int64_t wslot = (int64_t)blockIdx.x * kLaneWarps + wid;
     uint64_t *my_block = p.lane_ws + (wslot * cpw + (lane_used ? j : 0)) * p.lane_elems;
-    const uint64_t *in = s == 0 ? p.ptrace : my_block + p.lane_off[s];
+    const uint64_t *in = s == 0 ? trace : my_block + p.lane_off[s];
     // ring positions: index & mask (the trace and the slab are not rings)
     const uint32_t K = 1u << p.lane_ring_log2;
     const uint32_t in_mask = (RING && s != 0) ? K - 1u : 0xffffffffu;
@@ -413,10 +419,12 @@ des_lane_kernel(const __grid_constant__ DesParams p)
             // are fetched here, so that the load runs under the examine step
             const bool h_valid = (vmask & 4u) != 0u;
             const uint32_t h_sl = (it + 1u) & (kStage - 1);
-            const uint32_t h_qid = (uint32_t)wm.stage_e[h_sl][lane] & (uint32_t)qmask;   // unused unless h_valid
+            const uint64_t h_low = wm.stage_e[h_sl][lane] & qmask;       // unused unless h_valid
+            const uint32_t h_qid = (uint32_t)h_low & imask;
             const uint64_t h_base = wm.stage_b[h_sl][lane];
             uint32_t h_bits = 0;
-            if (BRANCHY && h_valid && bit >= 0 && IL_IN_RANGE(h_qid, p.n, p.status)) h_bits = p.bits[h_qid];
+            if (BRANCHY && rb > 0) h_bits = (uint32_t)(h_low >> qi);
+            else if (BRANCHY && h_valid && bit >= 0 && IL_IN_RANGE(h_qid, p.n, p.status)) h_bits = p.bits[h_qid];
             // feasibility only: the record that left in the previous iteration is tested now, its query's
             // arrival record having had an iteration to come in; the arrival record of a query that may
             // leave in this iteration is requested here
@@ -427,7 +435,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
             // (loaded straight into the register that is carried to the next iteration: nothing in this
             // iteration waits for it)
             if (FEAS && h_valid && (da < 0 || (db < 0 && bit >= 0)) && IL_IN_RANGE(h_qid, p.n, p.status))
-                late_arr = __ldg(p.ptrace + h_qid);
+                late_arr = __ldg(trace + h_qid);
             // likewise the next batch to hand on, if the one in hand is used up (a batch handed over in
             // this iteration is picked up in the next), and the table entry a close would need
             const bool f_valid = e_left == 0 && epos != lpos;
@@ -493,14 +501,14 @@ des_lane_kernel(const __grid_constant__ DesParams p)
 
             // ---- hand on the record picked up at the top of the iteration
             if (FORK) {
-                const uint64_t out = h_base | h_qid;
+                const uint64_t out = h_base | h_low;
                 const bool go_a = da >= 0 && (cbit_a < 0 || ((h_bits >> cbit_a) & 1u) == cval_a);
                 const bool go_b = db >= 0 && (cbit_b < 0 || ((h_bits >> cbit_b) & 1u) == cval_b);
                 if (h_valid) {
                     if (go_a && IL_IN_RANGE(tail_a, size_a, p.status)) out_a[tail_a] = out;
                     if (go_b && IL_IN_RANGE(tail_b, size_b, p.status)) out_b[tail_b] = out;
                     // this copy leaves: the query's slab entry keeps the latest of its copies
-                    if (!go_a && !go_b && IL_IN_RANGE(h_qid, p.n, p.status)) atomicMax(slab_row + h_qid, out);
+                    if (!go_a && !go_b && IL_IN_RANGE(h_qid, p.n, p.status)) atomicMax(slab_row + h_qid, (h_base >> rb) | h_qid);
                 }
                 tail_a += (h_valid && go_a) ? 1u : 0u;
                 tail_b += (h_valid && go_b) ? 1u : 0u;
@@ -508,10 +516,11 @@ des_lane_kernel(const __grid_constant__ DesParams p)
             } else if (BRANCHY) {
                 // under predicates: with lanes on both sides of a branch point in one warp this measured
                 // 10 % faster than a branch around the block; without routing the branch is the faster form
-                const uint64_t out = h_base | h_qid;
                 const bool to_b = bit >= 0 && ((h_bits >> bit) & 1u);
+                const bool leaves = to_b ? db < 0 : da < 0;
+                // (slab records are plain (finish, query) records whatever the streams carry)
+                const uint64_t out = leaves ? ((h_base >> rb) | h_qid) : (h_base | h_low);
                 if (FEAS) {
-                    const bool leaves = to_b ? db < 0 : da < 0;
                     if (h_valid && leaves) {
                         late_valid = true; late_fin = h_base;
                     } else if (h_valid) {

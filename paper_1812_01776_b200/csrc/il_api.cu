@@ -41,6 +41,8 @@ struct il_estimator {
 
     int64_t *d_arrival = nullptr;
     uint64_t *d_ptrace = nullptr;      // packed root stream
+    uint64_t *d_ptrace_b = nullptr;    // the same with the branch bits inside each record (lane kernel)
+    int rec_bits = 0;                  // branch bits a record of d_ptrace_b carries (0: there is none)
     bool can_pack = false;             // every reachable time fits a packed record
     bool fork = false;                 // fan-out: one query can enter two children of a stage
     bool join = false;                 // some stage has two incoming edges (implies fork: copies of a query exist)
@@ -349,7 +351,7 @@ void configure_lane_rings(il_estimator *e)
 
 void free_device(il_estimator *e)
 {
-    cudaFree(e->d_arrival); cudaFree(e->d_ptrace); cudaFree(e->d_bits); cudaFree(e->d_lat);
+    cudaFree(e->d_arrival); cudaFree(e->d_ptrace); cudaFree(e->d_ptrace_b); cudaFree(e->d_bits); cudaFree(e->d_lat);
     cudaFree(e->d_counters); cudaFree(e->d_status); cudaFree(e->d_maxrep);
     cudaFree(e->own_ws); cudaFree(e->d_cfg); cudaFree(e->d_out);
     if (e->h_counters) cudaFreeHost(e->h_counters);
@@ -981,6 +983,20 @@ int il_estimator_create_dag(const il_profiles *pr, const il_join_edges *jn, cons
             packed[(size_t)i] = ((uint64_t)tr->arrival_us[i] << qbits) | (uint64_t)i;
         IL_CUDA_E(cudaMalloc(&e->d_ptrace, (size_t)n_padded * 8));
         IL_CUDA_E(cudaMemcpy(e->d_ptrace, packed.data(), (size_t)n_padded * 8, cudaMemcpyHostToDevice));
+        // Branch bits inside the records, where the time range leaves room for them: a stage of the lane
+        // kernel then routes a query by the record it hands on instead of looking its bits up.
+        int nb = 0;
+        for (int s = 0; s < pr->n_stages; s++)
+            if (pr->cond_bit[s] >= 0) nb = std::max(nb, (int)pr->cond_bit[s] + 1);
+        if (nb > 0 && tr->branch_bits && !e->join &&
+            tr->arrival_us[n - 1] + worst < (INT64_C(1) << (63 - qbits - nb))) {
+            for (int64_t i = 0; i < n; i++)
+                packed[(size_t)i] = ((uint64_t)tr->arrival_us[i] << (qbits + nb)) |
+                                    ((uint64_t)(tr->branch_bits[i] & ((1u << nb) - 1u)) << qbits) | (uint64_t)i;
+            IL_CUDA_E(cudaMalloc(&e->d_ptrace_b, (size_t)n_padded * 8));
+            IL_CUDA_E(cudaMemcpy(e->d_ptrace_b, packed.data(), (size_t)n_padded * 8, cudaMemcpyHostToDevice));
+            e->rec_bits = nb;
+        }
     }
     IL_CUDA_E(cudaMalloc(&e->d_lat, e->smem));
     IL_CUDA_E(cudaMalloc(&e->d_counters, kCounters * sizeof(unsigned long long)));
@@ -994,6 +1010,7 @@ int il_estimator_create_dag(const il_profiles *pr, const il_join_edges *jn, cons
     IL_CUDA_E(cudaMemcpy(e->d_lat, pr->latency_us, e->smem, cudaMemcpyHostToDevice));
 #undef IL_CUDA_E
     bp.arrival = e->d_arrival; bp.bits = e->d_bits; bp.lat = e->d_lat; bp.ptrace = e->d_ptrace;
+    bp.ptrace_b = e->d_ptrace_b; bp.rec_bits = e->rec_bits;
     bp.counters = e->d_counters; bp.status = e->d_status;
 
     e->ctas_per_sm_wide = des_max_ctas_per_sm(e->smem);
@@ -1057,6 +1074,11 @@ int il_set_test_knob(il_estimator *e, int knob, int64_t value)
     if (knob == IL_KNOB_LANE_CTAS) {
         if (value < 0 || value > 16) return IL_ERR_INVALID_ARG;
         e->lane_ctas_knob = (int)value;
+        return IL_OK;
+    }
+    if (knob == IL_KNOB_BITS_IN_RECORDS) {
+        if (value != 0 && value != 1) return IL_ERR_INVALID_ARG;
+        e->base.rec_bits = (value == 1 && e->d_ptrace_b) ? e->rec_bits : 0;
         return IL_OK;
     }
     if (knob == IL_KNOB_ITER_LIMIT) {
@@ -1358,7 +1380,7 @@ int il_feasible_device(il_estimator *e, const il_stage_config *d_configs, int64_
     p.out_feasible = d_out_feasible;
     // latency > objective is tested on time fields shifted by qbits: keep the objective in that range
     // (latencies are at least 1 and every reachable time is below 2^(63 - qbits))
-    p.slo_us = std::min<int64_t>(std::max<int64_t>(slo_us, 0), INT64_C(1) << (62 - p.qbits));
+    p.slo_us = std::min<int64_t>(std::max<int64_t>(slo_us, 0), INT64_C(1) << (62 - p.qbits - p.rec_bits));
     p.miss_allow = (uint32_t)(e->n - (99 * e->n + 99) / 100);
     if (e->lane_wrap) IL_CUDA(cudaMemsetAsync(p.ovf, 0, (size_t)n_cand, st));
     const int64_t groups = (n_cand + e->cpw - 1) / e->cpw;

@@ -28,6 +28,11 @@ struct DesParams {
     const uint8_t *bits;          // [n]
     const int32_t *lat;           // [S][H][Bmax]
     const uint64_t *ptrace;       // [n] packed root stream (arrival << qbits) | index; packed kernel only
+    // Lane kernel, pipelines with branch points: when rec_bits > 0 a stream record also carries the
+    // query's branch bits, (time << (qbits + rec_bits)) | (bits << qbits) | query, and ptrace_b is the
+    // trace in that form, so no stage looks the bits up.  Slab records keep the plain form.
+    const uint64_t *ptrace_b;
+    int32_t rec_bits;
     int32_t qbits;                // bits of a packed record that hold the query index
     int32_t S, H, Bmax;
     int32_t n;                    // queries

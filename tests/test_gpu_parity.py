@@ -177,6 +177,32 @@ def test_configs_reduced(il, oracle, cid, n, C, variant):
     check(il, oracle, workloads.make(cid, n_queries=n, n_candidates=C), host=False, variant=variant)
 
 
+@pytest.mark.parametrize("in_records", [0, 1])
+@pytest.mark.parametrize("case", ["w3", "w5", "tree_rings", "fan_out", "feasible"])
+def test_branch_bits_in_records_or_looked_up(il, oracle, case, in_records):
+    """Pipelines with branch points on the lane kernel: the stream records carry the queries' branch
+    bits (the default where the time range leaves room) or every stage looks them up by query index.
+    Same integers either way: estimate, stream rings, fan-out, feasibility-only."""
+    knobs = {5: in_records}
+    if case == "w3":
+        check(il, oracle, workloads.make(3, n_queries=6001, n_candidates=200), host=False, variant=3, knobs=knobs)
+    elif case == "w5":
+        check(il, oracle, workloads.make(5, n_queries=4097, n_candidates=260), host=True, variant=3, knobs=knobs)
+    elif case == "tree_rings":
+        w = workloads.random_small(7, S=6, H=3, Bmax=33, n=959, C=40, max_replicas=8, tree=True, qps=400.0, cv=3.0,
+                                   lat_lo=1, lat_hi=20000, equal_stamp_every=3)
+        check(il, oracle, w, host=False, variant=3, knobs={1: 8, **knobs})
+    elif case == "fan_out":
+        check(il, oracle, workloads.fan_out_small(11, n=1500, C=48, max_replicas=8, Bmax=16), host=False, knobs=knobs)
+    else:
+        w = workloads.make(3, n_queries=6001, n_candidates=200)
+        exp = oracle.estimate_workload(w)[0]
+        with il.Estimator.from_workload(w) as est:
+            est.set_test_knob(5, in_records)
+            for slo in (w.slo_us, int(np.median(exp))):
+                assert np.array_equal(est.feasible(w.configs, slo), exp <= slo)
+
+
 def test_times_too_large_to_pack_fall_back_to_wide_kernel(il, oracle):
     """Arrival stamps near 2^58 leave no room for the query index in a 64-bit
     record: the library must pick the kernel with separate time and query

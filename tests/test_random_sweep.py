@@ -1,7 +1,7 @@
 """Randomised differential sweep: a few hundred seeded draws over everything that can vary -- topology (chains,
 trees, fan-out, joins), table sizes, replica limits, trace lengths from 1, tiny service times with runs of equal
 stamps, duplicate candidates, objectives at both extremes, every kernel variant, short stream rings, every setting
-of prefix sharing, host and device entry points -- each compared with the oracle on P99, misses, feasibility and
+of prefix sharing, branch bits inside the stream records or looked up, host and device entry points -- each compared with the oracle on P99, misses, feasibility and
 (for a quarter of them) the per-query latencies.  A sweep of 18,655 such draws (seeds from 5001) ran clean on a
 B200 when this file was written; the cases here are the first few hundred of the same generator."""
 import numpy as np
@@ -39,7 +39,7 @@ def draw(seed):
     w.slo_us = int(rng.choice([w.slo_us, 1, 10**9, int(np.median(w.latency_us)) * w.n_stages]))
     knobs = dict(variant=int(rng.integers(0, 5)), ring=int(rng.choice([0, 0, 6, 7, 9])),
                  share=int(rng.choice([0, 1, 2, 3])), host=bool(rng.integers(0, 2)),
-                 per_query=bool(rng.integers(0, 4) == 0))
+                 per_query=bool(rng.integers(0, 4) == 0), bits_in_records=seed % 2)
     return w, knobs
 
 
@@ -55,6 +55,7 @@ def test_random_sweep(oracle, block):
             if k["ring"]:
                 est.set_test_knob(1, k["ring"])
             est.set_test_knob(3, k["share"])
+            est.set_test_knob(5, k["bits_in_records"])
             if k["host"]:
                 p99, miss = est.estimate(w.configs, w.slo_us)
             else:
