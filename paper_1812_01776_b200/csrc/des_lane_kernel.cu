@@ -269,8 +269,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
     uint32_t low_pub = 0, low_new = 0, e_first = 0;
     bool low_pending = false, aborted = false;
     // feasibility only: a leaving record waits one iteration for the arrival time of its query
-    uint64_t late_fin = 0, late_arr = 0;
-    bool late_valid = false;
+    uint64_t late_fin = 0, late_arr = 0;     // late_fin == 0: no record is waiting (finish times are at least 1)
     uint32_t miss_local = 0;     // misses seen by this lane since it last added them to the group's count
     uint32_t av = 0;             // mailbox word this iteration works with: the one read an iteration ago
     int par = 0;                 // mailbox buffer this iteration publishes into; it reads the other one
@@ -405,7 +404,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                     lim_b = (RING && lane_b >= 0) ? K : 0xffffffffu;
                     low_pub = 0; low_new = 0; e_first = 0;
                     low_pending = false; aborted = false;
-                    late_valid = false;
+                    late_fin = 0;
                     miss_local = 0;
                     av = avail0;
                 }
@@ -428,14 +427,16 @@ des_lane_kernel(const __grid_constant__ DesParams p)
             // feasibility only: the record that left in the previous iteration is tested now, its query's
             // arrival record having had an iteration to come in; the arrival record of a query that may
             // leave in this iteration is requested here
-            if (FEAS) {      // counted in a register; the group's shared count is brought up to date every eighth iteration
-                miss_local += (late_valid && late_fin > (late_arr & ~qmask) + slo_q) ? 1u : 0u;
-                late_valid = false;
+            // (finish << q has no low bits, so finish > arrival + objective holds for the time fields iff it
+            // holds with the arrival record's low bits left in; counted in a register, the group's shared
+            // count is brought up to date every eighth iteration)
+            if (FEAS) miss_local += (late_fin > late_arr + slo_q) ? 1u : 0u;
+            // (every lane loads, lanes that hand nothing to the outside the trace's first record: no branch;
+            // straight into the register that is carried to the next iteration, so nothing here waits for it)
+            if (FEAS) {
+                const bool may_leave = h_valid && (da < 0 || (db < 0 && bit >= 0)) && IL_IN_RANGE(h_qid, p.n, p.status);
+                late_arr = __ldg(trace + (may_leave ? h_qid : 0u));
             }
-            // (loaded straight into the register that is carried to the next iteration: nothing in this
-            // iteration waits for it)
-            if (FEAS && h_valid && (da < 0 || (db < 0 && bit >= 0)) && IL_IN_RANGE(h_qid, p.n, p.status))
-                late_arr = __ldg(trace + h_qid);
             // likewise the next batch to hand on, if the one in hand is used up (a batch handed over in
             // this iteration is picked up in the next), and the table entry a close would need
             const bool f_valid = e_left == 0 && epos != lpos;
@@ -520,28 +521,20 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                 const bool leaves = to_b ? db < 0 : da < 0;
                 // (slab records are plain (finish, query) records whatever the streams carry)
                 const uint64_t out = leaves ? ((h_base >> rb) | h_qid) : (h_base | h_low);
-                if (FEAS) {
-                    if (h_valid && leaves) {
-                        late_valid = true; late_fin = h_base;
-                    } else if (h_valid) {
-                        uint64_t *dst = to_b ? out_b + (tail_b & mask_b) : out_a + (tail_a & mask_a);
-                        if (IL_IN_RANGE(to_b ? (tail_b & mask_b) : (tail_a & mask_a), to_b ? size_b : size_a, p.status))
-                            *dst = out;
-                    }
-                } else {
-                    uint64_t *dst = to_b ? out_b + (tail_b & mask_b) : out_a + (tail_a & mask_a);
-                    if (h_valid && IL_IN_RANGE(to_b ? (tail_b & mask_b) : (tail_a & mask_a), to_b ? size_b : size_a, p.status))
-                        *dst = out;
-                }
+                uint64_t *dst = to_b ? out_b + (tail_b & mask_b) : out_a + (tail_a & mask_a);
+                if (FEAS) late_fin = (h_valid && leaves) ? h_base : 0ull;
+                if (h_valid && !(FEAS && leaves) &&
+                    IL_IN_RANGE(to_b ? (tail_b & mask_b) : (tail_a & mask_a), to_b ? size_b : size_a, p.status))
+                    *dst = out;
                 tail_b += (h_valid && to_b) ? 1u : 0u;
                 tail_a += (h_valid && !to_b) ? 1u : 0u;
-            } else if (h_valid) {
-                if (FEAS && da < 0) {
-                    late_valid = true; late_fin = h_base;
-                } else if (IL_IN_RANGE(tail_a & mask_a, size_a, p.status)) {
-                    out_a[tail_a & mask_a] = h_base | h_qid;
+            } else {
+                if (FEAS) late_fin = (h_valid && da < 0) ? h_base : 0ull;
+                if (h_valid) {
+                    if (!(FEAS && da < 0) && IL_IN_RANGE(tail_a & mask_a, size_a, p.status))
+                        out_a[tail_a & mask_a] = h_base | h_qid;
+                    tail_a++;
                 }
-                tail_a++;
             }
             // ---- request the next record to hand on
             if (f_valid) {
@@ -568,7 +561,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                     cp_async8(&wm.stage_x[fx & (kStage - 1)][lane], in + (fx & in_mask));
                 fx++;
             }
-            done = end && b == 0 && epos == tpos && e_left == 0 && vmask == 0u && !(FEAS && late_valid);
+            done = end && b == 0 && epos == tpos && e_left == 0 && vmask == 0u && !(FEAS && late_fin != 0ull);
             if (--guard == 0) {
                 if (guard_hi == 0) { atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT); atomicOr(&p.counters[5], 1ull); done = true; }
                 else { guard_hi--; }      // guard wraps to 2^32 - 1 on the next decrement
