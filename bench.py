@@ -49,14 +49,14 @@ NCU_CAPTURES = {
     # whole streams (workloads 1, 2, 3, 5): 16,384 candidates x 8,000 queries of workload 2, all warp slots busy
     "des_lane_kernel": {
         "source": "paper_1812_01776_b200/csrc/des_lane_kernel.cu",
-        "source_sha256": "3fd986842724cfe7d9dd5a516c77ae3d2824430a26751e5975105068478747c6",
-        "dram_bytes_per_query_event": 8.86, "warp_inst_per_query_event": 6.60,
+        "source_sha256": "098d990650420ecbcf1ad1f20b385efe22a7b3639a4e478e5be71604a087ef6b",
+        "dram_bytes_per_query_event": 8.85, "warp_inst_per_query_event": 6.89,
         "summary": "profiles/des_lane_kernel_config2.md"},
     # stream rings (workload 4): 3,552 candidates x 20,000 queries of workload 4, all warp slots busy
     "des_lane_kernel:rings": {
         "source": "paper_1812_01776_b200/csrc/des_lane_kernel.cu",
-        "source_sha256": "3fd986842724cfe7d9dd5a516c77ae3d2824430a26751e5975105068478747c6",
-        "dram_bytes_per_query_event": 9.04, "warp_inst_per_query_event": 6.76,
+        "source_sha256": "098d990650420ecbcf1ad1f20b385efe22a7b3639a4e478e5be71604a087ef6b",
+        "dram_bytes_per_query_event": 9.03, "warp_inst_per_query_event": 7.68,
         "summary": "profiles/des_lane_kernel_config4_rings.md"},
     "des_packed_kernel": {
         "source": "paper_1812_01776_b200/csrc/des_packed_kernel.cu",

@@ -317,7 +317,7 @@ IL_API int il_traffic_envelope(il_estimator *est, const int64_t *window_us, int3
  *
  * Limit: the whole batch is evaluated in one pass, with at most 32 warps
  * resident, and must fit the array:
- *     256 + r * slot * min(32, n rounded up to 4) + (8 * n_queries' + 12) * n
+ *     256 + r * slot * min(32, n rounded up to 4) + (8 * n_queries' + 4) * n
  *         <= IL_STATIC_SCRATCH_BYTES
  * where n_queries' is n_queries rounded up to 32, slot is the number of
  * stream elements one warp keeps between stages (for a linear pipeline about

@@ -152,7 +152,7 @@ des_kernel(const __grid_constant__ DesParams p)
                                         my_cfg.max_batch > p.Bmax || my_cfg.replicas < 1 ||
                                         my_cfg.replicas > IL_MAX_REPLICAS);
         if (__any_sync(full, bad)) {
-            if (lane == 0) { atomicCAS(p.status, 0, IL_ERR_BAD_CONFIG); p.lat_or[c] = 0; }
+            if (lane == 0) atomicCAS(p.status, 0, IL_ERR_BAD_CONFIG);
             for (int i = lane; i < p.n; i += 32) p.slab[c * p.slab_stride + i] = 0;
             continue;
         }
@@ -163,7 +163,6 @@ des_kernel(const __grid_constant__ DesParams p)
             __syncwarp();
         }
         int32_t exits = 0;
-        uint64_t lat_or = 0;
         unsigned long long cand_batches = 0;
         bool over = false;      // more batches than the iteration bound allows: the candidate is given up
 
@@ -227,7 +226,6 @@ des_kernel(const __grid_constant__ DesParams p)
                         if (left && IL_IN_RANGE(q, p.n, p.status)) {
                             const int64_t l = tfin - p.arrival[q];
                             if (l > slab[q]) slab[q] = l;
-                            lat_or |= (uint64_t)l;
                         }
                         rt.a_tail += __popc(fa); rt.b_tail += __popc(fb);
                         exits += __popc(fl);
@@ -244,7 +242,6 @@ des_kernel(const __grid_constant__ DesParams p)
                             if (mine && IL_IN_RANGE(q, p.n, p.status)) {
                                 const int64_t l = tfin - p.arrival[q];
                                 slab[q] = l;   // trace order: the slab doubles as the per-query answer
-                                lat_or |= (uint64_t)l;
                             }
                             exits += __popc(ma);
                         } else {
@@ -261,7 +258,6 @@ des_kernel(const __grid_constant__ DesParams p)
                             if (mine && IL_IN_RANGE(q, p.n, p.status)) {
                                 const int64_t l = tfin - p.arrival[q];
                                 slab[q] = l;   // trace order: the slab doubles as the per-query answer
-                                lat_or |= (uint64_t)l;
                             }
                             exits += __popc(mb_);
                         } else {
@@ -341,11 +337,7 @@ des_kernel(const __grid_constant__ DesParams p)
             }
         }
 
-        // OR-reduce the latencies' bit pattern (tells the select kernel which digits matter)
-        const uint32_t lo = __reduce_or_sync(full, (uint32_t)lat_or);
-        const uint32_t hi = __reduce_or_sync(full, (uint32_t)(lat_or >> 32));
         if (lane == 0) {
-            p.lat_or[c] = ((uint64_t)hi << 32) | lo;
             if (!over && (int64_t)exits != (p.fork ? p.total_leaving : (int64_t)p.n)) atomicCAS(p.status, 0, IL_ERR_ITER_LIMIT);
         }
     }

@@ -117,11 +117,10 @@ struct WarpMem {
     // One copy per lane, so that lanes with different rows or batch sizes never meet in a bank.
     uint32_t (*lat)[32];         // [Bmax]
     // Staging rings filled by cp.async, [position][lane]: the next records of the lane's arrival stream
-    // (position = record index mod kStage), and the records it is handing on with the finish << q of
-    // their batch (position = iteration mod kStage)
+    // (position = record index mod kStage), and the records it is handing on (position = iteration
+    // mod kStage; the finish << q of their batch waits in a three-deep delay line of registers)
     uint64_t (*stage_x)[32];     // [kStage]
     uint64_t (*stage_e)[32];
-    uint64_t (*stage_b)[32];
     // Mailboxes, double-buffered by iteration parity: what iteration k publishes in buffer k & 1 is read
     // in iteration k + 1, while iteration k + 1 publishes into the other buffer; one warp barrier per
     // iteration then separates every write of a word from the reads of its previous value.
@@ -137,7 +136,7 @@ struct WarpMem {
 
 __host__ __device__ inline size_t warp_mem_bytes(int kr, int Bmax)
 {
-    return (size_t)kr * 32 * 12 + (size_t)3 * kStage * 32 * 8 + (size_t)(2 + 1 + 1) * 32 * 4 + (size_t)Bmax * 32 * 4;
+    return (size_t)kr * 32 * 12 + (size_t)2 * kStage * 32 * 8 + (size_t)(2 + 1 + 1) * 32 * 4 + (size_t)Bmax * 32 * 4;
 }
 
 __device__ __forceinline__ WarpMem warp_mem_at(unsigned char *base, int kr, int Bmax)
@@ -146,7 +145,6 @@ __device__ __forceinline__ WarpMem warp_mem_at(unsigned char *base, int kr, int 
     wm.key = reinterpret_cast<uint64_t (*)[32]>(base);          base += (size_t)kr * 256;
     wm.stage_x = reinterpret_cast<uint64_t (*)[32]>(base);      base += (size_t)kStage * 256;
     wm.stage_e = reinterpret_cast<uint64_t (*)[32]>(base);      base += (size_t)kStage * 256;
-    wm.stage_b = reinterpret_cast<uint64_t (*)[32]>(base);      base += (size_t)kStage * 256;
     wm.cnt = reinterpret_cast<uint32_t (*)[32]>(base);          base += (size_t)kr * 128;
     wm.lat = reinterpret_cast<uint32_t (*)[32]>(base);          base += (size_t)Bmax * 128;
     wm.avail = reinterpret_cast<uint32_t (*)[32]>(base);        base += 256;
@@ -257,6 +255,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
     uint32_t e_idx = 0;          // its next record in the arrival stream
     uint32_t e_left = 0;         // records of it not yet fetched
     uint32_t vmask = 0;          // bit k: the record fetched k + 1 iterations ago is on its way out
+    uint64_t eb1 = 0, eb2 = 0, eb3 = 0;   // finish << q of the batches of those records, a delay line in registers
     // fetch cursor of the arrival stream: records below fx have been requested; fx1..fx3 are its
     // values at the end of the previous three iterations, so records below fx3 have arrived
     uint32_t fx = 0, fx1 = 0, fx2 = 0, fx3 = 0;
@@ -420,7 +419,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
             const uint32_t h_sl = (it + 1u) & (kStage - 1);
             const uint64_t h_low = wm.stage_e[h_sl][lane] & qmask;       // unused unless h_valid
             const uint32_t h_qid = (uint32_t)h_low & imask;
-            const uint64_t h_base = wm.stage_b[h_sl][lane];
+            const uint64_t h_base = eb3;     // finish << q of the batch of the record requested three iterations ago
             uint32_t h_bits = 0;
             if (BRANCHY && rb > 0) h_bits = (uint32_t)(h_low >> qi);
             else if (BRANCHY && h_valid && bit >= 0 && IL_IN_RANGE(h_qid, p.n, p.status)) h_bits = p.bits[h_qid];
@@ -545,11 +544,12 @@ des_lane_kernel(const __grid_constant__ DesParams p)
                 epos++;
             }
             vmask = (vmask << 1) & 7u;
+            eb3 = eb2; eb2 = eb1;
             if (e_left > 0 && can_emit) {
                 const uint32_t sl = it & (kStage - 1);
                 if (IL_IN_RANGE(e_idx & in_mask, in_size, p.status))
                     cp_async8(&wm.stage_e[sl][lane], in + (e_idx & in_mask));
-                wm.stage_b[sl][lane] = e_base;
+                eb1 = e_base;
                 e_idx++; e_left--;
                 vmask |= 1u;
             }

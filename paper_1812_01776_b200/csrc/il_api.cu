@@ -96,7 +96,7 @@ struct Plan {
     int64_t chunk = 0;       // candidates per (simulate, select) pair
     int64_t fb_slots = 0;    // lane kernel with wrapping rings: warp slots of the kernel that takes over
                              // the candidates given up on ring overflow
-    size_t off_time = 0, off_qid = 0, off_slab = 0, off_or = 0, off_order = 0, off_ovf = 0, off_fb = 0, total = 0;
+    size_t off_time = 0, off_qid = 0, off_slab = 0, off_order = 0, off_ovf = 0, off_fb = 0, total = 0;
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -173,7 +173,6 @@ size_t layout(const il_estimator *e, Plan &pl)
     pl.off_time = off; off = align_up(off + (size_t)pl.slots * slot_time_bytes(e), 256);
     pl.off_qid = off;  off = align_up(off + (size_t)pl.slots * slot_qid_bytes(e), 256);
     pl.off_slab = off; off = align_up(off + (size_t)pl.chunk * e->n_pad * 8, 256);
-    pl.off_or = off;   off = align_up(off + (size_t)pl.chunk * 8, 256);
     pl.off_order = off; off = align_up(off + (size_t)pl.chunk * 4, 256);
     pl.off_ovf = off;  off = align_up(off + (size_t)pl.chunk, 256);
     pl.off_fb = off;   off = align_up(off + (size_t)pl.fb_slots * fb_slot_bytes(e), 256);
@@ -447,7 +446,6 @@ static DesParams chunk_params(const il_estimator *e, const Plan &pl, char *ws, c
     p.lane_ws = reinterpret_cast<uint64_t *>(ws + pl.off_time);
     p.slab = reinterpret_cast<int64_t *>(ws + pl.off_slab);
     p.slab_stride = e->n_pad;
-    p.lat_or = reinterpret_cast<uint64_t *>(ws + pl.off_or);
     p.order = reinterpret_cast<int32_t *>(ws + pl.off_order);
     p.ovf = reinterpret_cast<uint8_t *>(ws + pl.off_ovf);
     p.iter_limit = e->iter_limit;

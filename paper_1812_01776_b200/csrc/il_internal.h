@@ -70,7 +70,6 @@ struct DesParams {
     int32_t *ws_qid;              // [slots][slot_elems]
     int64_t *slab;                // [n_cand][slab_stride] exit latencies
     int64_t slab_stride;          // n rounded up to 32
-    uint64_t *lat_or;             // [n_cand] OR of all latencies of the candidate (wide kernel)
     unsigned long long *counters; // [0] next candidate, [1] batches dispatched, [2] algorithmic ops
     int *status;                  // first error seen by any warp (0 = none)
     // lane-parallel kernel only (des_lane_kernel.cu)

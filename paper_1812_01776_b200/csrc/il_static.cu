@@ -45,7 +45,7 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // Enqueues the whole call; on a failing CUDA call records it and returns IL_ERR_CUDA.
 static int enqueue_static(const BoundView &v, unsigned char *base, const il_stage_config *d_configs,
                           int64_t n_cand, int64_t slo_us, int64_t *d_out_p99, int64_t *d_out_miss,
-                          int64_t slots, size_t off_time, size_t off_qid, size_t off_slab, size_t off_or,
+                          int64_t slots, size_t off_time, size_t off_qid, size_t off_slab,
                           size_t off_order, int *h_status)
 {
 #define IL_ST(call)                                                          \
@@ -65,7 +65,6 @@ static int enqueue_static(const BoundView &v, unsigned char *base, const il_stag
     p.ws_qid = reinterpret_cast<int32_t *>(base + off_qid);
     p.slab = reinterpret_cast<int64_t *>(base + off_slab);
     p.slab_stride = v.n_pad;
-    p.lat_or = reinterpret_cast<uint64_t *>(base + off_or);
     p.order = reinterpret_cast<int32_t *>(base + off_order);
     OrderParams op;
     op.configs = d_configs; op.n_cand = n_cand; op.lat = v.base.lat;
@@ -112,7 +111,6 @@ extern "C" int il_estimate_device_static(il_estimator *est, const il_stage_confi
     if ((size_t)n_cand > IL_STATIC_SCRATCH_BYTES / 8 || (size_t)v.n_pad > IL_STATIC_SCRATCH_BYTES / 8)
         return IL_ERR_TOO_LARGE;
     off = align_up(off + (size_t)n_cand * v.n_pad * 8, 256);
-    const size_t off_or = off;   off = align_up(off + (size_t)n_cand * 8, 256);
     const size_t off_order = off; off = align_up(off + (size_t)n_cand * 4, 256);
     if (off > IL_STATIC_SCRATCH_BYTES) return IL_ERR_TOO_LARGE;
 
@@ -127,7 +125,7 @@ extern "C" int il_estimate_device_static(il_estimator *est, const il_stage_confi
 
     int status = 0;
     int rc = enqueue_static(v, base, d_configs, n_cand, slo_us, d_out_p99, d_out_miss, slots, off_time,
-                            off_qid, off_slab, off_or, off_order, &status);
+                            off_qid, off_slab, off_order, &status);
     // whatever was enqueued (all of it, or the part before a failing call) is
     // waited for: nothing may still be writing the shared array or the caller's
     // outputs when the call returns
