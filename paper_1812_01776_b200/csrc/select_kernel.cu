@@ -17,7 +17,7 @@
 // into shared memory, in the space of the histogram, and the select ends there;
 // otherwise passes with plain 13-bit digits over the bin's offsets narrow it
 // until that holds or no bit is left (all latencies equal: two passes).  A
-// thread requests the records of its next round before it uses those of the
+// thread requests the records of its next turn before it uses those of the
 // current one (eight independent 8-byte loads in flight), which is what the row
 // passes need to run near memory speed.
 #include "il_internal.h"
@@ -28,7 +28,7 @@ namespace {
 
 constexpr int kSelBins = 8192;       // bins of a histogram pass
 constexpr int kSelCap = 4096;        // latencies the shared-memory list holds (the same 32 KB)
-// Records a thread requests per round (it has two rounds in flight) and resident CTAs per SM.  Measured on
+// Records a thread requests per turn (it has two turns in flight) and resident CTAs per SM.  Measured on
 // 50,000- to 1,000,000-record rows: 4 x 4 as here 0.68 / 40.4 / 50.2 ms on three workloads, 8 x 4 0.70 / 40.8 /
 // 52.4, 4 x 6 (40 registers) 0.81 / 62.2 / 67.0, 2 x 6 0.74 / 56.1 / 62.3, 8 x 3 0.92 / 49.8 / 60.6.
 constexpr int kSelUnroll = 4;
@@ -94,7 +94,7 @@ __device__ __forceinline__ void row_pass(const SelectParams &p, const uint64_t *
     const uint64_t width_m1 = e >= 64 ? ~0ull : ((1ull << e) - 1ull);
     uint64_t *list = reinterpret_cast<uint64_t *>(hist);
     const int n = p.n;
-    // software pipeline: the records of the next round are requested before this round's are used
+    // software pipeline: the records of the next turn are requested before this turn's are used
     uint64_t nx[kSelUnroll];
 #pragma unroll
     for (int u = 0; u < kSelUnroll; u++) {
