@@ -145,7 +145,7 @@ size_t slot_time_bytes(const il_estimator *e)
 }
 size_t slot_qid_bytes(const il_estimator *e) { return is_lane(e) ? 0 : (size_t)e->slot_elems * 4; }
 size_t slot_bytes(const il_estimator *e) { return slot_time_bytes(e) + slot_qid_bytes(e); }
-size_t cand_bytes(const il_estimator *e) { return (size_t)e->n_pad * 8 + 13; }
+size_t cand_bytes(const il_estimator *e) { return (size_t)e->n_pad * 8 + 5; }   // slab row, order entry, overflow mark
 bool lane_fallback(const il_estimator *e) { return is_lane(e) && e->lane_wrap; }
 size_t fb_slot_bytes(const il_estimator *e) { return (size_t)e->slot_elems * 8; }
 

@@ -214,6 +214,21 @@ def test_times_too_large_to_pack_fall_back_to_wide_kernel(il, oracle):
     assert np.array_equal(p99, exp[0]) and np.array_equal(miss, exp[1])
 
 
+@pytest.mark.parametrize("variant", [0, 4, 1], ids=["auto", "packed", "wide"])
+def test_recommended_workspace_holds_the_batch_in_one_chunk(il, oracle, variant):
+    """A workspace of the size the library recommends for a batch takes that batch in one pass: a second
+    chunk of a few left-over candidates would cost a whole further walk over the trace."""
+    import torch
+    w = workloads.make(2, n_queries=3000, n_candidates=700)
+    exp = oracle.estimate_workload(w)
+    with il.Estimator.from_workload(w) as est:
+        est.set_variant(variant)
+        est.reserve_workspace(w.n_candidates)
+        a, b = est.estimate_device(torch.from_numpy(w.configs).cuda(), w.slo_us)
+        assert est.stats()["chunks"] == 1
+        assert np.array_equal(a.cpu().numpy(), exp[0]) and np.array_equal(b.cpu().numpy(), exp[1])
+
+
 @pytest.mark.parametrize("variant", [4, 3], ids=["packed", "lanes"])
 def test_multi_chunk_small_workspace(il, oracle, variant):
     """A workspace that holds only a few candidates forces many chunks."""
