@@ -66,6 +66,7 @@ NCU_CAPTURES = {
 }
 LANE_CTAS = None         # --lane-ctas: resident CTAs per SM of the lane kernel, for side measurements
 RING_LOG2 = None         # --ring-log2: ring length of the lane kernel's streams, for side measurements
+BITS_LOOKUP = False      # --bits-lookup: stages look the branch bits up instead of finding them in the records
 METRIC = "candidate_configs_per_s"
 UNIT = "candidates/s"
 
@@ -287,6 +288,8 @@ def measure(il, torch, w, dev, stream, flush, steps, warmup, e2e_steps, variant,
         est.set_test_knob(1, RING_LOG2)
     if LANE_CTAS is not None:
         est.set_test_knob(4, LANE_CTAS)
+    if BITS_LOOKUP:
+        est.set_test_knob(5, 0)
     kernel = est.kernel_name()
     ws_bytes = est.reserve_workspace(n_cand)
     cfg_pinned = torch.from_numpy(cfg_host).pin_memory()
@@ -595,10 +598,14 @@ def main():
                     help="resident CTAs per SM of the lane kernel (side measurements; default 4)")
     ap.add_argument("--ring-log2", type=int, default=None,
                     help="largest stream ring of the lane kernel, log2 records (side measurements; default 13)")
+    ap.add_argument("--bits-lookup", action="store_true",
+                    help="lane kernel: stages look the queries' branch bits up by index instead of carrying them "
+                         "in the stream records (side measurements)")
     args = ap.parse_args()
-    global RING_LOG2, LANE_CTAS
+    global RING_LOG2, LANE_CTAS, BITS_LOOKUP
     RING_LOG2 = args.ring_log2
     LANE_CTAS = args.lane_ctas
+    BITS_LOOKUP = args.bits_lookup
     if args.impl == "reference":
         run_reference(args)
     else:

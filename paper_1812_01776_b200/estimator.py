@@ -27,7 +27,7 @@ IL_ERR_TOO_LARGE = -9
 IL_ERR_BOUNDS = -10
 IL_VARIANT_AUTO, IL_VARIANT_WIDE, IL_VARIANT_STAGED, IL_VARIANT_LANES, IL_VARIANT_PACKED = 0, 1, 2, 3, 4
 IL_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
-IL_KNOB_LANE_RING_LOG2, IL_KNOB_ITER_LIMIT, IL_KNOB_SHARE_PREFIXES, IL_KNOB_LANE_CTAS = 1, 2, 3, 4
+IL_KNOB_LANE_RING_LOG2, IL_KNOB_ITER_LIMIT, IL_KNOB_SHARE_PREFIXES, IL_KNOB_LANE_CTAS, IL_KNOB_BITS_IN_RECORDS = 1, 2, 3, 4, 5
 
 EXPORTS = ["il_estimator_create", "il_estimator_destroy", "il_estimate", "il_estimate_device",
            "il_set_stream", "il_workspace_bytes", "il_workspace_min_bytes", "il_set_workspace",
