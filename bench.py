@@ -58,6 +58,13 @@ NCU_CAPTURES = {
         "source_sha256": "098d990650420ecbcf1ad1f20b385efe22a7b3639a4e478e5be71604a087ef6b",
         "dram_bytes_per_query_event": 9.03, "warp_inst_per_query_event": 7.68,
         "summary": "profiles/des_lane_kernel_config4_rings.md"},
+    # pipelines with branch points (workloads 3, 5; a lane idles while its stage has no query): 5,920 candidates x
+    # 20,000 queries of workload 3, all warp slots busy
+    "des_lane_kernel:tree": {
+        "source": "paper_1812_01776_b200/csrc/des_lane_kernel.cu",
+        "source_sha256": "098d990650420ecbcf1ad1f20b385efe22a7b3639a4e478e5be71604a087ef6b",
+        "dram_bytes_per_query_event": 8.85, "warp_inst_per_query_event": 12.74,
+        "summary": "profiles/des_lane_kernel_config3_branch_bits.md"},
     "des_packed_kernel": {
         "source": "paper_1812_01776_b200/csrc/des_packed_kernel.cu",
         "source_sha256": "",       # not captured again since the kernel got its node-stage entry and checks
@@ -104,11 +111,11 @@ def reduce_sum(values, dist=None, device=None):
     return t.tolist()
 
 
-def ncu_capture(kernel: str, rings: bool = False):
+def ncu_capture(kernel: str, rings: bool = False, tree: bool = False):
     """The capture record of `kernel` if it still describes the source in the tree, else None."""
     import hashlib
     name = kernel.split("<")[0]
-    cap = NCU_CAPTURES.get(name + ":rings") if rings else None
+    cap = NCU_CAPTURES.get(name + ":rings") if rings else (NCU_CAPTURES.get(name + ":tree") if tree else None)
     cap = cap or NCU_CAPTURES.get(name)
     if not cap:
         return None
@@ -358,7 +365,7 @@ def measure(il, torch, w, dev, stream, flush, steps, warmup, e2e_steps, variant,
     stream_bytes = (events_per_cand - n) * 2 * rec_bytes * n_cand   # written once, read once
     # the lane kernel keeps its streams in rings when whole streams of all resident candidates pass 48 GiB
     rings = kernel == "des_lane_kernel" and (events_per_cand - n) * 8 * 148 * 8 * (32 // S) > 48 * 2**30
-    cap = None if shared else ncu_capture(kernel, rings)
+    cap = None if shared else ncu_capture(kernel, rings, tree=bool((w.cond_bit >= 0).any()))
     alu_peak = issue_rate * 32.0
     hbm_note = ("latency slab written once + every inter-stage stream record written once "
                 "and read once (the streams are this design's, not the method's)")
