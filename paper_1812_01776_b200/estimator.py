@@ -377,6 +377,10 @@ class Estimator:
         want = il_workspace_bytes(self._h, n_candidates)
         with torch.cuda.device(self.device):
             free_b, _ = torch.cuda.mem_get_info()
+            if max_bytes is None and want > int(free_b * 0.8):
+                # blocks torch keeps cached from earlier tensors count as used: hand them back first
+                torch.cuda.empty_cache()
+                free_b, _ = torch.cuda.mem_get_info()
             cap = int(free_b * 0.8) if max_bytes is None else int(max_bytes)
             nbytes = max(min(want, cap), il_workspace_min_bytes(self._h))
             if self._ws is None or self._ws.numel() < nbytes:
