@@ -49,21 +49,21 @@ NCU_CAPTURES = {
     # whole streams (workloads 1, 2, 3, 5): 16,384 candidates x 8,000 queries of workload 2, all warp slots busy
     "des_lane_kernel": {
         "source": "paper_1812_01776_b200/csrc/des_lane_kernel.cu",
-        "source_sha256": "098d990650420ecbcf1ad1f20b385efe22a7b3639a4e478e5be71604a087ef6b",
-        "dram_bytes_per_query_event": 8.85, "warp_inst_per_query_event": 6.89,
+        "source_sha256": "7ced5906c1a2907bed48cee1217576a44e88a55664f1015da071eca0aecef96a",
+        "dram_bytes_per_query_event": 8.84, "warp_inst_per_query_event": 6.89,
         "summary": "profiles/des_lane_kernel_config2.md"},
     # stream rings (workload 4): 3,552 candidates x 20,000 queries of workload 4, all warp slots busy
     "des_lane_kernel:rings": {
         "source": "paper_1812_01776_b200/csrc/des_lane_kernel.cu",
-        "source_sha256": "098d990650420ecbcf1ad1f20b385efe22a7b3639a4e478e5be71604a087ef6b",
-        "dram_bytes_per_query_event": 9.03, "warp_inst_per_query_event": 7.68,
+        "source_sha256": "7ced5906c1a2907bed48cee1217576a44e88a55664f1015da071eca0aecef96a",
+        "dram_bytes_per_query_event": 8.99, "warp_inst_per_query_event": 7.68,
         "summary": "profiles/des_lane_kernel_config4_rings.md"},
     # pipelines with branch points (workloads 3, 5; a lane idles while its stage has no query): 5,920 candidates x
     # 20,000 queries of workload 3, all warp slots busy
     "des_lane_kernel:tree": {
         "source": "paper_1812_01776_b200/csrc/des_lane_kernel.cu",
-        "source_sha256": "098d990650420ecbcf1ad1f20b385efe22a7b3639a4e478e5be71604a087ef6b",
-        "dram_bytes_per_query_event": 8.85, "warp_inst_per_query_event": 12.74,
+        "source_sha256": "7ced5906c1a2907bed48cee1217576a44e88a55664f1015da071eca0aecef96a",
+        "dram_bytes_per_query_event": 8.84, "warp_inst_per_query_event": 12.74,
         "summary": "profiles/des_lane_kernel_config3_branch_bits.md"},
     "des_packed_kernel": {
         "source": "paper_1812_01776_b200/csrc/des_packed_kernel.cu",

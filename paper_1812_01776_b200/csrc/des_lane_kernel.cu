@@ -112,7 +112,7 @@ struct WarpMem {
     // taken over, waiting to be handed on, in key order.  Positions [lpos, tpos): the slots in use,
     // sorted by key.
     uint64_t (*key)[32];         // [kr] (finish << q) | index of the batch's first arrival
-    uint32_t (*cnt)[32];         // [kr] batch size
+    uint8_t (*cnt)[32];          // [kr] batch size (at most IL_MAX_BATCH = 64)
     // The lane's row of the profile, [b - 1][lane]: time of a batch of b on the stage's hardware type.
     // One copy per lane, so that lanes with different rows or batch sizes never meet in a bank.
     uint32_t (*lat)[32];         // [Bmax]
@@ -136,7 +136,7 @@ struct WarpMem {
 
 __host__ __device__ inline size_t warp_mem_bytes(int kr, int Bmax)
 {
-    return (size_t)kr * 32 * 12 + (size_t)2 * kStage * 32 * 8 + (size_t)(2 + 1 + 1) * 32 * 4 + (size_t)Bmax * 32 * 4;
+    return (size_t)kr * 32 * 9 + (size_t)2 * kStage * 32 * 8 + (size_t)(2 + 1 + 1) * 32 * 4 + (size_t)Bmax * 32 * 4;
 }
 
 __device__ __forceinline__ WarpMem warp_mem_at(unsigned char *base, int kr, int Bmax)
@@ -145,7 +145,7 @@ __device__ __forceinline__ WarpMem warp_mem_at(unsigned char *base, int kr, int 
     wm.key = reinterpret_cast<uint64_t (*)[32]>(base);          base += (size_t)kr * 256;
     wm.stage_x = reinterpret_cast<uint64_t (*)[32]>(base);      base += (size_t)kStage * 256;
     wm.stage_e = reinterpret_cast<uint64_t (*)[32]>(base);      base += (size_t)kStage * 256;
-    wm.cnt = reinterpret_cast<uint32_t (*)[32]>(base);          base += (size_t)kr * 128;
+    wm.cnt = reinterpret_cast<uint8_t (*)[32]>(base);           base += (size_t)kr * 32;
     wm.lat = reinterpret_cast<uint32_t (*)[32]>(base);          base += (size_t)Bmax * 128;
     wm.avail = reinterpret_cast<uint32_t (*)[32]>(base);        base += 256;
     wm.freed = reinterpret_cast<uint32_t *>(base);              base += 128;
@@ -478,7 +478,7 @@ des_lane_kernel(const __grid_constant__ DesParams p)
             }
             if (close) {
                 wm.key[pos & rmask][lane] = key;
-                wm.cnt[pos & rmask][lane] = (uint32_t)b;
+                wm.cnt[pos & rmask][lane] = (uint8_t)b;
             }
             ktail = (close && !sorted_insert) ? key : ktail;
             const bool at_front = close && pos == lpos;
